@@ -1,0 +1,209 @@
+/*
+ * mvla_prune.h -- C ABI of the B200 (sm_100a) prune step for multi-visual-modal
+ * VLA inference: tri-stage, modality-salience-aware token pruning
+ * ("2D or 3D: Who Governs Salience in VLA Models?", Alg. 1).
+ *
+ * One prune point inside the LLM prefill does, per sample:
+ *   salience  : attention of the instruction (text) queries over every 2D image
+ *               token and 3D point token (Sec. 3.2.1), reduced to one score per token;
+ *   carry-over: the scores and the four modality indicators are smoothed across
+ *               action steps (Alg. 1 step 1; Eqs. 8, 9);
+ *   budget    : the keep budget is split between 2D and 3D by the stage rules
+ *               (Sec. 4.1 dual threshold, Sec. 4.2 target-object rule, Sec. 4.4 fusion);
+ *   select    : the top-k tokens per modality, ties to the lower index (Eq. 10 as an index list);
+ *   compact   : surviving hidden / K / V rows are gathered into a dense layout (Sec. 4.4).
+ *
+ * Conventions
+ *   - Every function returns an int32 status (0 = MVLA_OK, negative = error) and never throws.
+ *   - "device pointer" = memory of the context's CUDA device; "host pointer" = ordinary memory.
+ *   - No function synchronises the stream; work is enqueued on `stream` (a cudaStream_t passed
+ *     as void*, NULL = the legacy default stream).  Host arrays (`samples`) are consumed before
+ *     the call returns.  The library keeps no caller pointer beyond the enqueued work.
+ *   - Input tensors are token-major and packed ragged: Q, K, V are [rows, n_heads, head_dim],
+ *     hidden is [rows, d_model], rows contiguous, dtype as given at create.  A sample owns the
+ *     rows [seq_off, seq_off + n_txt + n_2d + n_3d) split in three contiguous segments.
+ *     Base pointers must be 16-byte aligned.
+ *   - Visual tokens of a sample are numbered 2D first, then 3D ("visual order").  Arrays
+ *     `attn`, `l1`, `ahat` hold sum(n_2d + n_3d) floats, samples back to back in batch order.
+ *   - Inputs must be finite.
+ *   - A context is not thread-safe; use one per host thread / stream.
+ */
+#ifndef MVLA_PRUNE_H
+#define MVLA_PRUNE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes */
+#define MVLA_OK                 0
+#define MVLA_ERR_INVALID_ARG   (-1)  /* null / misaligned pointer, bad segment, bad ratio, bad flag */
+#define MVLA_ERR_UNSUPPORTED   (-2)  /* shape or dtype outside what was built (see mvla_prune_create) */
+#define MVLA_ERR_OOM           (-3)  /* workspace allocation failed */
+#define MVLA_ERR_CUDA          (-4)  /* a CUDA call failed (no device, launch error, ...) */
+#define MVLA_ERR_CAPACITY      (-5)  /* batch / segment larger than the capacities given at create */
+#define MVLA_ERR_TIMEOUT       (-6)  /* a bounded device-side wait gave up in an earlier call (sticky) */
+#define MVLA_ERR_STATE         (-7)  /* bad prune point or state slot */
+
+#define MVLA_DTYPE_BF16 0
+#define MVLA_DTYPE_FP32 1
+
+#define MVLA_SALIENCE_AUTO 0
+#define MVLA_SALIENCE_FMA  1
+
+#define MVLA_MODE_FIXED    0   /* per-modality keep ratios keep_2d / keep_3d */
+#define MVLA_MODE_ADAPTIVE 1   /* one total keep ratio, split by the stage rules */
+
+#define MVLA_FLAG_RESET_STATE     1u  /* restart the episode: this call is action step t = 1 */
+#define MVLA_FLAG_NO_STATE_UPDATE 2u  /* dry run: decide as usual but leave the smoothed state and t untouched */
+
+#define MVLA_SET_2D 1   /* candidate sets are bit sets */
+#define MVLA_SET_3D 2
+
+typedef struct mvla_ctx mvla_ctx;   /* opaque */
+
+/* Creation-time configuration.  Paper defaults (Sec. 5.4): tau_2d 0.08, tau_3d 0.20, beta 0.85,
+ * window_k 7.  eps_3d (default 0.02) quantifies "3D response near zero" of the target-object
+ * rule (Sec. 4.2); floor_ratio (default 0.10) is the share of each modality that always
+ * survives, the deterministic form of the 90 % background pruning (Sec. 4.2). */
+typedef struct mvla_config {
+    int32_t device;            /* CUDA device ordinal */
+    int32_t dtype;             /* MVLA_DTYPE_*: element type of q, k, v, hidden */
+    int32_t n_heads;           /* H; k/v heads == q heads */
+    int32_t head_dim;          /* d: 64 or 128 */
+    int32_t d_model;           /* D: hidden width, multiple of 8 (bf16) / 4 (fp32) */
+    int32_t max_batch;         /* capacity: samples per call */
+    int32_t max_text;          /* capacity: text tokens per sample, <= 64 */
+    int32_t max_2d;            /* capacity: 2D tokens per sample */
+    int32_t max_3d;            /* capacity: 3D tokens per sample; max_2d + max_3d <= 4096 */
+    int32_t n_prune_points;    /* independent smoothed states per slot (e.g. layers 2 and 8 -> 2) */
+    int32_t n_state_slots;     /* episodes tracked at once; 0 -> max_batch */
+    int32_t window_k;          /* Eq. 8 -> Eq. 9 switch */
+    int32_t cold_start_full_keep; /* 1: action step t = 1 keeps every token (Alg. 1 cold start) */
+    int32_t salience_path;     /* MVLA_SALIENCE_AUTO (0): tensor cores for bf16, FMA kernel for fp32;
+                                  MVLA_SALIENCE_FMA (1): the CUDA-core FMA kernel for either dtype */
+    double tau_2d, tau_3d;     /* Sec. 4.1 */
+    double beta;               /* Eq. 9 */
+    double eps_3d;
+    double floor_ratio;
+} mvla_config;
+
+/* One batch element (host array).  Offsets are rows relative to seq_off; the three segments
+ * must be disjoint and lie inside [0, n_txt + n_2d + n_3d).  n_txt >= 1, n_2d + n_3d >= 1. */
+typedef struct mvla_sample {
+    int32_t seq_off;           /* first row of the sample in the packed tensors */
+    int32_t off_txt, n_txt;
+    int32_t off_2d, n_2d;      /* multi-view images are one segment of views x patches */
+    int32_t off_3d, n_3d;
+    int32_t state_slot;        /* which smoothed state this sample continues, < n_state_slots */
+    double keep_2d, keep_3d;   /* FIXED: k_m = min(n_m, floor(keep_m * n_m + 0.5)) */
+    double keep_total;         /* ADAPTIVE: B = min(n_vis, floor(keep_total * n_vis + 0.5)) */
+} mvla_sample;
+
+/* Per-sample record of what the budget stage decided (device array, optional). */
+typedef struct mvla_diag {
+    int32_t t;                 /* 1-based action step this call was */
+    int32_t c_s1, c_s2, c_final; /* candidate sets (Sec. 4.1, 4.2, 4.4) */
+    int32_t budget, k_2d, k_3d;
+    int32_t reserved;
+    float x[4];                /* instantaneous [M^S1_2D, M^S1_3D, M^S2_2D, M^S2_3D] (Eq. 3-1, P2D, P3D) */
+    float mhat[4];             /* the same, smoothed (Eqs. 8, 9) */
+} mvla_diag;
+
+/* Inputs of the fused step (device pointers). hidden may be NULL in FIXED mode when
+ * out_hidden is NULL too. */
+typedef struct mvla_tensors {
+    const void *q, *k, *v;     /* [rows, H, d] */
+    const void *hidden;        /* [rows, D] */
+    int64_t rows;              /* rows allocated in each tensor (bounds the TMA descriptors) */
+} mvla_tensors;
+
+/* Outputs of the fused step (device pointers, caller-owned). */
+typedef struct mvla_outputs {
+    void *out_hidden;          /* [sum kept rows, D]     nullable (skipped) */
+    void *out_k, *out_v;       /* [sum kept rows, H, d]  nullable (skipped) */
+    int32_t *kept_idx;         /* [sum kept rows] positions relative to each sample's seq_off, ascending */
+    int32_t *out_offsets;      /* [batch + 1] row offsets of each sample in the outputs */
+    int32_t *budgets;          /* [batch][2] = (k_2d, k_3d)  nullable */
+    float *attn;               /* [sum n_vis] instantaneous scores a_j  nullable */
+    float *ahat;               /* [sum n_vis] smoothed scores used for ranking  nullable */
+    float *z;                  /* [sum n_vis] smoothed scores normalised to mean 1 per modality  nullable */
+    mvla_diag *diag;           /* [batch]  nullable */
+} mvla_outputs;
+
+/* Kept rows of a sample: n_txt + B where B = n_2d + n_3d on a cold-start step (t = 1 with
+ * cold_start_full_keep), else k_2d + k_3d (FIXED) or the total budget (ADAPTIVE); all host
+ * computable.  Allocating sum(n_txt + n_2d + n_3d) rows is always enough. */
+
+/*
+ * Create a context on cfg->device: workspace, smoothed state for n_prune_points x
+ * n_state_slots episodes, a device status word.  Supported: dtype bf16 or fp32,
+ * head_dim 64 or 128, max_text <= 64, max_2d + max_3d <= 4096, max_batch <= 64.
+ * The library owns *out until mvla_prune_destroy.  (Alg. 1 "Input" / "Init".)
+ * Errors: INVALID_ARG, UNSUPPORTED, OOM, CUDA (no usable device).
+ */
+int32_t mvla_prune_create(const mvla_config *cfg, mvla_ctx **out);
+
+/*
+ * Salience (Sec. 3.2.1; Eq. 3-3 takes the L1 norm of a token's attention vector):
+ *   l[h,i,j] = <q[h,i], k[h,j]> / sqrt(d)  for text queries i and visual keys j,
+ *   alpha    = softmax over all visual keys j (2D and 3D jointly),
+ *   a_j      = mean over heads h and text queries i of alpha[h,i,j].
+ * and, when both `hidden` and `l1_out` are non-null, the L1 feature norm
+ *   n_j = sum_c |hidden[j,c]| of each visual token (Sec. 3.1.2).
+ * samples: host array [batch].  q, k, hidden: device, packed, `rows` rows each.
+ * attn_out, l1_out: device, sum(n_vis) floats in visual order.  Stateless.
+ */
+int32_t mvla_salience(mvla_ctx *ctx, int32_t batch, const mvla_sample *samples,
+                      const void *q, const void *k, const void *hidden, int64_t rows,
+                      float *attn_out, float *l1_out, void *stream);
+
+/*
+ * Carry-over, budget and selection (Alg. 1 steps 1-4; Eqs. 8, 9, 10):
+ * smooths `attn` into the per-token state and the four indicators into the
+ * indicator state of (prune_point, state_slot), decides the per-modality budgets
+ * and writes, per sample, the kept positions in ascending order merged with all
+ * text positions.  Advances the slot's step counter t (host side) unless
+ * MVLA_FLAG_NO_STATE_UPDATE.  `l1` is required in ADAPTIVE mode.
+ * kept_idx: device, capacity >= sum kept rows; out_offsets: device [batch+1];
+ * budgets, ahat_out, z_out, diag: nullable device arrays.  z_out = the smoothed scores
+ * normalised to mean 1 inside each modality (ranking inside a modality is the same on either).
+ */
+int32_t mvla_select(mvla_ctx *ctx, int32_t prune_point, int32_t batch, const mvla_sample *samples,
+                    int32_t mode, uint32_t flags, const float *attn, const float *l1,
+                    int32_t *kept_idx, int32_t *out_offsets, int32_t *budgets,
+                    float *ahat_out, float *z_out, mvla_diag *diag, void *stream);
+
+/*
+ * Compaction (Sec. 4.4: tokens with mask 1 proceed, the rest are discarded):
+ *   out_X[out_offsets[b] + r, :] = X[seq_off_b + kept_idx[out_offsets[b] + r], :]
+ * for X in {hidden, k, v}; a null input/output pair is skipped.  Rows are copied
+ * bit-exactly in 16-byte vectors.  `total_kept` is the host-known number of output
+ * rows (= out_offsets[batch]).  Outputs must not alias inputs.
+ */
+int32_t mvla_compact(mvla_ctx *ctx, int32_t batch, const mvla_sample *samples,
+                     const int32_t *kept_idx, const int32_t *out_offsets, int32_t total_kept,
+                     const void *hidden, const void *k, const void *v,
+                     void *out_hidden, void *out_k, void *out_v, void *stream);
+
+/*
+ * The whole prune point (Alg. 1) as one submission: salience (+ L1 norms in
+ * ADAPTIVE mode), carry-over, budget, select, compact.  Equivalent to the three
+ * calls above on the same arguments.  `total_kept_out` (host, nullable) receives
+ * the number of output rows.
+ */
+int32_t mvla_prune_step(mvla_ctx *ctx, int32_t prune_point, int32_t batch,
+                        const mvla_sample *samples, int32_t mode, uint32_t flags,
+                        const mvla_tensors *in, const mvla_outputs *out,
+                        int32_t *total_kept_out, void *stream);
+
+/* Free everything the context owns.  NULL is accepted.  The caller must have
+ * synchronised any stream that still runs work enqueued through the context. */
+void mvla_prune_destroy(mvla_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MVLA_PRUNE_H */

@@ -1,0 +1,496 @@
+// C-ABI layer: argument validation, host-side budget arithmetic, workspace and smoothed state,
+// tensor-map construction, launch sequencing.  No stream synchronisation anywhere.
+#include "common.cuh"
+
+#include <cudaTypedefs.h>
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace mvla;
+
+struct mvla_ctx {
+    mvla_config cfg;
+    int n_slots;
+    int max_vis;
+    size_t elem;                 // bytes per input element
+    bool use_umma;               // bf16 tensor-core salience path
+    float* part;                 // [H][max_batch * max_vis] per-head partial scores
+    int64_t part_stride;
+    float* attn_ws;              // [max_batch * max_vis]
+    float* l1_ws;                // [max_batch * max_vis]
+    float* ahat_state;           // [n_prune_points][n_slots][max_vis]
+    float* mhat_state;           // [n_prune_points][n_slots][4]
+    std::vector<int32_t> t_host; // [n_prune_points][n_slots] steps absorbed so far
+    int* status_host;            // mapped pinned word written by kernels whose bounded wait gave up
+    int* status_dev;
+    cudaError_t last_cuda;
+    PFN_cuTensorMapEncodeTiled_v12000 encode;
+    // tensor maps are cached per (pointer, rows)
+    const void* tm_ptr[2];
+    int64_t tm_rows[2];
+    CUtensorMap tm[2];
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard()
+    {
+        if (ok && prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+inline int32_t rhu(double x) { return static_cast<int32_t>(std::floor(x + 0.5)); }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int32_t fail_cuda(mvla_ctx* ctx, cudaError_t e)
+{
+    ctx->last_cuda = e;
+    return e == cudaErrorMemoryAllocation ? MVLA_ERR_OOM : MVLA_ERR_CUDA;
+}
+
+int32_t validate_samples(const mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, int32_t mode,
+                         int64_t rows)
+{
+    if (batch < 1 || !samples) return MVLA_ERR_INVALID_ARG;
+    if (batch > ctx->cfg.max_batch) return MVLA_ERR_CAPACITY;
+    if (mode != MVLA_MODE_FIXED && mode != MVLA_MODE_ADAPTIVE) return MVLA_ERR_INVALID_ARG;
+    for (int b = 0; b < batch; ++b) {
+        const mvla_sample& s = samples[b];
+        if (s.n_txt < 1 || s.n_2d < 0 || s.n_3d < 0 || s.n_2d + s.n_3d < 1 || s.seq_off < 0) return MVLA_ERR_INVALID_ARG;
+        if (s.n_txt > ctx->cfg.max_text || s.n_2d > ctx->cfg.max_2d || s.n_3d > ctx->cfg.max_3d) return MVLA_ERR_CAPACITY;
+        const int seq = s.n_txt + s.n_2d + s.n_3d;
+        const int off[3] = {s.off_txt, s.off_2d, s.off_3d}, len[3] = {s.n_txt, s.n_2d, s.n_3d};
+        for (int i = 0; i < 3; ++i) {
+            if (off[i] < 0 || off[i] + len[i] > seq) return MVLA_ERR_INVALID_ARG;
+            for (int j = i + 1; j < 3; ++j)
+                if (len[i] > 0 && len[j] > 0 && off[i] < off[j] + len[j] && off[j] < off[i] + len[i])
+                    return MVLA_ERR_INVALID_ARG;       // segments overlap
+        }
+        if (rows >= 0 && static_cast<int64_t>(s.seq_off) + seq > rows) return MVLA_ERR_INVALID_ARG;
+        if (s.state_slot < 0 || s.state_slot >= ctx->n_slots) return MVLA_ERR_STATE;
+        const double keeps[3] = {s.keep_2d, s.keep_3d, s.keep_total};
+        for (double kq : keeps)
+            if (!(kq >= 0.0) || !std::isfinite(kq)) return MVLA_ERR_INVALID_ARG;
+    }
+    return MVLA_OK;
+}
+
+// Everything about a call that the host can decide: layout offsets, budgets, state addressing,
+// the smoothing weights of this action step.
+struct Plan {
+    std::vector<SampleDev> s;
+    int32_t total_vis = 0;
+    int32_t total_out = 0;
+};
+
+int32_t make_plan(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, int32_t mode,
+                  uint32_t flags, bool with_state, Plan* plan)
+{
+    plan->s.resize(batch);
+    const mvla_config& c = ctx->cfg;
+    if (with_state) {
+        if (prune_point < 0 || prune_point >= c.n_prune_points) return MVLA_ERR_STATE;
+        for (int b = 0; b < batch; ++b)
+            for (int b2 = b + 1; b2 < batch; ++b2)
+                if (samples[b].state_slot == samples[b2].state_slot) return MVLA_ERR_STATE;   // two writers of one state
+    }
+    int32_t vis_off = 0, out_off = 0;
+    for (int b = 0; b < batch; ++b) {
+        const mvla_sample& in = samples[b];
+        SampleDev d;
+        std::memset(&d, 0, sizeof d);
+        d.seq_off = in.seq_off; d.off_txt = in.off_txt; d.n_txt = in.n_txt;
+        d.off_2d = in.off_2d; d.n_2d = in.n_2d; d.off_3d = in.off_3d; d.n_3d = in.n_3d;
+        const int nv = in.n_2d + in.n_3d;
+        d.vis_off = vis_off;
+        vis_off += nv;
+        d.k_2d_fixed = -1;
+        d.t = 1; d.update_state = 0; d.c_prev = 0.f; d.c_new = 1.f;
+        if (with_state) {
+            const int sidx = prune_point * ctx->n_slots + in.state_slot;
+            const int t_prev = (flags & MVLA_FLAG_RESET_STATE) ? 0 : ctx->t_host[sidx];
+            const int t = t_prev + 1;
+            d.t = t;
+            d.state_off = sidx * ctx->max_vis;
+            d.mstate_off = sidx;
+            d.update_state = (flags & MVLA_FLAG_NO_STATE_UPDATE) ? 0 : 1;
+            if (t <= 1) { d.c_prev = 0.f; d.c_new = 1.f; }                                   // X^_1 = X_1
+            else if (t < c.window_k) {                                                        // Eq. 8
+                d.c_prev = static_cast<float>(static_cast<double>(t - 1) / t);
+                d.c_new = static_cast<float>(1.0 / t);
+            } else {                                                                          // Eq. 9
+                d.c_prev = static_cast<float>(c.beta);
+                d.c_new = static_cast<float>(1.0 - c.beta);
+            }
+            if (t == 1 && c.cold_start_full_keep) {                                           // Alg. 1 cold start
+                d.budget = nv;
+                d.k_2d_fixed = in.n_2d;
+            } else if (mode == MVLA_MODE_FIXED) {
+                const int k2 = std::min(in.n_2d, rhu(in.keep_2d * in.n_2d));
+                const int k3 = std::min(in.n_3d, rhu(in.keep_3d * in.n_3d));
+                d.budget = k2 + k3;
+                d.k_2d_fixed = k2;
+            } else {
+                const int B = std::min(nv, rhu(in.keep_total * nv));
+                d.budget = B;
+                d.kmin_2d = std::min(static_cast<int>(std::ceil(c.floor_ratio * in.n_2d)),
+                                     static_cast<int>(std::floor(static_cast<double>(B) * in.n_2d / nv)));
+                d.kmin_3d = std::min(static_cast<int>(std::ceil(c.floor_ratio * in.n_3d)),
+                                     static_cast<int>(std::floor(static_cast<double>(B) * in.n_3d / nv)));
+            }
+            d.n_out = in.n_txt + d.budget;
+            d.out_off = out_off;
+            out_off += d.n_out;
+        }
+        plan->s[b] = d;
+    }
+    plan->total_vis = vis_off;
+    plan->total_out = out_off;
+    return MVLA_OK;
+}
+
+void commit_steps(mvla_ctx* ctx, int32_t prune_point, const Plan& plan, const mvla_sample* samples)
+{
+    for (size_t b = 0; b < plan.s.size(); ++b)
+        if (plan.s[b].update_state) ctx->t_host[prune_point * ctx->n_slots + samples[b].state_slot] = plan.s[b].t;
+}
+
+BatchDesc chunk_of(const Plan& plan, int first, int n)
+{
+    BatchDesc bd;
+    std::memset(&bd, 0, sizeof bd);
+    bd.n = n;
+    for (int i = 0; i < n; ++i) bd.s[i] = plan.s[first + i];
+    return bd;
+}
+
+int tiles_of(const SampleDev& s)
+{
+    return (s.n_2d + kKeyTile - 1) / kKeyTile + (s.n_3d + kKeyTile - 1) / kKeyTile;
+}
+
+// 3-D view (head_dim, heads, rows) of a token-major [rows, H, d] bf16 tensor; boxes of 64 x 1 x
+// `box_rows` land in shared memory as `box_rows` rows of 128 bytes with the 128-byte swizzle.
+int32_t tensor_map(mvla_ctx* ctx, int which, const void* ptr, int64_t rows, int box_rows, const CUtensorMap** out)
+{
+    if (ctx->tm_ptr[which] == ptr && ctx->tm_rows[which] == rows) {
+        *out = &ctx->tm[which];
+        return MVLA_OK;
+    }
+    const mvla_config& c = ctx->cfg;
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(c.head_dim), static_cast<cuuint64_t>(c.n_heads),
+                          static_cast<cuuint64_t>(rows)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(c.head_dim) * 2, static_cast<cuuint64_t>(c.head_dim) * c.n_heads * 2};
+    cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(box_rows)};
+    cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = ctx->encode(&ctx->tm[which], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims,
+                                   strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        ctx->tm_ptr[which] = nullptr;
+        return MVLA_ERR_CUDA;
+    }
+    ctx->tm_ptr[which] = ptr;
+    ctx->tm_rows[which] = rows;
+    *out = &ctx->tm[which];
+    return MVLA_OK;
+}
+
+int32_t check_sticky(mvla_ctx* ctx)
+{
+    return (ctx->status_host && *reinterpret_cast<volatile int*>(ctx->status_host) != 0) ? MVLA_ERR_TIMEOUT : MVLA_OK;
+}
+
+// Salience of one chunk into ctx->part (+ L1 norms into `l1` when asked).
+int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, const void* k, int64_t rows,
+                           const void* hidden, float* l1, cudaStream_t st)
+{
+    const mvla_config& c = ctx->cfg;
+    int max_tiles = 1, max_txt = 1;
+    for (int b = 0; b < bd.n; ++b) {
+        max_tiles = std::max(max_tiles, tiles_of(bd.s[b]));
+        max_txt = std::max(max_txt, bd.s[b].n_txt);
+    }
+    const int tiles_per_cta = (max_tiles + kMaxCluster - 1) / kMaxCluster;
+    const int cluster = (max_tiles + tiles_per_cta - 1) / tiles_per_cta;
+    const int npad = (max_txt + 15) / 16 * 16;
+    const CUtensorMap *tq = nullptr, *tk = nullptr;
+    if (ctx->use_umma) {
+        int32_t r = tensor_map(ctx, 0, q, rows, 16, &tq);
+        if (r != MVLA_OK) return r;
+        r = tensor_map(ctx, 1, k, rows, kKeyTile, &tk);
+        if (r != MVLA_OK) return r;
+    }
+    cudaError_t e = launch_salience(bd, c.dtype, c.n_heads, c.head_dim, q, k, tq, tk, ctx->use_umma, tiles_per_cta,
+                                    cluster, npad, ctx->part, ctx->part_stride, ctx->status_dev, st);
+    if (e == cudaErrorInvalidConfiguration) return MVLA_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    if (hidden && l1) {
+        e = launch_l1norm(bd, c.dtype, c.d_model, hidden, l1, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
+    return MVLA_OK;
+}
+
+GateParams gate_params(const mvla_ctx* ctx, int32_t mode, bool has_l1)
+{
+    GateParams gp;
+    gp.tau_2d = static_cast<float>(ctx->cfg.tau_2d);
+    gp.tau_3d = static_cast<float>(ctx->cfg.tau_3d);
+    gp.eps_3d = static_cast<float>(ctx->cfg.eps_3d);
+    gp.adaptive = mode == MVLA_MODE_ADAPTIVE;
+    gp.has_l1 = has_l1;
+    return gp;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
+{
+    if (!cfg || !out) return MVLA_ERR_INVALID_ARG;
+    *out = nullptr;
+    const mvla_config& c = *cfg;
+    if (c.n_heads < 1 || c.d_model < 1 || c.max_batch < 1 || c.max_text < 1 || c.max_2d < 0 || c.max_3d < 0 ||
+        c.max_2d + c.max_3d < 1 || c.n_prune_points < 1 || c.n_state_slots < 0 || c.window_k < 1 || c.device < 0)
+        return MVLA_ERR_INVALID_ARG;
+    if (!(c.beta >= 0.0 && c.beta <= 1.0) || !(c.floor_ratio >= 0.0 && c.floor_ratio <= 1.0) ||
+        !std::isfinite(c.tau_2d) || !std::isfinite(c.tau_3d) || !std::isfinite(c.eps_3d))
+        return MVLA_ERR_INVALID_ARG;
+    if (c.dtype != MVLA_DTYPE_BF16 && c.dtype != MVLA_DTYPE_FP32) return MVLA_ERR_UNSUPPORTED;
+    if (c.salience_path != MVLA_SALIENCE_AUTO && c.salience_path != MVLA_SALIENCE_FMA) return MVLA_ERR_INVALID_ARG;
+    if (c.head_dim != 64 && c.head_dim != 128) return MVLA_ERR_UNSUPPORTED;
+    if (c.max_text > kMaxText || c.max_2d + c.max_3d > kMaxVis || c.max_batch > 64) return MVLA_ERR_UNSUPPORTED;
+    const size_t elem = c.dtype == MVLA_DTYPE_BF16 ? 2 : 4;
+    if ((static_cast<size_t>(c.d_model) * elem) % 16 != 0) return MVLA_ERR_UNSUPPORTED;
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || c.device >= ndev) {
+        cudaGetLastError();
+        return MVLA_ERR_CUDA;
+    }
+    DeviceGuard guard(c.device);
+    if (!guard.ok) return MVLA_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, c.device) != cudaSuccess) return MVLA_ERR_CUDA;
+    if (prop.major != 10) return MVLA_ERR_UNSUPPORTED;        // built for sm_100a only
+
+    mvla_ctx* ctx = new (std::nothrow) mvla_ctx();
+    if (!ctx) return MVLA_ERR_OOM;
+    ctx->cfg = c;
+    ctx->n_slots = c.n_state_slots > 0 ? c.n_state_slots : c.max_batch;
+    ctx->max_vis = c.max_2d + c.max_3d;
+    ctx->elem = elem;
+    ctx->use_umma = c.dtype == MVLA_DTYPE_BF16;
+    if (c.salience_path == MVLA_SALIENCE_FMA) ctx->use_umma = false;
+    ctx->part = ctx->attn_ws = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
+    ctx->status_host = ctx->status_dev = nullptr;
+    ctx->last_cuda = cudaSuccess;
+    ctx->tm_ptr[0] = ctx->tm_ptr[1] = nullptr;
+    ctx->tm_rows[0] = ctx->tm_rows[1] = -1;
+    ctx->encode = nullptr;
+    ctx->t_host.assign(static_cast<size_t>(c.n_prune_points) * ctx->n_slots, 0);
+
+    const size_t vis_all = static_cast<size_t>(c.max_batch) * ctx->max_vis;
+    ctx->part_stride = static_cast<int64_t>(vis_all);
+    const size_t n_state = static_cast<size_t>(c.n_prune_points) * ctx->n_slots;
+    cudaError_t e = cudaSuccess;
+    auto alloc = [&](float** p, size_t n) {
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(p), n * sizeof(float));
+        if (e == cudaSuccess) e = cudaMemset(*p, 0, n * sizeof(float));
+    };
+    alloc(&ctx->part, vis_all * c.n_heads);
+    alloc(&ctx->attn_ws, vis_all);
+    alloc(&ctx->l1_ws, vis_all);
+    alloc(&ctx->ahat_state, n_state * ctx->max_vis);
+    alloc(&ctx->mhat_state, n_state * 4);
+    if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&ctx->status_host), sizeof(int), cudaHostAllocMapped);
+    if (e == cudaSuccess) {
+        *ctx->status_host = 0;
+        e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&ctx->status_dev), ctx->status_host, 0);
+    }
+    if (e == cudaSuccess && ctx->use_umma) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres);
+        if (e == cudaSuccess && (qres != cudaDriverEntryPointSuccess || !fn)) e = cudaErrorNotSupported;
+        ctx->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+    }
+    if (e != cudaSuccess) {
+        const int32_t rc = e == cudaErrorMemoryAllocation ? MVLA_ERR_OOM : MVLA_ERR_CUDA;
+        cudaGetLastError();
+        mvla_prune_destroy(ctx);
+        return rc;
+    }
+    *out = ctx;
+    return MVLA_OK;
+}
+
+void mvla_prune_destroy(mvla_ctx* ctx)
+{
+    if (!ctx) return;
+    DeviceGuard guard(ctx->cfg.device);
+    cudaFree(ctx->part);
+    cudaFree(ctx->attn_ws);
+    cudaFree(ctx->l1_ws);
+    cudaFree(ctx->ahat_state);
+    cudaFree(ctx->mhat_state);
+    if (ctx->status_host) cudaFreeHost(ctx->status_host);
+    delete ctx;
+}
+
+int32_t mvla_salience(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const void* q, const void* k,
+                      const void* hidden, int64_t rows, float* attn_out, float* l1_out, void* stream)
+{
+    if (!ctx || !q || !k || !attn_out || rows < 1) return MVLA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(hidden)) return MVLA_ERR_INVALID_ARG;
+    int32_t rc = check_sticky(ctx);
+    if (rc != MVLA_OK) return rc;
+    rc = validate_samples(ctx, batch, samples, MVLA_MODE_FIXED, rows);
+    if (rc != MVLA_OK) return rc;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return MVLA_ERR_CUDA;
+    Plan plan;
+    rc = make_plan(ctx, 0, batch, samples, MVLA_MODE_FIXED, 0, false, &plan);
+    if (rc != MVLA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool want_l1 = hidden && l1_out;
+    for (int first = 0; first < batch; first += kMaxChunk) {
+        const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
+        rc = run_salience_chunk(ctx, bd, q, k, rows, want_l1 ? hidden : nullptr, l1_out, st);
+        if (rc != MVLA_OK) return rc;
+    }
+    const cudaError_t e = launch_head_reduce(ctx->part, ctx->part_stride, ctx->cfg.n_heads, plan.total_vis, attn_out, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    return MVLA_OK;
+}
+
+int32_t mvla_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, int32_t mode,
+                    uint32_t flags, const float* attn, const float* l1, int32_t* kept_idx, int32_t* out_offsets,
+                    int32_t* budgets, float* ahat_out, float* z_out, mvla_diag* diag, void* stream)
+{
+    if (!ctx || !attn || !kept_idx || !out_offsets) return MVLA_ERR_INVALID_ARG;
+    if (flags & ~(MVLA_FLAG_RESET_STATE | MVLA_FLAG_NO_STATE_UPDATE)) return MVLA_ERR_INVALID_ARG;
+    int32_t rc = check_sticky(ctx);
+    if (rc != MVLA_OK) return rc;
+    rc = validate_samples(ctx, batch, samples, mode, -1);
+    if (rc != MVLA_OK) return rc;
+    if (mode == MVLA_MODE_ADAPTIVE && !l1) return MVLA_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return MVLA_ERR_CUDA;
+    Plan plan;
+    rc = make_plan(ctx, prune_point, batch, samples, mode, flags, true, &plan);
+    if (rc != MVLA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const GateParams gp = gate_params(ctx, mode, l1 != nullptr);
+    for (int first = 0; first < batch; first += kMaxChunk) {
+        const int n = std::min(kMaxChunk, batch - first);
+        const BatchDesc bd = chunk_of(plan, first, n);
+        const cudaError_t e = launch_select(bd, gp, attn, nullptr, 0, ctx->cfg.n_heads, l1, ctx->ahat_state,
+                                            ctx->mhat_state, kept_idx, out_offsets, first, plan.total_out,
+                                            first + n == batch, budgets, nullptr, ahat_out, z_out, diag, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
+    commit_steps(ctx, prune_point, plan, samples);
+    return MVLA_OK;
+}
+
+int32_t mvla_compact(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const int32_t* kept_idx,
+                     const int32_t* out_offsets, int32_t total_kept, const void* hidden, const void* k,
+                     const void* v, void* out_hidden, void* out_k, void* out_v, void* stream)
+{
+    if (!ctx || !kept_idx || !out_offsets || total_kept < 0) return MVLA_ERR_INVALID_ARG;
+    const void* src[3] = {hidden, k, v};
+    void* dst[3] = {out_hidden, out_k, out_v};
+    for (int i = 0; i < 3; ++i) {
+        if (!src[i] || !dst[i]) continue;
+        if (!aligned16(src[i]) || !aligned16(dst[i]) || src[i] == dst[i]) return MVLA_ERR_INVALID_ARG;
+    }
+    int32_t rc = check_sticky(ctx);
+    if (rc != MVLA_OK) return rc;
+    rc = validate_samples(ctx, batch, samples, MVLA_MODE_FIXED, -1);
+    if (rc != MVLA_OK) return rc;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return MVLA_ERR_CUDA;
+    Plan plan;
+    rc = make_plan(ctx, 0, batch, samples, MVLA_MODE_FIXED, 0, false, &plan);
+    if (rc != MVLA_OK) return rc;
+    CompactJob job;
+    const int32_t kv_bytes = static_cast<int32_t>(ctx->cfg.n_heads * ctx->cfg.head_dim * ctx->elem);
+    for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
+    job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int first = 0; first < batch; first += kMaxChunk) {
+        const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
+        const cudaError_t e = launch_compact(bd, job, kept_idx, total_kept, 0, out_offsets, first, batch, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
+    return MVLA_OK;
+}
+
+int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples,
+                        int32_t mode, uint32_t flags, const mvla_tensors* in, const mvla_outputs* out,
+                        int32_t* total_kept_out, void* stream)
+{
+    if (!ctx || !in || !out || !in->q || !in->k || !out->kept_idx || !out->out_offsets || in->rows < 1)
+        return MVLA_ERR_INVALID_ARG;
+    if (flags & ~(MVLA_FLAG_RESET_STATE | MVLA_FLAG_NO_STATE_UPDATE)) return MVLA_ERR_INVALID_ARG;
+    if (mode == MVLA_MODE_ADAPTIVE && !in->hidden) return MVLA_ERR_INVALID_ARG;
+    const void* src[3] = {in->hidden, in->k, in->v};
+    void* dst[3] = {out->out_hidden, out->out_k, out->out_v};
+    if (!aligned16(in->q)) return MVLA_ERR_INVALID_ARG;
+    for (int i = 0; i < 3; ++i) {
+        if (!aligned16(src[i]) || !aligned16(dst[i])) return MVLA_ERR_INVALID_ARG;
+        if (dst[i] && (!src[i] || src[i] == dst[i])) return MVLA_ERR_INVALID_ARG;
+    }
+    int32_t rc = check_sticky(ctx);
+    if (rc != MVLA_OK) return rc;
+    rc = validate_samples(ctx, batch, samples, mode, in->rows);
+    if (rc != MVLA_OK) return rc;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return MVLA_ERR_CUDA;
+    Plan plan;
+    rc = make_plan(ctx, prune_point, batch, samples, mode, flags, true, &plan);
+    if (rc != MVLA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool adaptive = mode == MVLA_MODE_ADAPTIVE;
+    const GateParams gp = gate_params(ctx, mode, adaptive);
+    CompactJob job;
+    const int32_t kv_bytes = static_cast<int32_t>(ctx->cfg.n_heads * ctx->cfg.head_dim * ctx->elem);
+    for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
+    job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
+
+    for (int first = 0; first < batch; first += kMaxChunk) {
+        const int n = std::min(kMaxChunk, batch - first);
+        const BatchDesc bd = chunk_of(plan, first, n);
+        rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, ctx->l1_ws, st);
+        if (rc != MVLA_OK) return rc;
+        cudaError_t e = launch_select(bd, gp, nullptr, ctx->part, ctx->part_stride, ctx->cfg.n_heads,
+                                      adaptive ? ctx->l1_ws : nullptr, ctx->ahat_state, ctx->mhat_state,
+                                      out->kept_idx, out->out_offsets, first, plan.total_out, first + n == batch,
+                                      out->budgets, out->attn, out->ahat, out->z, out->diag, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        const int32_t row0 = bd.s[0].out_off;
+        const int32_t nrows = bd.s[n - 1].out_off + bd.s[n - 1].n_out - row0;
+        e = launch_compact(bd, job, out->kept_idx, nrows, row0, nullptr, first, batch, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
+    commit_steps(ctx, prune_point, plan, samples);
+    if (total_kept_out) *total_kept_out = plan.total_out;
+    return MVLA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,87 @@
+// Internal declarations shared by the kernels and the C-ABI layer.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "mvla_prune.h"
+
+namespace mvla {
+
+constexpr int kMaxChunk = 32;        // samples carried by one launch (descriptors travel as kernel parameters)
+constexpr int kKeyTile = 128;        // visual keys per tile = rows of one MMA
+constexpr int kMaxCluster = 8;       // portable cluster size
+constexpr int kMaxText = 64;
+constexpr int kMaxVis = 4096;
+constexpr uint32_t kSpinLimit = 1u << 22;   // bounded device-side waits (each try sleeps, see wait loops)
+
+// Device-side view of one sample; everything the host can compute is computed there.
+struct SampleDev {
+    int32_t seq_off, off_txt, n_txt, off_2d, n_2d, off_3d, n_3d;
+    int32_t vis_off;        // offset of the sample in packed [sum n_vis] arrays
+    int32_t out_off;        // first output row
+    int32_t n_out;          // kept rows = n_txt + budget
+    int32_t budget;         // kept visual tokens (host known)
+    int32_t k_2d_fixed;     // >= 0: host-decided split (FIXED mode or cold start); -1: split on device
+    int32_t kmin_2d, kmin_3d;   // ADAPTIVE floors
+    int32_t state_off;      // offset of this (prune point, slot) in the per-token state array
+    int32_t mstate_off;     // index of this (prune point, slot) in the indicator state array (x4 floats)
+    int32_t t;              // 1-based action step this call is
+    int32_t update_state;   // 0: dry run
+    float c_prev, c_new;    // state update weights: xhat = c_prev * xhat + c_new * x
+};
+
+struct BatchDesc {
+    SampleDev s[kMaxChunk];
+    int32_t n;
+};
+
+struct GateParams {
+    float tau_2d, tau_3d, eps_3d;
+    int32_t adaptive;       // mode
+    int32_t has_l1;
+};
+
+// ---- launchers (each enqueues on `stream` and returns the launch status) ----
+
+// Salience: per-head partial scores part[h][vis] (already scaled by 1/(H n_t)).
+// `use_umma`: tensor-core path (bf16 only).  tmaps: device-usable tensor maps (passed by value).
+cudaError_t launch_salience(const BatchDesc& bd, int dtype, int n_heads, int head_dim,
+                            const void* q, const void* k, const CUtensorMap* tmap_q,
+                            const CUtensorMap* tmap_k, bool use_umma, int tiles_per_cta,
+                            int cluster, int npad, float* part, int64_t part_stride,
+                            int* status, cudaStream_t stream);
+
+// attn[j] = sum_h part[h][j]  (fixed head order).
+cudaError_t launch_head_reduce(const float* part, int64_t part_stride, int n_heads, int total_vis,
+                               float* attn, cudaStream_t stream);
+
+// L1 feature norms of the visual rows.
+cudaError_t launch_l1norm(const BatchDesc& bd, int dtype, int d_model, const void* hidden,
+                          float* l1, cudaStream_t stream);
+
+// Carry-over + budget + top-k + emission; one CTA per sample.
+// Scores come either from `attn` (part == nullptr) or from per-head partials.
+cudaError_t launch_select(const BatchDesc& bd, const GateParams& gp, const float* attn,
+                          const float* part, int64_t part_stride, int n_heads, const float* l1,
+                          float* ahat_state, float* mhat_state, int32_t* kept_idx,
+                          int32_t* out_offsets, int chunk_first, int32_t total_out, int write_total,
+                          int32_t* budgets, float* attn_out, float* ahat_out, float* z_out,
+                          mvla_diag* diag, cudaStream_t stream);
+
+// Row gather of up to three tensors.
+struct CompactJob {
+    const void* src[3];
+    void* dst[3];
+    int32_t row_bytes[3];
+};
+// Rows [chunk_row0, chunk_row0 + chunk_rows) of the output.  With `out_offsets` (device) the owning
+// sample of a row is looked up there over the whole batch and rows of samples outside this launch's
+// descriptors are skipped; without it the descriptors' host-computed out_off is used.
+cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int32_t* kept_idx,
+                           int32_t chunk_rows, int32_t chunk_row0, const int32_t* out_offsets,
+                           int32_t chunk_first, int32_t batch_total, cudaStream_t stream);
+
+}  // namespace mvla

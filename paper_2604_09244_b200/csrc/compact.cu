@@ -1,0 +1,107 @@
+// Compaction (Sec. 4.4 of the paper: tokens whose mask is 1 proceed, the others are discarded):
+// gathers the kept rows of hidden / K / V into the dense pruned layout.
+//
+// Pure data movement, HBM bound.  One warp moves one 2 KB segment of one row of one tensor: four
+// 16-byte loads per lane are issued back to back (512 bytes per lane-round in flight per warp),
+// then four stores.  The loads bypass L1 (read once), the stores are streaming.
+#include "common.cuh"
+
+namespace mvla {
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+constexpr int kSegBytes = 2048;     // 32 lanes x 4 x 16 B
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(uint4* p, const uint4& v)
+{
+    asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+struct CompactArgs {
+    const uint8_t* src[3];
+    uint8_t* dst[3];
+    int32_t row_bytes[3];
+    int32_t segs[3];          // 2 KB segments per row
+    int32_t seg_begin[4];     // prefix sums of segs per row over the (up to) three tensors
+};
+
+// grid.x covers chunk_rows * segs_per_row_all warp-units.
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+compact_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CompactArgs a, const int32_t* __restrict__ kept_idx,
+               int32_t chunk_rows, int32_t chunk_row0, const int32_t* __restrict__ out_offsets,
+               int32_t chunk_first, int32_t batch_total)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t unit = static_cast<int64_t>(blockIdx.x) * kWarpsPerBlock + (threadIdx.x >> 5);
+    const int per_row = a.seg_begin[3];
+    if (unit >= static_cast<int64_t>(chunk_rows) * per_row) return;
+    const int r = static_cast<int>(unit / per_row);       // output row inside this chunk
+    const int u = static_cast<int>(unit - static_cast<int64_t>(r) * per_row);
+    const int orow = chunk_row0 + r;
+
+    // which sample owns output row `orow` (samples are few: linear scan)
+    int b = 0;
+    if (out_offsets) {            // offsets known only on the device: scan the whole batch
+        while (b + 1 < batch_total && orow >= out_offsets[b + 1]) ++b;
+        b -= chunk_first;
+        if (b < 0 || b >= bd.n) return;      // row belongs to another launch's samples
+    } else {
+        while (b + 1 < bd.n && orow >= bd.s[b + 1].out_off) ++b;
+    }
+    const int64_t srow = static_cast<int64_t>(bd.s[b].seq_off) + kept_idx[orow];
+
+    const int tsel = u >= a.seg_begin[2] ? 2 : (u >= a.seg_begin[1] ? 1 : 0);
+    const int seg = u - a.seg_begin[tsel];
+    const int rb = a.row_bytes[tsel];
+    const uint8_t* sp = a.src[tsel] + srow * rb + static_cast<int64_t>(seg) * kSegBytes;
+    uint8_t* dp = a.dst[tsel] + static_cast<int64_t>(orow) * rb + static_cast<int64_t>(seg) * kSegBytes;
+    const int nbytes = min(kSegBytes, rb - seg * kSegBytes);
+    const int nvec = nbytes >> 4;
+
+    uint4 v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int idx = lane + i * 32;
+        if (idx < nvec) v[i] = ld_stream(reinterpret_cast<const uint4*>(sp) + idx);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int idx = lane + i * 32;
+        if (idx < nvec) st_stream(reinterpret_cast<uint4*>(dp) + idx, v[i]);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int32_t* kept_idx,
+                           int32_t chunk_rows, int32_t chunk_row0, const int32_t* out_offsets,
+                           int32_t chunk_first, int32_t batch_total, cudaStream_t stream)
+{
+    CompactArgs a;
+    int total = 0;
+    for (int i = 0; i < 3; ++i) {
+        const bool on = job.src[i] && job.dst[i];
+        a.src[i] = static_cast<const uint8_t*>(job.src[i]);
+        a.dst[i] = static_cast<uint8_t*>(job.dst[i]);
+        a.row_bytes[i] = job.row_bytes[i];
+        a.segs[i] = on ? (job.row_bytes[i] + kSegBytes - 1) / kSegBytes : 0;
+        a.seg_begin[i] = total;
+        total += a.segs[i];
+    }
+    a.seg_begin[3] = total;
+    if (total == 0 || chunk_rows <= 0) return cudaSuccess;
+    const int64_t units = static_cast<int64_t>(chunk_rows) * total;
+    const int64_t blocks = (units + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    compact_kernel<<<static_cast<unsigned>(blocks), kWarpsPerBlock * 32, 0, stream>>>(
+        bd, a, kept_idx, chunk_rows, chunk_row0, out_offsets, chunk_first, batch_total);
+    return cudaGetLastError();
+}
+
+}  // namespace mvla

@@ -1,0 +1,557 @@
+// Salience of the visual tokens (Sec. 3.2.1 of the paper): scaled dot-product logits of the text
+// queries against the visual keys, softmax over all visual keys, mean over heads and queries.
+//
+// Work split: one thread-block cluster per (sample, head); each CTA of the cluster owns
+// `tiles_per_cta` tiles of 128 keys.  A CTA produces the logits of its keys against all text
+// queries (tensor cores for bf16: TMA -> shared memory -> tcgen05.mma -> tensor memory; plain
+// FMAs for fp32), reduces a local softmax maximum and denominator per query, exchanges those with
+// the other CTAs of the cluster through distributed shared memory, and writes, per key, the
+// head's contribution  sum_i softmax(l[h,i,:])_j / (H n_t)  to part[h][j].  Heads are summed
+// later in a fixed order so that the result does not depend on scheduling.
+#include "common.cuh"
+
+#include <math_constants.h>
+
+namespace mvla {
+namespace {
+
+// ------------------------------------------------------------------ small PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\t"
+                 "barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_peer_f32(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t remote;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint64_t global_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait: gives up after about one second and reports false.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    const uint64_t t0 = global_ns();
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if (global_ns() - t0 > 1000000000ull) break;
+    }
+    return false;
+}
+// One box of a 3-D tiled tensor map -> this CTA's shared memory; completion counted on `bar`.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
+                                            uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "setp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 16 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
+{
+    uint32_t r[16];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32"
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor: K-major tile, 128-byte rows, 128-byte swizzle, groups of 8 rows
+// 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);          // start address
+    d |= static_cast<uint64_t>(1) << 16;                         // leading byte offset (unused here)
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;                 // stride byte offset
+    d |= static_cast<uint64_t>(1) << 46;                         // descriptor version
+    d |= static_cast<uint64_t>(2) << 61;                         // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t idesc_bf16_m128(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// Reduce 16 per-thread values across the 32 lanes of a warp in 16 shuffles.  On return lane L
+// holds the result of column col16(L); lanes L and L^1 hold the same column.
+template <bool IS_MAX>
+__device__ __forceinline__ float warp_reduce16(float (&v)[16], int lane)
+{
+#pragma unroll
+    for (int w = 8; w >= 1; w >>= 1) {
+        const int off = w * 2;
+        const bool up = (lane & off) != 0;
+#pragma unroll
+        for (int i = 0; i < w; ++i) {
+            const float send = up ? v[i] : v[i + w];
+            const float keep = up ? v[i + w] : v[i];
+            const float got = __shfl_xor_sync(0xffffffffu, send, off);
+            v[i] = IS_MAX ? fmaxf(keep, got) : keep + got;
+        }
+    }
+    const float got = __shfl_xor_sync(0xffffffffu, v[0], 1);
+    return IS_MAX ? fmaxf(v[0], got) : v[0] + got;
+}
+__device__ __forceinline__ int col16(int lane)
+{
+    return ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+}
+
+struct TileInfo {
+    int valid;   // keys of this tile that exist (0: tile past the end)
+    int row0;    // first row in the packed tensors
+    int vis0;    // visual index of the first key
+};
+__device__ __forceinline__ TileInfo tile_info(const SampleDev& s, int tt)
+{
+    const int t2 = (s.n_2d + kKeyTile - 1) / kKeyTile;
+    const int t3 = (s.n_3d + kKeyTile - 1) / kKeyTile;
+    TileInfo ti{0, 0, 0};
+    if (tt < t2) {
+        const int st = tt * kKeyTile;
+        ti.valid = min(kKeyTile, s.n_2d - st);
+        ti.row0 = s.seq_off + s.off_2d + st;
+        ti.vis0 = st;
+    } else if (tt < t2 + t3) {
+        const int st = (tt - t2) * kKeyTile;
+        ti.valid = min(kKeyTile, s.n_3d - st);
+        ti.row0 = s.seq_off + s.off_3d + st;
+        ti.vis0 = s.n_2d + st;
+    }
+    return ti;
+}
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+constexpr int kThreads = 128;
+
+// ------------------------------------------------------------------ the kernel
+// grid = (cluster size, n_heads, samples), cluster = (cluster size, 1, 1), block = 128 threads.
+// Thread r owns key r of each tile (tensor-memory lane r).
+template <typename T, bool UMMA>
+__global__ void __launch_bounds__(kThreads, 1)
+salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
+                const __grid_constant__ CUtensorMap tmap_k, const T* __restrict__ q,
+                const T* __restrict__ k, int n_heads, int head_dim, int tiles_per_cta, int npad,
+                float* __restrict__ part, int64_t part_stride, int* status)
+{
+    extern __shared__ uint8_t dyn_smem_raw[];
+    uint8_t* dyn_smem = dyn_smem_raw + ((1024u - (smem_u32(dyn_smem_raw) & 1023u)) & 1023u);   // swizzle atoms are 1 KB
+    __shared__ float s_m[kMaxText];          // local max per query (log2 domain), -inf replaced by 0
+    __shared__ float s_w[kMaxText];          // final weight per query
+    __shared__ float s_stat[2][kMaxText];    // what peers read: raw local max, local sum
+    __shared__ float s_wred[4][kMaxText];
+    __shared__ __align__(8) uint64_t s_bar[2];
+    __shared__ uint32_t s_tmem;
+
+    const SampleDev& s = bd.s[blockIdx.z];
+    const int h = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t crank = cluster_ctarank();
+    const uint32_t csize = gridDim.x;
+    const int d = head_dim;
+    const int64_t row_elems = static_cast<int64_t>(n_heads) * d;
+    // logits are kept in the log2 domain: y = <q, k> * log2(e) / sqrt(d)
+    const float cscale = 1.4426950408889634f * rsqrtf(static_cast<float>(d));
+    const int tt0 = static_cast<int>(crank) * tiles_per_cta;
+
+    uint32_t tmem_base = 0, tmem_cols = 0;
+    const int tcol = npad <= 16 ? 16 : (npad <= 32 ? 32 : 64);   // tensor-memory columns reserved per tile
+    float* Ls = nullptr;   // fp32 path: logits [tile][query][key]
+    bool ok = true;
+
+    if constexpr (UMMA) {
+        const int khalves = d / 64;                           // 64 bf16 = one 128-byte swizzle row
+        uint8_t* Ks = dyn_smem;                               // [tile][khalf][128 rows x 128 B]
+        uint8_t* Qs = dyn_smem + static_cast<size_t>(tiles_per_cta) * khalves * 16384;   // [khalf][npad rows x 128 B]
+        const uint32_t bar_full = smem_u32(&s_bar[0]), bar_mma = smem_u32(&s_bar[1]);
+        tmem_cols = 32;
+        while (tmem_cols < static_cast<uint32_t>(tiles_per_cta * tcol)) tmem_cols <<= 1;
+        if (tid == 0) {
+            mbar_init(bar_full, 1);
+            mbar_init(bar_mma, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        if (warp == 0) {
+            __syncwarp();
+            tmem_alloc(smem_u32(&s_tmem), tmem_cols);
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        tmem_base = s_tmem;
+
+        if (tid == 0) {
+            int live = 0;
+            for (int t = 0; t < tiles_per_cta; ++t) live += tile_info(s, tt0 + t).valid > 0;
+            const uint32_t bytes = static_cast<uint32_t>(khalves) * (npad * 128 + live * 16384);
+            mbar_expect_tx(bar_full, bytes);
+            for (int kh = 0; kh < khalves; ++kh)
+                for (int c = 0; c < npad / 16; ++c)
+                    tma_load_3d(smem_u32(Qs + kh * npad * 128 + c * 2048), &tmap_q, kh * 64, h,
+                                s.seq_off + s.off_txt + c * 16, bar_full);
+            for (int t = 0; t < tiles_per_cta; ++t) {
+                const TileInfo ti = tile_info(s, tt0 + t);
+                if (ti.valid <= 0) continue;
+                for (int kh = 0; kh < khalves; ++kh)
+                    tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * 64, h, ti.row0, bar_full);
+            }
+            bool got = mbar_wait(bar_full, 0);
+            if (!got) {                       // report, then give the copies one more bounded chance to land
+                *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
+                got = mbar_wait(bar_full, 0);
+            }
+            if (got) {
+                tc_fence_after();
+                const uint32_t idesc = idesc_bf16_m128(npad);
+                for (int t = 0; t < tiles_per_cta; ++t) {
+                    if (tile_info(s, tt0 + t).valid <= 0) continue;
+                    for (int kb = 0; kb < d / 16; ++kb) {
+                        const int kh = kb >> 2, kin = kb & 3;      // 4 K-steps of 16 inside a 64-wide half
+                        const uint64_t a = smem_desc_sw128(smem_u32(Ks + (t * khalves + kh) * 16384) + kin * 32);
+                        const uint64_t b = smem_desc_sw128(smem_u32(Qs + kh * npad * 128) + kin * 32);
+                        umma_bf16(tmem_base + t * tcol, a, b, idesc, kb > 0 ? 1u : 0u);
+                    }
+                }
+            }
+            umma_commit(bar_mma);             // arrives once every MMA issued above has finished
+        }
+        __syncwarp();
+        if (!mbar_wait(bar_mma, 0)) {
+            ok = false;
+            *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
+        }
+        ok = __syncthreads_and(ok) != 0;      // block-uniform from here on (aligned instructions follow)
+        tc_fence_after();
+    } else {
+        // fp32 / generic path: stage Q and one key tile in shared memory as fp32, FMA the logits.
+        float* Qs = reinterpret_cast<float*>(dyn_smem);               // [npad][d]
+        float* Ks = Qs + npad * d;                                    // [128][d + 1]
+        Ls = Ks + kKeyTile * (d + 1);                                 // [tile][npad][128]
+        const int kp = d + 1;
+        for (int idx = tid; idx < npad * d; idx += kThreads) {
+            const int i = idx / d, c = idx - i * d;
+            Qs[idx] = i < s.n_txt
+                ? to_f32(q[static_cast<int64_t>(s.seq_off + s.off_txt + i) * row_elems + static_cast<int64_t>(h) * d + c])
+                : 0.f;
+        }
+        for (int t = 0; t < tiles_per_cta; ++t) {
+            const TileInfo ti = tile_info(s, tt0 + t);
+            if (ti.valid <= 0) continue;
+            __syncthreads();
+            for (int idx = tid; idx < kKeyTile * d; idx += kThreads) {
+                const int r = idx / d, c = idx - r * d;
+                Ks[r * kp + c] = r < ti.valid
+                    ? to_f32(k[static_cast<int64_t>(ti.row0 + r) * row_elems + static_cast<int64_t>(h) * d + c])
+                    : 0.f;
+            }
+            __syncthreads();
+            const float* kr = Ks + tid * kp;
+            for (int cb = 0; cb < npad; cb += 16) {
+                float acc[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+                for (int c = 0; c < d; c += 4) {
+                    const float k0 = kr[c], k1 = kr[c + 1], k2 = kr[c + 2], k3 = kr[c + 3];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float4 q4 = *reinterpret_cast<const float4*>(Qs + (cb + i) * d + c);
+                        acc[i] = fmaf(k0, q4.x, acc[i]);
+                        acc[i] = fmaf(k1, q4.y, acc[i]);
+                        acc[i] = fmaf(k2, q4.z, acc[i]);
+                        acc[i] = fmaf(k3, q4.w, acc[i]);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    Ls[(t * npad + cb + i) * kKeyTile + tid] = tid < ti.valid ? acc[i] * cscale : -CUDART_INF_F;
+            }
+        }
+        __syncthreads();
+    }
+
+    // Loads the 16 logits (log2 domain) of this thread's key for queries [cb, cb+16) of tile t.
+    auto load_chunk = [&](int t, int cb, int valid, float (&v)[16]) {
+        if constexpr (UMMA) {
+            tmem_ld16(tmem_base + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(t * tcol + cb), v);
+            const bool live = tid < valid;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = live ? v[i] * cscale : -CUDART_INF_F;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = Ls[(t * npad + cb + i) * kKeyTile + tid];
+        }
+    };
+
+    // ---- pass 1: local maximum per query over this CTA's keys
+    for (int cb = 0; cb < npad; cb += 16) {
+        float m[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) m[i] = -CUDART_INF_F;
+        for (int t = 0; t < tiles_per_cta; ++t) {
+            const int valid = tile_info(s, tt0 + t).valid;
+            if (valid <= 0 || !ok) continue;
+            float v[16];
+            load_chunk(t, cb, valid, v);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) m[i] = fmaxf(m[i], v[i]);
+        }
+        const float red = warp_reduce16<true>(m, lane);
+        if ((lane & 1) == 0) s_wred[warp][cb + col16(lane)] = red;
+    }
+    __syncthreads();
+    if (tid < npad) {
+        const float m = fmaxf(fmaxf(s_wred[0][tid], s_wred[1][tid]), fmaxf(s_wred[2][tid], s_wred[3][tid]));
+        s_stat[0][tid] = m;
+        s_m[tid] = (m == -CUDART_INF_F) ? 0.f : m;
+    }
+    __syncthreads();
+
+    // ---- pass 2: local softmax denominator per query
+    for (int cb = 0; cb < npad; cb += 16) {
+        float sum[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) sum[i] = 0.f;
+        for (int t = 0; t < tiles_per_cta; ++t) {
+            const int valid = tile_info(s, tt0 + t).valid;
+            if (valid <= 0 || !ok) continue;
+            float v[16];
+            load_chunk(t, cb, valid, v);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) sum[i] += exp2f(v[i] - s_m[cb + i]);
+        }
+        const float red = warp_reduce16<false>(sum, lane);
+        if ((lane & 1) == 0) s_wred[warp][cb + col16(lane)] = red;
+    }
+    __syncthreads();
+    if (tid < npad) s_stat[1][tid] = (s_wred[0][tid] + s_wred[1][tid]) + (s_wred[2][tid] + s_wred[3][tid]);
+    __syncthreads();
+
+    // ---- exchange (max, sum) with the other key tiles of this (sample, head)
+    cluster_sync_all();
+    if (tid < npad) {
+        const uint32_t a_m = smem_u32(&s_stat[0][tid]), a_s = smem_u32(&s_stat[1][tid]);
+        float gmax = -CUDART_INF_F;
+        for (uint32_t r = 0; r < csize; ++r) gmax = fmaxf(gmax, ld_peer_f32(a_m, r));
+        float z = 0.f;
+        for (uint32_t r = 0; r < csize; ++r) {
+            const float mr = ld_peer_f32(a_m, r);
+            if (mr > -CUDART_INF_F) z += ld_peer_f32(a_s, r) * exp2f(mr - gmax);
+        }
+        const float inv_hn = 1.f / (static_cast<float>(n_heads) * static_cast<float>(s.n_txt));
+        s_w[tid] = (tid < s.n_txt && z > 0.f) ? exp2f(s_m[tid] - gmax) / z * inv_hn : 0.f;
+    }
+    __syncthreads();
+
+    // ---- pass 3: per key, sum over queries of the normalised probabilities
+    for (int t = 0; t < tiles_per_cta; ++t) {
+        const TileInfo ti = tile_info(s, tt0 + t);
+        if (ti.valid <= 0) continue;
+        float acc = 0.f;
+        if (ok) {
+            for (int cb = 0; cb < npad; cb += 16) {
+                float v[16];
+                load_chunk(t, cb, ti.valid, v);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float e = exp2f(v[i] - s_m[cb + i]);
+                    acc += (cb + i < s.n_txt) ? e * s_w[cb + i] : 0.f;
+                }
+            }
+        }
+        if (tid < ti.valid)
+            part[static_cast<int64_t>(h) * part_stride + s.vis_off + ti.vis0 + tid] = acc;
+    }
+
+    // peers may still be reading this CTA's statistics
+    __syncthreads();
+    cluster_sync_all();
+    if constexpr (UMMA) {
+        tc_fence_before();
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+// ------------------------------------------------------------------ head reduce, L1 norms
+__global__ void head_reduce_kernel(const float* __restrict__ part, int64_t part_stride, int n_heads,
+                                   int total_vis, float* __restrict__ attn)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= total_vis) return;
+    float acc = 0.f;
+    for (int h = 0; h < n_heads; ++h) acc += part[static_cast<int64_t>(h) * part_stride + j];
+    attn[j] = acc;
+}
+
+// One warp per visual row; 16-byte loads; fixed reduction order.
+template <typename T>
+__global__ void __launch_bounds__(256)
+l1norm_kernel(const __grid_constant__ BatchDesc bd, int d_model, const T* __restrict__ hidden,
+              float* __restrict__ l1)
+{
+    const SampleDev& s = bd.s[blockIdx.y];
+    const int nv = s.n_2d + s.n_3d;
+    const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (j >= nv) return;
+    const int lane = threadIdx.x & 31;
+    const int row = s.seq_off + (j < s.n_2d ? s.off_2d + j : s.off_3d + (j - s.n_2d));
+    constexpr int kVec = 16 / sizeof(T);
+    const uint4* src = reinterpret_cast<const uint4*>(hidden + static_cast<int64_t>(row) * d_model);
+    const int nvec = d_model / kVec;
+    float acc = 0.f;
+    for (int i = lane; i < nvec; i += 32) {
+        const uint4 u = __ldg(src + i);
+        if constexpr (sizeof(T) == 2) {
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                acc += fabsf(__uint_as_float(w[e] << 16));           // low bf16
+                acc += fabsf(__uint_as_float(w[e] & 0xFFFF0000u));   // high bf16
+            }
+        } else {
+            acc += fabsf(__uint_as_float(u.x)) + fabsf(__uint_as_float(u.y)) +
+                   fabsf(__uint_as_float(u.z)) + fabsf(__uint_as_float(u.w));
+        }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (lane == 0) l1[s.vis_off + j] = acc;
+}
+
+template <typename T, bool UMMA>
+cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int head_dim, const void* q, const void* k,
+                              const CUtensorMap* tq, const CUtensorMap* tk, int tiles_per_cta, int cluster,
+                              int npad, float* part, int64_t part_stride, int* status, cudaStream_t stream)
+{
+    size_t smem;
+    if (UMMA)
+        smem = 1024 + static_cast<size_t>(head_dim / 64) * (static_cast<size_t>(tiles_per_cta) * 16384 + npad * 128);
+    else
+        smem = 1024 + sizeof(float) * (static_cast<size_t>(npad) * head_dim + kKeyTile * (head_dim + 1) +
+                                static_cast<size_t>(tiles_per_cta) * npad * kKeyTile);
+    if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
+    auto kern = salience_kernel<T, UMMA>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cluster, n_heads, bd.n);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    static const CUtensorMap zero_map = {};
+    return cudaLaunchKernelEx(&cfg, kern, bd, tq ? *tq : zero_map, tk ? *tk : zero_map,
+                              static_cast<const T*>(q), static_cast<const T*>(k), n_heads, head_dim,
+                              tiles_per_cta, npad, part, part_stride, status);
+}
+
+}  // namespace
+
+cudaError_t launch_salience(const BatchDesc& bd, int dtype, int n_heads, int head_dim, const void* q,
+                            const void* k, const CUtensorMap* tmap_q, const CUtensorMap* tmap_k,
+                            bool use_umma, int tiles_per_cta, int cluster, int npad, float* part,
+                            int64_t part_stride, int* status, cudaStream_t stream)
+{
+    if (dtype == MVLA_DTYPE_BF16) {
+        if (use_umma)
+            return launch_salience_t<__nv_bfloat16, true>(bd, n_heads, head_dim, q, k, tmap_q, tmap_k, tiles_per_cta,
+                                                          cluster, npad, part, part_stride, status, stream);
+        return launch_salience_t<__nv_bfloat16, false>(bd, n_heads, head_dim, q, k, nullptr, nullptr, tiles_per_cta,
+                                                       cluster, npad, part, part_stride, status, stream);
+    }
+    return launch_salience_t<float, false>(bd, n_heads, head_dim, q, k, nullptr, nullptr, tiles_per_cta, cluster,
+                                           npad, part, part_stride, status, stream);
+}
+
+cudaError_t launch_head_reduce(const float* part, int64_t part_stride, int n_heads, int total_vis, float* attn,
+                               cudaStream_t stream)
+{
+    if (total_vis <= 0) return cudaSuccess;
+    head_reduce_kernel<<<(total_vis + 255) / 256, 256, 0, stream>>>(part, part_stride, n_heads, total_vis, attn);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_l1norm(const BatchDesc& bd, int dtype, int d_model, const void* hidden, float* l1,
+                          cudaStream_t stream)
+{
+    int max_nv = 0;
+    for (int b = 0; b < bd.n; ++b) max_nv = max(max_nv, bd.s[b].n_2d + bd.s[b].n_3d);
+    if (max_nv == 0) return cudaSuccess;
+    const dim3 grid((max_nv + 7) / 8, bd.n);
+    if (dtype == MVLA_DTYPE_BF16)
+        l1norm_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(bd, d_model, static_cast<const __nv_bfloat16*>(hidden), l1);
+    else
+        l1norm_kernel<float><<<grid, 256, 0, stream>>>(bd, d_model, static_cast<const float*>(hidden), l1);
+    return cudaGetLastError();
+}
+
+}  // namespace mvla

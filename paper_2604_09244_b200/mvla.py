@@ -1,0 +1,279 @@
+"""Thin ctypes binding of ``libmvla_prune.so`` (see ``include/mvla_prune.h``).
+
+Argument marshalling only: every step of the prune path runs in the CUDA
+library.  PyTorch supplies device memory and streams.  There is no CPU
+fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmvla_prune.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_OOM, ERR_CUDA = -1, -2, -3, -4
+ERR_CAPACITY, ERR_TIMEOUT, ERR_STATE = -5, -6, -7
+_ERR_NAMES = {-1: "MVLA_ERR_INVALID_ARG", -2: "MVLA_ERR_UNSUPPORTED", -3: "MVLA_ERR_OOM",
+              -4: "MVLA_ERR_CUDA", -5: "MVLA_ERR_CAPACITY", -6: "MVLA_ERR_TIMEOUT",
+              -7: "MVLA_ERR_STATE"}
+DTYPE_BF16, DTYPE_FP32 = 0, 1
+MODE_FIXED, MODE_ADAPTIVE = 0, 1
+FLAG_RESET_STATE, FLAG_NO_STATE_UPDATE = 1, 2
+SALIENCE_AUTO, SALIENCE_FMA = 0, 1
+SET_2D, SET_3D = 1, 2
+
+EXPORTS = ("mvla_prune_create", "mvla_salience", "mvla_select", "mvla_compact",
+           "mvla_prune_step", "mvla_prune_destroy")
+
+
+class MvlaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where} failed: {_ERR_NAMES.get(code, code)}")
+
+
+class Config(C.Structure):
+    _fields_ = [("device", C.c_int32), ("dtype", C.c_int32), ("n_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("d_model", C.c_int32), ("max_batch", C.c_int32),
+                ("max_text", C.c_int32), ("max_2d", C.c_int32), ("max_3d", C.c_int32),
+                ("n_prune_points", C.c_int32), ("n_state_slots", C.c_int32),
+                ("window_k", C.c_int32), ("cold_start_full_keep", C.c_int32),
+                ("salience_path", C.c_int32),
+                ("tau_2d", C.c_double), ("tau_3d", C.c_double), ("beta", C.c_double),
+                ("eps_3d", C.c_double), ("floor_ratio", C.c_double)]
+
+
+class CSample(C.Structure):
+    _fields_ = [("seq_off", C.c_int32), ("off_txt", C.c_int32), ("n_txt", C.c_int32),
+                ("off_2d", C.c_int32), ("n_2d", C.c_int32), ("off_3d", C.c_int32),
+                ("n_3d", C.c_int32), ("state_slot", C.c_int32),
+                ("keep_2d", C.c_double), ("keep_3d", C.c_double), ("keep_total", C.c_double)]
+
+
+class CDiag(C.Structure):
+    _fields_ = [("t", C.c_int32), ("c_s1", C.c_int32), ("c_s2", C.c_int32), ("c_final", C.c_int32),
+                ("budget", C.c_int32), ("k_2d", C.c_int32), ("k_3d", C.c_int32),
+                ("reserved", C.c_int32), ("x", C.c_float * 4), ("mhat", C.c_float * 4)]
+
+
+class CTensors(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("hidden", C.c_void_p),
+                ("rows", C.c_int64)]
+
+
+class COutputs(C.Structure):
+    _fields_ = [("out_hidden", C.c_void_p), ("out_k", C.c_void_p), ("out_v", C.c_void_p),
+                ("kept_idx", C.c_void_p), ("out_offsets", C.c_void_p), ("budgets", C.c_void_p),
+                ("attn", C.c_void_p), ("ahat", C.c_void_p), ("z", C.c_void_p), ("diag", C.c_void_p)]
+
+
+def load_library(path: str = LIB_PATH) -> C.CDLL:
+    if not os.path.exists(path):
+        raise OSError(f"{path} is missing: build it with `python -m paper_2604_09244_b200.build` "
+                      "(there is no fallback path)")
+    lib = C.CDLL(path)
+    vp, i32, u32, i64 = C.c_void_p, C.c_int32, C.c_uint32, C.c_int64
+    sp = C.POINTER(CSample)
+    lib.mvla_prune_create.argtypes = [C.POINTER(Config), C.POINTER(vp)]
+    lib.mvla_prune_create.restype = i32
+    lib.mvla_salience.argtypes = [vp, i32, sp, vp, vp, vp, i64, vp, vp, vp]
+    lib.mvla_salience.restype = i32
+    lib.mvla_select.argtypes = [vp, i32, i32, sp, i32, u32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.mvla_select.restype = i32
+    lib.mvla_compact.argtypes = [vp, i32, sp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.mvla_compact.restype = i32
+    lib.mvla_prune_step.argtypes = [vp, i32, i32, sp, i32, u32, C.POINTER(CTensors),
+                                    C.POINTER(COutputs), C.POINTER(i32), vp]
+    lib.mvla_prune_step.restype = i32
+    lib.mvla_prune_destroy.argtypes = [vp]
+    lib.mvla_prune_destroy.restype = None
+    return lib
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = load_library()
+    return _lib
+
+
+def c_samples(samples: Sequence) -> "C.Array[CSample]":
+    """From objects with the descriptor's field names (``workloads.Sample``)."""
+    arr = (CSample * len(samples))()
+    for i, s in enumerate(samples):
+        arr[i] = CSample(int(s.seq_off), int(s.off_txt), int(s.n_txt), int(s.off_2d), int(s.n_2d),
+                         int(s.off_3d), int(s.n_3d), int(getattr(s, "state_slot", 0)),
+                         float(s.keep_2d), float(s.keep_3d), float(s.keep_total))
+    return arr
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
+    return t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+@dataclass
+class StepOutputs:
+    """Caller-owned device buffers of one fused step (sized for the worst case)."""
+    out_hidden: Optional[torch.Tensor]
+    out_k: Optional[torch.Tensor]
+    out_v: Optional[torch.Tensor]
+    kept_idx: torch.Tensor
+    out_offsets: torch.Tensor
+    budgets: torch.Tensor
+    attn: Optional[torch.Tensor] = None
+    ahat: Optional[torch.Tensor] = None
+    z: Optional[torch.Tensor] = None
+    diag: Optional[torch.Tensor] = None   # int32 view of mvla_diag records, [batch, 16]
+    total_kept: int = 0
+
+
+class PruneContext:
+    """Owns one ``mvla_ctx``."""
+
+    def __init__(self, *, dtype: torch.dtype, n_heads: int, head_dim: int, d_model: int,
+                 max_batch: int, max_text: int, max_2d: int, max_3d: int, n_prune_points: int = 1,
+                 n_state_slots: int = 0, tau_2d: float = 0.08, tau_3d: float = 0.20,
+                 beta: float = 0.85, window_k: int = 7, eps_3d: float = 0.02,
+                 floor_ratio: float = 0.10, cold_start_full_keep: int = 1,
+                 salience_path: int = SALIENCE_AUTO, device: Optional[int] = None):
+        self._h = C.c_void_p()
+        self._lib = lib()
+        if device is None:
+            device = torch.cuda.current_device()
+        self.device = torch.device("cuda", device)
+        self.torch_dtype = dtype
+        code = {torch.bfloat16: DTYPE_BF16, torch.float32: DTYPE_FP32}[dtype]
+        self.cfg = Config(device, code, n_heads, head_dim, d_model, max_batch, max_text, max_2d,
+                          max_3d, n_prune_points, n_state_slots, window_k, cold_start_full_keep,
+                          salience_path, tau_2d, tau_3d, beta, eps_3d, floor_ratio)
+        rc = self._lib.mvla_prune_create(C.byref(self.cfg), C.byref(self._h))
+        if rc != OK:
+            self._h = C.c_void_p()
+            raise MvlaError(rc, "mvla_prune_create")
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            torch.cuda.synchronize(self.device)
+            self._lib.mvla_prune_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- allocation helpers (shapes only) ---------------------------------
+    def alloc_outputs(self, samples: Sequence, *, hidden=True, kv=True, extras=False) -> StepOutputs:
+        rows = sum(s.n_txt + s.n_2d + s.n_3d for s in samples)
+        nvis = sum(s.n_2d + s.n_3d for s in samples)
+        c, dev, dt = self.cfg, self.device, self.torch_dtype
+        mk = lambda *shape, dtype=dt: torch.empty(*shape, dtype=dtype, device=dev)
+        return StepOutputs(
+            out_hidden=mk(rows, c.d_model) if hidden else None,
+            out_k=mk(rows, c.n_heads, c.head_dim) if kv else None,
+            out_v=mk(rows, c.n_heads, c.head_dim) if kv else None,
+            kept_idx=mk(rows, dtype=torch.int32),
+            out_offsets=mk(len(samples) + 1, dtype=torch.int32),
+            budgets=mk(len(samples), 2, dtype=torch.int32),
+            attn=mk(nvis, dtype=torch.float32) if extras else None,
+            ahat=mk(nvis, dtype=torch.float32) if extras else None,
+            z=mk(nvis, dtype=torch.float32) if extras else None,
+            diag=torch.zeros(len(samples), 16, dtype=torch.int32, device=dev) if extras else None)
+
+    # -- the six entry points ----------------------------------------------
+    def salience(self, samples, q, k, hidden=None, *, attn_out=None, l1_out=None, stream=None):
+        cs = samples if isinstance(samples, C.Array) else c_samples(samples)
+        nvis = sum(s.n_2d + s.n_3d for s in cs)
+        if attn_out is None:
+            attn_out = torch.empty(nvis, dtype=torch.float32, device=self.device)
+        if hidden is not None and l1_out is None:
+            l1_out = torch.empty(nvis, dtype=torch.float32, device=self.device)
+        rc = self._lib.mvla_salience(self._h, len(cs), cs, _ptr(q), _ptr(k), _ptr(hidden), q.shape[0],
+                                     _ptr(attn_out), _ptr(l1_out), _stream(stream))
+        if rc != OK:
+            raise MvlaError(rc, "mvla_salience")
+        return attn_out, l1_out
+
+    def select(self, prune_point, samples, mode, attn, l1=None, *, flags=0, out: StepOutputs = None,
+               stream=None) -> StepOutputs:
+        cs = samples if isinstance(samples, C.Array) else c_samples(samples)
+        if out is None:
+            out = self.alloc_outputs(cs, hidden=False, kv=False, extras=True)
+        rc = self._lib.mvla_select(self._h, prune_point, len(cs), cs, mode, flags, _ptr(attn), _ptr(l1),
+                                   _ptr(out.kept_idx), _ptr(out.out_offsets), _ptr(out.budgets),
+                                   _ptr(out.ahat), _ptr(out.z), _ptr(out.diag), _stream(stream))
+        if rc != OK:
+            raise MvlaError(rc, "mvla_select")
+        return out
+
+    def compact(self, samples, kept_idx, out_offsets, total_kept, hidden=None, k=None, v=None, *,
+                out_hidden=None, out_k=None, out_v=None, stream=None):
+        cs = samples if isinstance(samples, C.Array) else c_samples(samples)
+        mk = lambda src: None if src is None else torch.empty((total_kept,) + tuple(src.shape[1:]),
+                                                              dtype=src.dtype, device=src.device)
+        out_hidden = mk(hidden) if out_hidden is None else out_hidden
+        out_k = mk(k) if out_k is None else out_k
+        out_v = mk(v) if out_v is None else out_v
+        rc = self._lib.mvla_compact(self._h, len(cs), cs, _ptr(kept_idx), _ptr(out_offsets), int(total_kept),
+                                    _ptr(hidden), _ptr(k), _ptr(v), _ptr(out_hidden), _ptr(out_k),
+                                    _ptr(out_v), _stream(stream))
+        if rc != OK:
+            raise MvlaError(rc, "mvla_compact")
+        return out_hidden, out_k, out_v
+
+    def prune_step(self, prune_point, samples, mode, q, k, v, hidden, *, flags=0,
+                   out: StepOutputs = None, stream=None) -> StepOutputs:
+        cs = samples if isinstance(samples, C.Array) else c_samples(samples)
+        if out is None:
+            out = self.alloc_outputs(cs, hidden=hidden is not None, kv=v is not None, extras=True)
+        tin = CTensors(_ptr(q), _ptr(k), _ptr(v), _ptr(hidden), q.shape[0])
+        tout = COutputs(_ptr(out.out_hidden), _ptr(out.out_k), _ptr(out.out_v), _ptr(out.kept_idx),
+                        _ptr(out.out_offsets), _ptr(out.budgets), _ptr(out.attn), _ptr(out.ahat),
+                        _ptr(out.z), _ptr(out.diag))
+        total = C.c_int32(0)
+        rc = self._lib.mvla_prune_step(self._h, prune_point, len(cs), cs, mode, flags, C.byref(tin),
+                                       C.byref(tout), C.byref(total), _stream(stream))
+        if rc != OK:
+            raise MvlaError(rc, "mvla_prune_step")
+        out.total_kept = total.value
+        return out
+
+
+def context_for(wl, *, max_batch=None, n_prune_points=1, salience_path=SALIENCE_AUTO,
+                device=None) -> PruneContext:
+    """A context sized for a synthetic workload (see ``workloads``)."""
+    dt = {"bf16": torch.bfloat16, "fp32": torch.float32}[wl.dtype]
+    return PruneContext(dtype=dt, n_heads=wl.n_heads, head_dim=wl.head_dim, d_model=wl.d_model,
+                        max_batch=max_batch or len(wl.samples),
+                        max_text=max(s.n_txt for s in wl.samples),
+                        max_2d=max(max(s.n_2d for s in wl.samples), 1),
+                        max_3d=max(max(s.n_3d for s in wl.samples), 1),
+                        n_prune_points=n_prune_points, tau_2d=wl.tau_2d, tau_3d=wl.tau_3d,
+                        beta=wl.beta, window_k=wl.window_k, eps_3d=wl.eps_3d,
+                        floor_ratio=wl.floor_ratio, cold_start_full_keep=wl.cold_start_full_keep,
+                        salience_path=salience_path, device=device)
+
+
+def to_device(arr, dtype: str, device) -> torch.Tensor:
+    """float32 numpy array holding dtype-exact values -> device tensor of that dtype."""
+    t = torch.from_numpy(arr)
+    if dtype == "bf16":
+        t = t.to(torch.bfloat16)      # exact: the values are already bf16-representable
+    return t.to(device).contiguous()

@@ -1,0 +1,283 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU oracle on the same
+seeded inputs.  Integer results (kept indices given identical scores, compacted rows) must be
+bit-exact; salience scores within 2e-3 relative (bf16 inputs, fp32 accumulate)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_09244_b200 import mvla
+from paper_2604_09244_b200 import workloads as W
+from parity_util import (assert_salience_close, check_compaction, device_tensors, diag_records,
+                         run_and_check_step)
+
+pytestmark = pytest.mark.gpu
+
+
+# ------------------------------------------------------------------ compaction
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_compact_bit_exact_ragged(dtype):
+    wl = W.small_workload(21, batch=3, D=264 if dtype == "bf16" else 260, H=3, d=64, dtype=dtype,
+                          n_txt=(5, 19, 1), n_2d=(70, 130, 3), n_3d=(150, 37, 9))
+    ctx = mvla.context_for(wl)
+    dev = device_tensors(wl)
+    rng = np.random.default_rng(0)
+    kept, offs = [], [0]
+    for s in wl.samples:
+        k = np.sort(rng.choice(s.seq_len, size=int(rng.integers(1, s.seq_len + 1)), replace=False))
+        kept.append(k.astype(np.int32))
+        offs.append(offs[-1] + len(k))
+    kept_d = torch.from_numpy(np.concatenate(kept)).cuda()
+    offs_d = torch.tensor(offs, dtype=torch.int32).cuda()
+    oh, ok, ov = ctx.compact(wl.samples, kept_d, offs_d, offs[-1], dev["hidden"], dev["k"], dev["v"])
+    torch.cuda.synchronize()
+
+    class Out:
+        out_hidden, out_k, out_v = oh, ok, ov
+    for b, s in enumerate(wl.samples):
+        check_compaction(wl.steps[0], Out, s, kept[b], offs[b], dtype)
+    # a skipped pair stays untouched
+    oh2, ok2, ov2 = ctx.compact(wl.samples, kept_d, offs_d, offs[-1], None, dev["k"], None)
+    assert oh2 is None and ov2 is None
+    torch.cuda.synchronize()
+    assert torch.equal(ok2, ok)
+    ctx.close()
+
+
+# ------------------------------------------------------------------ selection on given scores
+def test_select_exact_with_ties_and_edge_budgets():
+    rng = np.random.default_rng(5)
+    cases = [(40, 50, 0.5, 0.5), (1, 300, 1.0, 0.01), (257, 0, 0.3, 0.3), (0, 129, 0.0, 0.7),
+             (1000, 1500, 0.1, 0.9), (64, 64, 0.0, 0.0), (33, 95, 1.0, 1.0)]
+    for n2, n3, k2r, k3r in cases:
+        s = W.layout_2d_3d_txt(0, 7, n2, n3, keep_2d=k2r, keep_3d=k3r)
+        ctx = mvla.PruneContext(dtype=torch.float32, n_heads=2, head_dim=64, d_model=64, max_batch=1,
+                                max_text=8, max_2d=max(n2, 1), max_3d=max(n3, 1), cold_start_full_keep=0)
+        # few distinct values -> many exact ties at the k-th boundary
+        attn = rng.integers(1, 6, size=n2 + n3).astype(np.float32)
+        attn /= attn.sum()
+        out = ctx.select(0, [s], mvla.MODE_FIXED, torch.from_numpy(attn).cuda())
+        torch.cuda.synchronize()
+        k2, k3 = out.budgets.cpu().numpy()[0]
+        assert (k2, k3) == oracle.budget_fixed(s)
+        offs = out.out_offsets.cpu().numpy()
+        kept = out.kept_idx.cpu().numpy()[:offs[1]]
+        ref = oracle.select(oracle.normalise(attn.astype(np.float64), n2, n3), s, int(k2), int(k3))
+        assert np.array_equal(kept, ref), (n2, n3)
+        assert np.array_equal(out.ahat.cpu().numpy(), attn)
+        ctx.close()
+
+
+def test_select_text_first_and_negative_scores():
+    s = W.Sample(seq_off=0, off_txt=0, n_txt=3, off_2d=3, n_2d=200, off_3d=203, n_3d=77,
+                 keep_2d=0.25, keep_3d=0.5)
+    ctx = mvla.PruneContext(dtype=torch.float32, n_heads=2, head_dim=64, d_model=64, max_batch=1, max_text=8,
+                            max_2d=200, max_3d=77, cold_start_full_keep=0)
+    rng = np.random.default_rng(1)
+    attn = rng.standard_normal(277).astype(np.float32)          # the ordering must hold for any sign
+    out = ctx.select(0, [s], mvla.MODE_FIXED, torch.from_numpy(attn).cuda())
+    torch.cuda.synchronize()
+    kept = out.kept_idx.cpu().numpy()[:out.out_offsets.cpu().numpy()[1]]
+    ref = oracle.select(attn.astype(np.float64), s, 50, 39)
+    assert np.array_equal(kept, ref)
+    ctx.close()
+
+
+# ------------------------------------------------------------------ salience
+@pytest.mark.parametrize("dtype,path", [("fp32", mvla.SALIENCE_AUTO), ("bf16", mvla.SALIENCE_FMA),
+                                        ("bf16", mvla.SALIENCE_AUTO)])
+@pytest.mark.parametrize("text_first", [False, True])
+def test_salience_small_ragged(dtype, path, text_first):
+    wl = W.small_workload(31, batch=3, D=256, H=4, d=64 if dtype == "fp32" else 128, dtype=dtype,
+                          n_txt=(5, 19, 33), n_2d=(70, 130, 1), n_3d=(150, 37, 300), text_first=text_first)
+    ctx = mvla.context_for(wl, salience_path=path)
+    dev = device_tensors(wl)
+    attn, l1 = ctx.salience(wl.samples, dev["q"], dev["k"], dev["hidden"])
+    torch.cuda.synchronize()
+    attn, l1 = attn.cpu().numpy(), l1.cpu().numpy()
+    t = wl.steps[0]
+    vis = 0
+    for s in wl.samples:
+        ref = oracle.salience(t.q, t.k, wl.n_heads, wl.head_dim, s)
+        assert_salience_close(attn[vis:vis + s.n_vis], ref)
+        assert abs(attn[vis:vis + s.n_vis].sum() - 1.0) < 1e-4
+        np.testing.assert_allclose(l1[vis:vis + s.n_vis], oracle.l1norm(t.hidden, wl.d_model, s), rtol=1e-5)
+        vis += s.n_vis
+    ctx.close()
+
+
+def test_salience_many_tiles_and_max_text():
+    # 2500 keys -> 21 tiles -> 3 tiles per CTA in a cluster of 7; 64 text queries (the maximum)
+    wl = W.small_workload(32, batch=1, D=128, H=2, d=128, dtype="bf16", n_txt=(64,), n_2d=(1100,), n_3d=(1400,))
+    for path in (mvla.SALIENCE_AUTO, mvla.SALIENCE_FMA):
+        ctx = mvla.context_for(wl, salience_path=path)
+        dev = device_tensors(wl)
+        attn, _ = ctx.salience(wl.samples, dev["q"], dev["k"])
+        torch.cuda.synchronize()
+        t = wl.steps[0]
+        assert_salience_close(attn.cpu().numpy(), oracle.salience(t.q, t.k, 2, 128, wl.samples[0]))
+        ctx.close()
+
+
+def test_tensor_core_and_fma_paths_agree():
+    wl = W.config2_single_frame(seed=7)
+    dev = device_tensors(wl)
+    res = []
+    for path in (mvla.SALIENCE_AUTO, mvla.SALIENCE_FMA):
+        ctx = mvla.context_for(wl, salience_path=path)
+        attn, _ = ctx.salience(wl.samples, dev["q"], dev["k"])
+        torch.cuda.synchronize()
+        res.append(attn.cpu().numpy())
+        ctx.close()
+    np.testing.assert_allclose(res[0], res[1], rtol=1e-4, atol=1e-9)
+
+
+# ------------------------------------------------------------------ the fused step on the five workloads
+def _fresh_states(wl):
+    return [oracle.State(s.n_vis) for s in wl.samples]
+
+
+def test_step_config1_tiny_fp32():
+    wl = W.config1_tiny()
+    ctx = mvla.context_for(wl)
+    out, refs = run_and_check_step(ctx, wl, 0, _fresh_states(wl))
+    kept = out.kept_idx.cpu().numpy()[:out.total_kept]
+    assert np.array_equal(kept, refs[0].kept_idx)
+    ctx.close()
+
+
+@pytest.mark.parametrize("seed", [1, 11, 12, 13])
+def test_step_config2_single_frame(seed):
+    wl = W.config2_single_frame(seed=seed)
+    ctx = mvla.context_for(wl)
+    out, refs = run_and_check_step(ctx, wl, 0, _fresh_states(wl))
+    assert tuple(out.budgets.cpu().numpy()[0]) == (102, 154)
+    assert out.total_kept == 288
+    ctx.close()
+
+
+@pytest.mark.parametrize("seed", [2, 21])
+def test_step_config3_multi_view_two_points(seed):
+    wl = W.config3_multi_view(seed=seed)
+    ctx = mvla.context_for(wl, n_prune_points=2)
+    out, refs = run_and_check_step(ctx, wl, 0, _fresh_states(wl), prune_point=0)
+    assert out.total_kept == 48 + 448
+    # second point: the generator re-projects the rows the ORACLE kept at the first point
+    r = refs[0]
+    wl2 = W.config3_second_point(wl, r.kept_idx, r.k_2d, r.k_3d)
+    out2, refs2 = run_and_check_step(ctx, wl2, 0, _fresh_states(wl2), prune_point=1)
+    assert out2.total_kept == 48 + 112
+    ctx.close()
+
+
+def test_step_config4_batched_serving():
+    wl = W.config4_batched()
+    ctx = mvla.context_for(wl)
+    out, refs = run_and_check_step(ctx, wl, 0, _fresh_states(wl))
+    offs = out.out_offsets.cpu().numpy()
+    assert len(offs) == 17 and (np.diff(offs) > 0).all()
+    ctx.close()
+
+
+def test_step_config5_action_iteration():
+    wl = W.config5_action_iteration()
+    ctx = mvla.context_for(wl)
+    states = _fresh_states(wl)
+    s = wl.samples[0]
+    for t in range(len(wl.steps)):
+        out, refs = run_and_check_step(ctx, wl, t, states, flags=mvla.FLAG_RESET_STATE if t == 0 else 0)
+        if t == 0:
+            assert out.total_kept == s.seq_len                       # cold start keeps everything
+            assert np.array_equal(out.kept_idx.cpu().numpy()[:s.seq_len], np.arange(s.seq_len))
+        else:
+            assert out.total_kept == s.n_txt + 384
+        assert diag_records(out, 1)[0]["t"] == t + 1
+    ctx.close()
+
+
+def test_step_small_ragged_batch_with_state_and_dry_run():
+    wl = W.small_workload(41, batch=3, D=256, H=4, d=128, dtype="bf16", n_txt=(5, 19, 33),
+                          n_2d=(70, 130, 260), n_3d=(150, 37, 300), keep=(0.4, 0.3, 0.55), steps=9,
+                          cold_start=1)
+    ctx = mvla.context_for(wl)
+    states = _fresh_states(wl)
+    for t in range(9):                                                # crosses the Eq. 8 -> Eq. 9 switch at t = 7
+        out, refs = run_and_check_step(ctx, wl, t, states)
+        if t == 3:                                                    # a dry run leaves state and t untouched
+            dev = device_tensors(wl, t)
+            dry = ctx.prune_step(0, wl.samples, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"],
+                                 flags=mvla.FLAG_NO_STATE_UPDATE)
+            torch.cuda.synchronize()
+            assert diag_records(dry, 3)[0]["t"] == 5
+    ctx.close()
+
+
+@pytest.mark.parametrize("scale,expect", [(0.05, mvla.SET_2D), (0.136, mvla.SET_2D | mvla.SET_3D), (0.30, mvla.SET_3D)])
+def test_paper_default_thresholds_all_three_branches(scale, expect):
+    # 3D hidden rows scaled by s give a feature-norm share of about s/(1+s): 0.048, 0.12, 0.23 against
+    # the paper's default thresholds 0.08 / 0.20
+    wl = W.small_workload(51, batch=1, D=512, H=4, d=128, dtype="bf16", n_txt=(9,), n_2d=(200,), n_3d=(280,),
+                          keep=(0.35,), scale_3d=scale, spike_frac=0.0)
+    wl.tau_2d, wl.tau_3d = 0.08, 0.20
+    ctx = mvla.context_for(wl)
+    out, refs = run_and_check_step(ctx, wl, 0, _fresh_states(wl))
+    assert diag_records(out, 1)[0]["c_s1"] == expect == refs[0].c_s1
+    ctx.close()
+
+
+def test_results_are_deterministic():
+    wl = W.config2_single_frame(seed=3)
+    ctx = mvla.context_for(wl)
+    dev = device_tensors(wl)
+    outs = []
+    for _ in range(3):
+        o = ctx.prune_step(0, wl.samples, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"],
+                           flags=mvla.FLAG_RESET_STATE)
+        torch.cuda.synchronize()
+        outs.append((o.attn.clone(), o.kept_idx.clone(), o.out_hidden.clone()))
+    for a in outs[1:]:
+        assert all(torch.equal(x, y) for x, y in zip(a, outs[0]))
+    ctx.close()
+
+
+# ------------------------------------------------------------------ boundary behaviour
+def test_error_codes_never_fault():
+    wl = W.small_workload(61, batch=2, D=256, H=4, d=128, dtype="bf16")
+    ctx = mvla.context_for(wl)
+    dev = device_tensors(wl)
+    good = list(wl.samples)
+
+    def code(fn):
+        with pytest.raises(mvla.MvlaError) as e:
+            fn()
+        return e.value.code
+
+    import copy
+    bad = copy.deepcopy(good); bad[0].n_txt = 0
+    assert code(lambda: ctx.salience(bad, dev["q"], dev["k"])) == mvla.ERR_INVALID_ARG
+    bad = copy.deepcopy(good); bad[0].off_3d = bad[0].off_2d          # overlapping segments
+    assert code(lambda: ctx.salience(bad, dev["q"], dev["k"])) == mvla.ERR_INVALID_ARG
+    bad = copy.deepcopy(good); bad[1].n_2d = 10 ** 6
+    assert code(lambda: ctx.salience(bad, dev["q"], dev["k"])) == mvla.ERR_CAPACITY
+    bad = copy.deepcopy(good); bad[1].seq_off = 10 ** 6               # beyond the rows given
+    assert code(lambda: ctx.salience(bad, dev["q"], dev["k"])) == mvla.ERR_INVALID_ARG
+    bad = copy.deepcopy(good); bad[1].state_slot = bad[0].state_slot  # two writers of one state
+    assert code(lambda: ctx.prune_step(0, bad, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"])) == mvla.ERR_STATE
+    assert code(lambda: ctx.prune_step(3, good, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"])) == mvla.ERR_STATE
+    assert code(lambda: ctx.prune_step(0, good, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"], flags=8)) == mvla.ERR_INVALID_ARG
+    assert code(lambda: ctx.prune_step(0, good * 2, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"])) == mvla.ERR_CAPACITY
+    misaligned = dev["q"].view(-1)[1:1 + dev["q"].numel() - 8].contiguous()
+    # .contiguous() of a slice is a fresh allocation, so build a truly misaligned pointer by hand
+    import ctypes as C
+    cs = mvla.c_samples(good)
+    rc = ctx._lib.mvla_salience(ctx._h, 2, cs, dev["q"].data_ptr() + 2, dev["k"].data_ptr(), None,
+                                dev["q"].shape[0], torch.empty(1000, device="cuda").data_ptr(), None, 0)
+    assert rc == mvla.ERR_INVALID_ARG
+    # the context is still usable afterwards
+    ctx.prune_step(0, good, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"])
+    torch.cuda.synchronize()
+    ctx.close()
+    with pytest.raises(mvla.MvlaError) as e:
+        mvla.PruneContext(dtype=torch.bfloat16, n_heads=4, head_dim=96, d_model=256, max_batch=1, max_text=8,
+                          max_2d=8, max_3d=8)
+    assert e.value.code == mvla.ERR_UNSUPPORTED
