@@ -1,0 +1,392 @@
+#!/usr/bin/env python
+"""Benchmark of the MVLA prune step (salience -> carry-over/budget -> top-k select -> compaction).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A "step" is one fused prune step (`mvla_prune_step` through the C ABI) over one batch of seeded
+synthetic input.  The default workload is the 7B-shaped single frame (32 text + 256 2D + 512 3D
+tokens, D=4096, 32 heads x 128, bf16, keep 40 % / 30 %).  Prints ONE JSON line.
+
+* `value`: visual tokens pruned per second, whole job, inputs resident in HBM.  The steps are
+  captured in CUDA graphs (one step per rotated input set) and replayed; CUDA events bracket the
+  K timed steps; inputs rotate over enough distinct sets to exceed L2.
+* `e2e`: the same metric with the step's inputs copied from pinned host memory and its results
+  copied back inside the timed region.
+* `roofline`: the dominant kernel's stage timed alone through its own C-ABI entry point.
+* `cpu_baseline` / `--impl reference`: the fp64 CPU oracle, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+L2_BYTES = 126 * 1024 * 1024
+HBM_FALLBACK_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------- helpers
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": HBM_FALLBACK_GBS}, "fallback"
+
+
+def make_workload(name: str):
+    from paper_2604_09244_b200 import workloads as W
+    if name == "config2":
+        return W.config2_single_frame(), "configs[1]: 7B-shaped single frame, batch 1, D=4096, 32 heads x 128, " \
+                                         "32 text + 256 2D + 512 3D tokens, bf16, FIXED keep 2D 40 % / 3D 30 %"
+    if name == "config1":
+        return W.config1_tiny(), "configs[0]: tiny reference, fp32"
+    if name == "config3":
+        return W.config3_multi_view(), "configs[2]: multi-view, first prune point, adaptive keep 25 %"
+    if name == "config4":
+        return W.config4_batched(), "configs[3]: batched serving, batch 16, adaptive per-sample keep"
+    if name == "config5":
+        return W.config5_action_iteration(T=2), "configs[4]: action iteration, one step (t=2), adaptive keep 30 %"
+    raise SystemExit(f"unknown workload {name}")
+
+
+def algorithmic_bytes(wl, kept_rows: int):
+    """Bytes the method must move per step (read K and Q of the visual/text rows, read hidden for the
+    norms in ADAPTIVE mode, read+write the kept rows of hidden/K/V, ~12 bytes of scores per token)."""
+    e = 2 if wl.dtype == "bf16" else 4
+    hd = wl.n_heads * wl.head_dim
+    nv = wl.total_vis
+    nt = sum(s.n_txt for s in wl.samples)
+    sal = (nv + nt) * hd * e
+    l1 = nv * wl.d_model * e if wl.mode == 1 else 0
+    comp = 2 * kept_rows * (wl.d_model + 2 * hd) * e
+    return {"salience": sal, "l1": l1, "compact": comp, "scores": 12 * nv,
+            "total": sal + l1 + comp + 12 * nv}
+
+
+class ClockSampler:
+    """SM clock and throttle reasons sampled (read only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40,
+                 "sw_thermal_slowdown": 0x20, "hw_power_brake_slowdown": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr:
+            self._thr.join(timeout=2)
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def time_oracle(wl, max_steps: int, max_seconds: float):
+    """The oracle as it stands: full prune steps (all samples) + compaction of hidden/K/V, repeated
+    `max_steps` times or until `max_seconds` of CPU work.  Returns (seconds per step, steps, cores)."""
+    import numpy as np
+    import oracle
+    t = wl.steps[-1]
+    p = oracle.params_of(wl)
+    n = 0
+    t0 = time.perf_counter()
+    while True:
+        for s in wl.samples:
+            st = oracle.State(s.n_vis)
+            r = oracle.prune_step(t.q, t.k, t.hidden if wl.mode == 1 else None, wl.n_heads, wl.head_dim,
+                                  wl.d_model, s, p, wl.mode, st)
+            for src in (t.hidden, t.k, t.v):
+                oracle.compact(src, s.seq_off, r.kept_idx)
+        n += 1
+        el = time.perf_counter() - t0
+        if el >= max_seconds or n >= max_steps:
+            break
+    cores = min(oracle.num_threads(), wl.n_heads, len(os.sched_getaffinity(0)))
+    return el / n, n, cores
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    wl, desc = make_workload(args.workload)
+    # warm-up then K timed oracle steps
+    time_oracle(wl, max(1, args.warmup), 30.0)
+    sec, n, cores = time_oracle(wl, args.steps, 150.0)     # bounded: at most about 2.5 minutes
+    val = wl.total_vis / sec
+    line = {"impl": "reference", "metric": "visual_tokens_per_s_pruned", "value": val, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": n, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+            "latency_us": sec * 1e6, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": desc, "note": "fp64 CPU oracle on host cores; each step is one full prune step"},
+            "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                             "sample": f"{n} full prune steps of the workload (all samples, all stages)"},
+            "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def run_ours(args, rank, local, world):
+    import numpy as np
+    import torch
+    from paper_2604_09244_b200 import dist as D
+    from paper_2604_09244_b200 import mvla
+
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    wl, desc = make_workload(args.workload)
+    step_t = wl.steps[-1]
+    names = ("q", "k", "v", "hidden")
+    host = {n: (torch.from_numpy(getattr(step_t, n)).to(torch.bfloat16) if wl.dtype == "bf16"
+                else torch.from_numpy(getattr(step_t, n))).contiguous() for n in names}
+    in_bytes = sum(t.numel() * t.element_size() for t in host.values())
+
+    ctx = mvla.context_for(wl)
+    probe = ctx.alloc_outputs(wl.samples, extras=False)
+    out_bytes_alloc = sum(t.numel() * t.element_size() for t in (probe.out_hidden, probe.out_k, probe.out_v))
+    n_sets = max(4, int(np.ceil(1.5 * L2_BYTES / (in_bytes + out_bytes_alloc))))
+    n_sets = min(n_sets, 64)
+    # distinct input sets: same values, distinct addresses (the cache cannot tell values apart)
+    sets = [{n: host[n].to(dev) for n in names} for _ in range(n_sets)]
+    outs = [probe] + [ctx.alloc_outputs(wl.samples, extras=False) for _ in range(n_sets - 1)]
+    cs = mvla.c_samples(wl.samples)
+    flags = mvla.FLAG_RESET_STATE if not wl.cold_start_full_keep else 0
+    if wl.cold_start_full_keep:      # absorb the cold-start step so that the timed steps prune
+        ctx.prune_step(0, cs, wl.mode, sets[0]["q"], sets[0]["k"], sets[0]["v"], sets[0]["hidden"], out=outs[0])
+        flags = mvla.FLAG_NO_STATE_UPDATE
+
+    def step(i, stream=None):
+        s, o = sets[i % n_sets], outs[i % n_sets]
+        return ctx.prune_step(0, cs, wl.mode, s["q"], s["k"], s["v"], s["hidden"], flags=flags, out=o, stream=stream)
+
+    o0 = step(0)
+    torch.cuda.synchronize()
+    kept_rows = o0.total_kept
+    launches_per_step = 3 + (1 if wl.mode == 1 else 0)
+
+    # ---- device-resident timing: graphs of n_sets steps
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for i in range(n_sets):
+            step(i)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(n_sets):
+            step(i)
+    replays = max(1, int(np.ceil(args.steps / n_sets)))
+    warm_replays = max(1, int(np.ceil(max(3, args.warmup) / n_sets)))
+    K = replays * n_sets
+    for _ in range(warm_replays):
+        graph.replay()
+    torch.cuda.synchronize()
+    D.barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clk:
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(replays):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+    D.barrier(world)
+    ms = D.max_over_ranks(e0.elapsed_time(e1), world, dev)
+    ms_per_step = ms / K
+    tokens_per_step = wl.total_vis * world
+    value = tokens_per_step / (ms_per_step * 1e-3)
+
+    # ---- isolated latency: one step at a time, synchronised (no overlap between steps)
+    lat = []
+    for i in range(64):
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        step(i)
+        b.record()
+        torch.cuda.synchronize()
+        lat.append(a.elapsed_time(b) * 1e3)
+    lat.sort()
+
+    # ---- per-stage timing through the stage entry points (graphs, rotating sets)
+    attn_b = [torch.empty(wl.total_vis, dtype=torch.float32, device=dev) for _ in range(n_sets)]
+    l1_b = [torch.empty(wl.total_vis, dtype=torch.float32, device=dev) for _ in range(n_sets)]
+    adaptive = wl.mode == 1
+
+    def st_salience(i):
+        s = sets[i % n_sets]
+        ctx.salience(cs, s["q"], s["k"], s["hidden"] if adaptive else None, attn_out=attn_b[i % n_sets],
+                     l1_out=l1_b[i % n_sets] if adaptive else None)
+
+    def st_select(i):
+        ctx.select(0, cs, wl.mode, attn_b[i % n_sets], l1_b[i % n_sets] if adaptive else None, flags=flags,
+                   out=outs[i % n_sets])
+
+    def st_compact(i):
+        s, o = sets[i % n_sets], outs[i % n_sets]
+        ctx.compact(cs, o.kept_idx, o.out_offsets, kept_rows, s["hidden"], s["k"], s["v"],
+                    out_hidden=o.out_hidden, out_k=o.out_k, out_v=o.out_v)
+
+    stage_us = {}
+    for name, fn in (("salience", st_salience), ("select", st_select), ("compact", st_compact)):
+        for i in range(n_sets):
+            fn(i)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(n_sets):
+                fn(i)
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = max(1, replays // 2)
+        a.record()
+        for _ in range(reps):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        stage_us[name] = a.elapsed_time(b) * 1e3 / (reps * n_sets)
+
+    # ---- end to end: pinned host inputs -> device, step, results -> pinned host
+    pin_in = {n: host[n].pin_memory() for n in names}
+    stage_in = {n: torch.empty_like(host[n], device=dev) for n in names}
+    o = outs[0]
+    res_dev = [o.out_hidden[:kept_rows], o.out_k[:kept_rows], o.out_v[:kept_rows], o.kept_idx[:kept_rows],
+               o.out_offsets, o.budgets]
+    res_host = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in res_dev]
+    h2d = in_bytes
+    d2h = sum(t.numel() * t.element_size() for t in res_dev)
+
+    def e2e_step():
+        for n in names:
+            stage_in[n].copy_(pin_in[n], non_blocking=True)
+        ctx.prune_step(0, cs, wl.mode, stage_in["q"], stage_in["k"], stage_in["v"], stage_in["hidden"],
+                       flags=flags, out=o)
+        for dst, src in zip(res_host, res_dev):
+            dst.copy_(src, non_blocking=True)
+
+    e2e_steps = max(20, min(args.steps, 400))
+    for _ in range(5):
+        e2e_step()
+    torch.cuda.synchronize()
+    D.barrier(world)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    b.record()
+    torch.cuda.synchronize()
+    e2e_ms = D.max_over_ranks(a.elapsed_time(b), world, dev) / e2e_steps
+    e2e_value = tokens_per_step / (e2e_ms * 1e-3)
+
+    if rank != 0:
+        return
+    peaks, peak_kind = measured_peaks()
+    ab = algorithmic_bytes(wl, kept_rows)
+    stage_bytes = {"salience": ab["salience"] + ab["l1"], "select": ab["scores"], "compact": ab["compact"]}
+    dom = max(stage_us, key=stage_us.get)
+    achieved = stage_bytes[dom] / (stage_us[dom] * 1e-6) / 1e9
+    roof = {"bound": "hbm", "kernel": {"salience": "salience_kernel", "select": "select_kernel",
+                                        "compact": "compact_kernel"}[dom],
+            "achieved": achieved, "peak": peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+            "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+            "bytes_per_launch": stage_bytes[dom], "us_per_launch": stage_us[dom]}
+    step_gbs = ab["total"] / (ms_per_step * 1e-3) / 1e9
+
+    cpu_sec, cpu_n, cores = time_oracle(wl, 10 ** 6, 10.0)
+    line = {"metric": "visual_tokens_per_s_pruned", "value": value, "unit": "tokens/s", "n_gpus": world,
+            "steps": K, "warmup": warm_replays * n_sets, "ms_per_step": ms_per_step,
+            "latency_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": wl.dtype if wl.dtype != "fp32" else "f32", "data": "synthetic",
+            "config": {"workload": desc, "l2": f"inputs and outputs rotate over {n_sets} distinct sets "
+                                               f"({(in_bytes + out_bytes_alloc) * n_sets / 2**20:.0f} MiB > L2)",
+                       "timing": "CUDA events around CUDA-graph replays of back-to-back steps",
+                       "kept_rows": kept_rows, "parallelism": f"replicas x{world}"},
+            "clocks": clk.summary(),
+            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms},
+            "gpu_launches": K * launches_per_step,
+            "roofline": roof,
+            "step_hbm": {"algorithmic_bytes": ab["total"], "achieved_gbs": step_gbs,
+                         "frac_of_peak": step_gbs / peaks["hbm_gbs"], "peak_kind": peak_kind},
+            "isolated_latency_us": {"p10": lat[6], "median": lat[32], "p90": lat[57]},
+            "stage_us": stage_us,
+            "cpu_baseline": {"value": wl.total_vis / cpu_sec, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                             "sample": f"{cpu_n} full prune steps of the same workload in {cpu_sec * cpu_n:.1f} s",
+                             "ms_per_step": cpu_sec * 1e3}}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config2")
+    args = ap.parse_args()
+
+    if args.impl == "reference":
+        rank = int(os.environ.get("RANK", 0))
+        if args.steps == 20000:          # the GPU arm's default; the CPU oracle needs far fewer
+            args.steps, args.warmup = 100, 3
+        run_reference(args, rank)
+        return
+    from paper_2604_09244_b200 import dist as D
+    rank, local, world = D.init("nccl")
+    try:
+        run_ours(args, rank, local, world)
+    finally:
+        import torch.distributed as dist
+        if dist.is_initialized():
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -94,8 +94,14 @@ def lib():
                                         C.c_int32, C.POINTER(CState), ip, C.POINTER(CDiag),
                                         dp, dp, dp, dp]
         L.oracle_prune_step.restype = C.c_int32
+        L.oracle_num_threads.argtypes = []
+        L.oracle_num_threads.restype = C.c_int32
         _lib = L
     return _lib
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
 
 
 # --------------------------------------------------------------------------

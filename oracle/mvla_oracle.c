@@ -300,3 +300,11 @@ int32_t oracle_prune_step(const float *q, const float *k, const float *hidden,
     free(a); free(z); free(l1);
     return n_kept;
 }
+
+/* Threads the head loop of oracle_salience may use (reporting only). */
+#ifdef _OPENMP
+#include <omp.h>
+int32_t oracle_num_threads(void) { return (int32_t)omp_get_max_threads(); }
+#else
+int32_t oracle_num_threads(void) { return 1; }
+#endif

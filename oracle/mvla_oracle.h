@@ -125,6 +125,9 @@ int32_t oracle_prune_step(const float *q, const float *k, const float *hidden,
                           oracle_state *st, int32_t *kept_idx, oracle_diag *diag,
                           double *attn_out, double *l1_out, double *ahat_out, double *z_out);
 
+/* Threads the head loop of oracle_salience may use (reporting only). */
+int32_t oracle_num_threads(void);
+
 #ifdef __cplusplus
 }
 #endif

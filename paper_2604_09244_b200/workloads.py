@@ -133,11 +133,12 @@ def layout_2d_3d_txt(seq_off: int, n_txt: int, n_2d: int, n_3d: int, **kw) -> Sa
 # --------------------------------------------------------------------------
 # drawing
 # --------------------------------------------------------------------------
-def _draw_weights(rng: np.random.Generator, D: int):
+def _draw_weights(rng: np.random.Generator, D: int, out: int = 0):
+    out = out or D          # projection width H*d (equal to D in the paper-shaped workloads)
     std = 1.0 / np.sqrt(D)
-    wq = rng.standard_normal((D, D), dtype=np.float32) * np.float32(std)
-    wk = rng.standard_normal((D, D), dtype=np.float32) * np.float32(std)
-    wv = rng.standard_normal((D, D), dtype=np.float32) * np.float32(std)
+    wq = rng.standard_normal((D, out), dtype=np.float32) * np.float32(std)
+    wk = rng.standard_normal((D, out), dtype=np.float32) * np.float32(std)
+    wv = rng.standard_normal((D, out), dtype=np.float32) * np.float32(std)
     return wq, wk, wv
 
 
@@ -333,7 +334,7 @@ def small_workload(seed: int, *, batch=2, D=256, H=4, d=64, dtype="bf16", mode=M
         samples.append(s)
         off += s.seq_len
     hidden = rng.standard_normal((off, D), dtype=np.float32)
-    w = _draw_weights(rng, D)
+    w = _draw_weights(rng, D, H * d)
     for s in samples:
         if spike_frac > 0:
             hidden[s.seq_off + _spike_rows(rng, s, spike_frac)] *= np.float32(4.0)

@@ -234,7 +234,8 @@ def test_results_are_deterministic():
         o = ctx.prune_step(0, wl.samples, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"],
                            flags=mvla.FLAG_RESET_STATE)
         torch.cuda.synchronize()
-        outs.append((o.attn.clone(), o.kept_idx.clone(), o.out_hidden.clone()))
+        n = o.total_kept                                            # rows past it are unwritten scratch
+        outs.append((o.attn.clone(), o.kept_idx[:n].clone(), o.out_hidden[:n].clone(), o.out_k[:n].clone()))
     for a in outs[1:]:
         assert all(torch.equal(x, y) for x, y in zip(a, outs[0]))
     ctx.close()
