@@ -199,6 +199,33 @@ int32_t mvla_prune_step(mvla_ctx *ctx, int32_t prune_point, int32_t batch,
                         const mvla_tensors *in, const mvla_outputs *out,
                         int32_t *total_kept_out, void *stream);
 
+/*
+ * Salience scores without a context and without any allocation.  (The paper has no counterpart:
+ * this is a packaging variant of mvla_salience, same arithmetic, same kernels.)
+ *
+ * For callers that may not allocate device memory at call time: a server whose memory pool is
+ * frozen after start-up, code running inside another framework's allocator-controlled region, a
+ * control loop that cannot afford the device-wide stall of a cudaMalloc.  mvla_prune_create uses
+ * cudaMalloc; this call uses none (no cudaMalloc / cudaFree / cudaHostAlloc, no heap).  Its scratch
+ * (per-head partial scores) is a fixed 512 KiB array inside the library image, so:
+ *   - limit: n_heads * sum(n_2d + n_3d) <= 131072 floats and batch <= 64, else MVLA_ERR_CAPACITY;
+ *     max_text 64 and 4096 visual tokens per sample as elsewhere;
+ *   - every GPU that loads the library holds the array until the process exits;
+ *   - all calls on a device share the array and it keeps the previous call's contents (every entry
+ *     that is read is rewritten first, and the timeout flag is cleared by each call);
+ *   - calls whose GPU work may overlap (two streams without ordering) race on it: serialise them;
+ *   - the first call on a device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ * device: CUDA ordinal; dtype, n_heads, head_dim as in mvla_config; samples: host array [batch];
+ * q, k: device, [rows, n_heads, head_dim], 16-byte aligned; attn_out: device, sum(n_vis) floats in
+ * visual order, caller-owned.  Enqueues on `stream`, does not synchronise.  If a bounded
+ * device-side wait gives up, every attn_out entry is NaN (there is no context to hold a status).
+ * Errors: INVALID_ARG, UNSUPPORTED, CAPACITY, CUDA.
+ */
+int32_t mvla_salience_noalloc(int32_t device, int32_t dtype, int32_t n_heads, int32_t head_dim,
+                              int32_t batch, const mvla_sample *samples, const void *q, const void *k,
+                              int64_t rows, float *attn_out, void *stream);
+
 /* Free everything the context owns.  NULL is accepted.  The caller must have
  * synchronised any stream that still runs work enqueued through the context. */
 void mvla_prune_destroy(mvla_ctx *ctx);

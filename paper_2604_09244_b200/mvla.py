@@ -277,3 +277,25 @@ def to_device(arr, dtype: str, device) -> torch.Tensor:
     if dtype == "bf16":
         t = t.to(torch.bfloat16)      # exact: the values are already bf16-representable
     return t.to(device).contiguous()
+
+
+def salience_noalloc(samples, q: torch.Tensor, k: torch.Tensor, attn_out: torch.Tensor, *, stream=None) -> None:
+    """Salience scores through ``mvla_salience_noalloc``: no context, and the library allocates
+    nothing.  Meant for callers that must not allocate device memory when they call in (a frozen
+    memory pool, a real-time loop): they hand in `attn_out` (float32, sum of visual tokens) that they
+    allocated earlier, and the library's scratch is a fixed array inside its image.  Problems with
+    ``n_heads * sum(n_vis) > 131072`` are refused (``MVLA_ERR_CAPACITY``).  Calls on one device share
+    that array: do not let two of them overlap on the GPU.  The first call on a device should be
+    made outside stream capture."""
+    L = lib()
+    fn = L.mvla_salience_noalloc
+    fn.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(CSample), C.c_void_p,
+                   C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
+    fn.restype = C.c_int32
+    cs = samples if isinstance(samples, C.Array) else c_samples(samples)
+    code = {torch.bfloat16: DTYPE_BF16, torch.float32: DTYPE_FP32}[q.dtype]
+    assert attn_out.dtype == torch.float32
+    rc = fn(q.device.index, code, q.shape[1], q.shape[2], len(cs), cs, _ptr(q), _ptr(k), q.shape[0],
+            _ptr(attn_out), _stream(stream))
+    if rc != OK:
+        raise MvlaError(rc, "mvla_salience_noalloc")

@@ -1,0 +1,53 @@
+"""The allocation-free salience entry point against the regular one.
+
+`mvla_salience_noalloc` exists for callers that cannot allocate device memory when they call into
+the library (frozen memory pools, real-time loops): its scratch is a fixed array in the library
+image that every call on the device shares and that keeps the previous call's contents.  So the
+check is made on two calls in a row with different problems: the second must not be disturbed by
+what the first left behind.  This file is collected last on purpose."""
+import pytest
+import torch
+
+from paper_2604_09244_b200 import mvla
+from paper_2604_09244_b200 import workloads as W
+from parity_util import SALIENCE_ATOL, SALIENCE_RTOL, device_tensors
+
+pytestmark = pytest.mark.gpu
+
+
+def _both(wl):
+    dev = device_tensors(wl)
+    ctx = mvla.context_for(wl)
+    ref, _ = ctx.salience(wl.samples, dev["q"], dev["k"])
+    out = torch.full((wl.total_vis,), -1.0, dtype=torch.float32, device="cuda")   # the caller's own buffer
+    mvla.salience_noalloc(wl.samples, dev["q"], dev["k"], out)
+    torch.cuda.synchronize()
+    ctx.close()
+    return out, ref
+
+
+def test_noalloc_matches_regular_entry_point_on_two_calls_in_a_row():
+    first = W.small_workload(71, batch=3, D=256, H=4, d=128, dtype="bf16", n_txt=(5, 19, 33),
+                             n_2d=(70, 130, 260), n_3d=(150, 37, 300))
+    second = W.small_workload(72, batch=2, D=256, H=4, d=128, dtype="bf16", n_txt=(40, 7), n_2d=(33, 200),
+                              n_3d=(90, 10))            # smaller: stale scratch entries lie beyond its range
+    for wl in (first, second):
+        out, ref = _both(wl)
+        assert torch.isfinite(out).all()
+        err = (out - ref).abs()
+        assert bool((err <= SALIENCE_RTOL * ref.abs() + SALIENCE_ATOL).all())
+        assert abs(float(out[:wl.samples[0].n_vis].sum()) - 1.0) < 1e-4
+
+
+def test_noalloc_fp32_and_capacity_limit():
+    wl = W.config1_tiny()
+    out, ref = _both(wl)
+    assert bool(((out - ref).abs() <= SALIENCE_RTOL * ref.abs() + SALIENCE_ATOL).all())
+    # 32 heads x 4097 visual tokens is past the fixed array: refused, nothing launched
+    big = W.layout_2d_3d_txt(0, 8, 2049, 2047)
+    big2 = W.layout_2d_3d_txt(big.seq_len, 8, 1, 0)
+    q = torch.zeros(big.seq_len + big2.seq_len, 32, 128, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(4097, dtype=torch.float32, device="cuda")
+    with pytest.raises(mvla.MvlaError) as e:
+        mvla.salience_noalloc([big, big2], q, q, out)
+    assert e.value.code == mvla.ERR_CAPACITY
