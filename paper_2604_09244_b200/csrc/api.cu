@@ -24,6 +24,7 @@ struct mvla_ctx {
     float* l1_ws;                // [max_batch * max_vis]
     float* ahat_state;           // [n_prune_points][n_slots][max_vis]
     float* mhat_state;           // [n_prune_points][n_slots][4]
+    unsigned long long* acc64;   // [max_batch * max_vis] fixed-point score accumulators, zero between calls
     std::vector<int32_t> t_host; // [n_prune_points][n_slots] steps absorbed so far
     int* status_host;            // mapped pinned word written by kernels whose bounded wait gave up
     int* status_dev;
@@ -213,10 +214,13 @@ int32_t check_sticky(mvla_ctx* ctx)
     return (ctx->status_host && *reinterpret_cast<volatile int*>(ctx->status_host) != 0) ? MVLA_ERR_TIMEOUT : MVLA_OK;
 }
 
-// Salience of one chunk into ctx->part (+ L1 norms into `l1` when asked).
+// Salience of one chunk (+ L1 norms into `l1` when asked).  The per-head contributions land in
+// ctx->part, or, when `want_acc64` and the register-resident tensor-core kernel covers the shape, in the
+// fixed-point accumulators ctx->acc64 (*used_acc64 = true).
 int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, const void* k, int64_t rows,
-                           const void* hidden, float* l1, cudaStream_t st)
+                           const void* hidden, float* l1, bool want_acc64, bool* used_acc64, cudaStream_t st)
 {
+    if (used_acc64) *used_acc64 = false;
     const mvla_config& c = ctx->cfg;
     int max_tiles = 1, max_txt = 1;
     for (int b = 0; b < bd.n; ++b) {
@@ -233,14 +237,21 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
         r = tensor_map(ctx, 1, k, rows, kKeyTile, &tk);
         if (r != MVLA_OK) return r;
     }
-    cudaError_t e = launch_salience(bd, c.dtype, c.n_heads, c.head_dim, q, k, tq, tk, ctx->use_umma, tiles_per_cta,
-                                    cluster, npad, ctx->part, ctx->part_stride, ctx->status_dev, st);
-    if (e == cudaErrorInvalidConfiguration) return MVLA_ERR_UNSUPPORTED;
-    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    cudaError_t e;
     if (hidden && l1) {
         e = launch_l1norm(bd, c.dtype, c.d_model, hidden, l1, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
+    if (ctx->use_umma && fast_salience_supported(tiles_per_cta)) {
+        e = launch_salience_fast(bd, c.n_heads, c.head_dim, tq, tk, tiles_per_cta, cluster, npad, ctx->part,
+                                 ctx->part_stride, want_acc64 ? ctx->acc64 : nullptr, ctx->status_dev, st);
+        if (used_acc64) *used_acc64 = want_acc64;
+    } else {
+        e = launch_salience(bd, c.dtype, c.n_heads, c.head_dim, q, k, tq, tk, ctx->use_umma, tiles_per_cta,
+                            cluster, npad, ctx->part, ctx->part_stride, ctx->status_dev, st);
+    }
+    if (e == cudaErrorInvalidConfiguration) return MVLA_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
     return MVLA_OK;
 }
 
@@ -297,6 +308,7 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     ctx->use_umma = c.dtype == MVLA_DTYPE_BF16;
     if (c.salience_path == MVLA_SALIENCE_FMA) ctx->use_umma = false;
     ctx->part = ctx->attn_ws = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
+    ctx->acc64 = nullptr;
     ctx->status_host = ctx->status_dev = nullptr;
     ctx->last_cuda = cudaSuccess;
     ctx->tm_ptr[0] = ctx->tm_ptr[1] = nullptr;
@@ -317,6 +329,8 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     alloc(&ctx->l1_ws, vis_all);
     alloc(&ctx->ahat_state, n_state * ctx->max_vis);
     alloc(&ctx->mhat_state, n_state * 4);
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->acc64), vis_all * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(ctx->acc64, 0, vis_all * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&ctx->status_host), sizeof(int), cudaHostAllocMapped);
     if (e == cudaSuccess) {
         *ctx->status_host = 0;
@@ -348,6 +362,7 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     cudaFree(ctx->l1_ws);
     cudaFree(ctx->ahat_state);
     cudaFree(ctx->mhat_state);
+    cudaFree(ctx->acc64);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     delete ctx;
 }
@@ -370,7 +385,7 @@ int32_t mvla_salience(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, 
     const bool want_l1 = hidden && l1_out;
     for (int first = 0; first < batch; first += kMaxChunk) {
         const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
-        rc = run_salience_chunk(ctx, bd, q, k, rows, want_l1 ? hidden : nullptr, l1_out, st);
+        rc = run_salience_chunk(ctx, bd, q, k, rows, want_l1 ? hidden : nullptr, l1_out, false, nullptr, st);
         if (rc != MVLA_OK) return rc;
     }
     const cudaError_t e = launch_head_reduce(ctx->part, ctx->part_stride, ctx->cfg.n_heads, plan.total_vis, attn_out, st);
@@ -399,9 +414,15 @@ int32_t mvla_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvl
     for (int first = 0; first < batch; first += kMaxChunk) {
         const int n = std::min(kMaxChunk, batch - first);
         const BatchDesc bd = chunk_of(plan, first, n);
-        const cudaError_t e = launch_select(bd, gp, attn, nullptr, 0, ctx->cfg.n_heads, l1, ctx->ahat_state,
-                                            ctx->mhat_state, kept_idx, out_offsets, first, plan.total_out,
-                                            first + n == batch, budgets, nullptr, ahat_out, z_out, diag, st);
+        SelectIO io;
+        std::memset(&io, 0, sizeof io);
+        io.attn = attn; io.n_heads = ctx->cfg.n_heads; io.l1 = l1;
+        io.ahat_state = ctx->ahat_state; io.mhat_state = ctx->mhat_state;
+        io.kept_idx = kept_idx; io.out_offsets = out_offsets; io.budgets = budgets;
+        io.ahat_out = ahat_out; io.z_out = z_out; io.diag = diag;
+        io.chunk_first = first; io.total_out = plan.total_out; io.write_total = first + n == batch;
+        io.n_in_launch = n;
+        const cudaError_t e = launch_select(bd, gp, io, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
     commit_steps(ctx, prune_point, plan, samples);
@@ -476,12 +497,22 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     for (int first = 0; first < batch; first += kMaxChunk) {
         const int n = std::min(kMaxChunk, batch - first);
         const BatchDesc bd = chunk_of(plan, first, n);
-        rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, ctx->l1_ws, st);
+        bool used_acc64 = false;
+        rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, ctx->l1_ws, true,
+                                &used_acc64, st);
         if (rc != MVLA_OK) return rc;
-        cudaError_t e = launch_select(bd, gp, nullptr, ctx->part, ctx->part_stride, ctx->cfg.n_heads,
-                                      adaptive ? ctx->l1_ws : nullptr, ctx->ahat_state, ctx->mhat_state,
-                                      out->kept_idx, out->out_offsets, first, plan.total_out, first + n == batch,
-                                      out->budgets, out->attn, out->ahat, out->z, out->diag, st);
+        SelectIO io;
+        std::memset(&io, 0, sizeof io);
+        io.n_heads = ctx->cfg.n_heads;
+        if (used_acc64) io.acc64 = ctx->acc64;
+        else { io.part = ctx->part; io.part_stride = ctx->part_stride; }
+        io.l1 = adaptive ? ctx->l1_ws : nullptr;
+        io.ahat_state = ctx->ahat_state; io.mhat_state = ctx->mhat_state;
+        io.kept_idx = out->kept_idx; io.out_offsets = out->out_offsets; io.budgets = out->budgets;
+        io.attn_out = out->attn; io.ahat_out = out->ahat; io.z_out = out->z; io.diag = out->diag;
+        io.chunk_first = first; io.total_out = plan.total_out; io.write_total = first + n == batch;
+        io.n_in_launch = n;
+        cudaError_t e = launch_select(bd, gp, io, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
         const int32_t row0 = bd.s[0].out_off;
         const int32_t nrows = bd.s[n - 1].out_off + bd.s[n - 1].n_out - row0;

@@ -44,7 +44,41 @@ struct GateParams {
     int32_t has_l1;
 };
 
+// Scores arrive either as fp32 (`attn`), as per-head fp32 partials (`part`), or as 64-bit fixed-point
+// sums over heads (`acc64`, scale 2^60, exact and order independent; cleared after reading).
+struct SelectIO {
+    const float* attn;
+    const float* part;
+    int64_t part_stride;
+    int n_heads;
+    unsigned long long* acc64;
+    const float* l1;
+    float* ahat_state;
+    float* mhat_state;
+    int32_t* kept_idx;
+    int32_t* out_offsets;
+    int32_t* budgets;
+    float* attn_out;
+    float* ahat_out;
+    float* z_out;
+    mvla_diag* diag;
+    int32_t chunk_first;     // index of the launch's first sample in the whole batch
+    int32_t total_out;
+    int32_t write_total;     // this launch holds the batch's last sample
+    int32_t n_in_launch;
+};
+
 // ---- launchers (each enqueues on `stream` and returns the launch status) ----
+
+// bf16 tensor-core salience with logits held in registers (one or two key tiles per CTA).  With
+// `acc64` the per-head contributions are added into 64-bit fixed-point accumulators (scale 2^60, one
+// per visual token, zero on entry); without it they go to part[h][vis] as in launch_salience.
+bool fast_salience_supported(int tiles_per_cta);
+cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int head_dim, const CUtensorMap* tmap_q,
+                                 const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
+                                 float* part, int64_t part_stride, unsigned long long* acc64, int* status,
+                                 cudaStream_t stream);
+
 
 // Salience: per-head partial scores part[h][vis] (already scaled by 1/(H n_t)).
 // `use_umma`: tensor-core path (bf16 only).  tmaps: device-usable tensor maps (passed by value).
@@ -62,14 +96,8 @@ cudaError_t launch_head_reduce(const float* part, int64_t part_stride, int n_hea
 cudaError_t launch_l1norm(const BatchDesc& bd, int dtype, int d_model, const void* hidden,
                           float* l1, cudaStream_t stream);
 
-// Carry-over + budget + top-k + emission; one CTA per sample.
-// Scores come either from `attn` (part == nullptr) or from per-head partials.
-cudaError_t launch_select(const BatchDesc& bd, const GateParams& gp, const float* attn,
-                          const float* part, int64_t part_stride, int n_heads, const float* l1,
-                          float* ahat_state, float* mhat_state, int32_t* kept_idx,
-                          int32_t* out_offsets, int chunk_first, int32_t total_out, int write_total,
-                          int32_t* budgets, float* attn_out, float* ahat_out, float* z_out,
-                          mvla_diag* diag, cudaStream_t stream);
+// Carry-over + budget + top-k + emission; one CTA per sample (io.n_in_launch = bd.n).
+cudaError_t launch_select(const BatchDesc& bd, const GateParams& gp, const SelectIO& io, cudaStream_t stream);
 
 // Row gather of up to three tensors.
 struct CompactJob {

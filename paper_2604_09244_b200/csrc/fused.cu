@@ -1,0 +1,321 @@
+// Fast salience kernel for bf16 (Sec. 3.2.1 of the paper).
+//
+// Same decomposition as the generic salience kernel (one cluster per (sample, head), one CTA per one or
+// two tiles of 128 keys; TMA -> shared memory -> tcgen05.mma -> tensor memory), but built as one short
+// dependency chain, because at ~40 KB of input per CTA the kernel is latency bound:
+//   * the loads are issued before anything else; tensor-memory allocation overlaps with them;
+//   * each thread reads ALL its logits from tensor memory once (one wide tcgen05.ld) and keeps them in
+//     registers through max -> exp2 -> sum -> weighted sum;
+//   * the per-query (max, sum) pairs travel between the CTAs of a cluster as plain remote shared-memory
+//     stores, spread over all threads, followed by ONE remote mbarrier arrive per peer (release /
+//     acquire at cluster scope): no cluster-wide hardware barrier and no chain of fences on the
+//     critical path;
+//   * per-head contributions are added into one 64-bit fixed-point accumulator per token (scale 2^60):
+//     integer adds commute, so the sum over heads is exact and independent of scheduling.
+#include "common.cuh"
+#include "device_utils.cuh"
+#include "select_impl.cuh"
+#include "tmem_ld.cuh"
+
+#include <algorithm>
+#include <cstring>
+
+namespace mvla {
+namespace {
+
+constexpr int kFastThreads = 128;
+
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void st_peer_f32x2(uint32_t local_addr, uint32_t rank, float2 v)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(remote), "f"(v.x), "f"(v.y) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_peer_release(uint32_t local_bar, uint32_t rank)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_bar), "r"(rank));
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+// Bounded wait with acquire at cluster scope (the arrivals come from other CTAs).
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    const uint64_t t0 = global_ns();
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((it & 63u) == 63u && global_ns() - t0 > 1000000000ull) break;
+    }
+    return false;
+}
+
+// grid = (cluster size, n_heads, samples), cluster = (cluster size, 1, 1), 128 threads.
+// TCOL: tensor-memory columns per tile (>= padded query count); NTILE: key tiles per CTA.
+template <int TCOL, int NTILE>
+__global__ void __launch_bounds__(kFastThreads, 1)
+salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
+                     const __grid_constant__ CUtensorMap tmap_k, int n_heads, int head_dim, int npad,
+                     float* __restrict__ part, int64_t part_stride, unsigned long long* __restrict__ acc64,
+                     int* status)
+{
+    constexpr int CC = TCOL * NTILE;
+    extern __shared__ uint8_t dyn_smem_raw[];
+    uint8_t* dyn_smem = dyn_smem_raw + ((1024u - (smem_u32(dyn_smem_raw) & 1023u)) & 1023u);   // swizzle atoms are 1 KB
+    __shared__ float s_m[kMaxText];                       // local max per query (log2 domain), -inf replaced by 0
+    __shared__ float s_w[kMaxText];                       // final weight per query
+    __shared__ float2 s_peer[kMaxCluster][kMaxText];      // (raw local max, local sum) of every CTA of the cluster
+    __shared__ float2 s_loc[kMaxText];                    // this CTA's pairs, staged for the push
+    __shared__ float s_wred[4][kMaxText];
+    __shared__ __align__(8) uint64_t s_bar[3];
+    __shared__ uint32_t s_tmem;
+
+    const SampleDev& s = bd.s[blockIdx.z];
+    const int h = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t crank = cluster_ctarank();
+    const uint32_t csize = gridDim.x;
+    const int d = head_dim;
+    const int khalves = d / 64;                           // 64 bf16 = one 128-byte swizzle row
+    const float cscale = 1.4426950408889634f * rsqrtf(static_cast<float>(d));   // log2 domain
+    const int tt0 = static_cast<int>(crank) * NTILE;
+    uint8_t* Ks = dyn_smem;                               // [tile][khalf][128 rows x 128 B]
+    uint8_t* Qs = dyn_smem + static_cast<size_t>(NTILE) * khalves * 16384;   // [khalf][npad rows x 128 B]
+    const uint32_t bar_full = smem_u32(&s_bar[0]), bar_mma = smem_u32(&s_bar[1]), bar_x = smem_u32(&s_bar[2]);
+
+    int valid[NTILE], vis0[NTILE];
+    bool any_live = false;
+#pragma unroll
+    for (int t = 0; t < NTILE; ++t) {
+        const TileInfo ti = tile_info(s, tt0 + t);
+        valid[t] = ti.valid;
+        vis0[t] = ti.vis0;
+        any_live |= ti.valid > 0;
+    }
+
+    if (tid == 0) {                           // the loads go out first; everything else overlaps with them
+        prefetch_tensormap(&tmap_q);
+        prefetch_tensormap(&tmap_k);
+        mbar_init(bar_full, 1);
+        mbar_init(bar_mma, 1);
+        mbar_init(bar_x, csize);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        int live = 0;
+#pragma unroll
+        for (int t = 0; t < NTILE; ++t) live += valid[t] > 0;
+        mbar_expect_tx(bar_full, static_cast<uint32_t>(khalves) * (npad * 128 + live * 16384));
+        for (int kh = 0; kh < khalves; ++kh)
+            for (int c = 0; c < npad / 16; ++c)
+                tma_load_3d(smem_u32(Qs + kh * npad * 128 + c * 2048), &tmap_q, kh * 64, h,
+                            s.seq_off + s.off_txt + c * 16, bar_full);
+#pragma unroll
+        for (int t = 0; t < NTILE; ++t) {
+            if (valid[t] <= 0) continue;
+            const int row0 = tile_info(s, tt0 + t).row0;
+            for (int kh = 0; kh < khalves; ++kh)
+                tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * 64, h, row0, bar_full);
+        }
+    }
+    if (tid < kMaxText) s_w[tid] = 0.f;
+    __syncwarp();
+    cluster_arrive_release();                 // publishes this CTA's barriers; matched by the wait before the first remote store
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < static_cast<uint32_t>(CC)) tmem_cols <<= 1;
+    if (warp == 1) tmem_alloc(smem_u32(&s_tmem), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem;
+
+    if (tid == 0) {
+        bool got = mbar_wait(bar_full, 0);
+        if (!got) {                           // report, then give the copies one more bounded chance to land
+            *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
+            got = mbar_wait(bar_full, 0);
+        }
+        if (got) {
+            tc_fence_after();
+            const uint32_t idesc = idesc_bf16_m128(npad);
+#pragma unroll
+            for (int t = 0; t < NTILE; ++t) {
+                if (valid[t] <= 0) continue;
+                for (int kb = 0; kb < d / 16; ++kb) {
+                    const int kh = kb >> 2, kin = kb & 3;          // 4 K-steps of 16 inside a 64-wide half
+                    const uint64_t a = smem_desc_sw128(smem_u32(Ks + (t * khalves + kh) * 16384) + kin * 32);
+                    const uint64_t b = smem_desc_sw128(smem_u32(Qs + kh * npad * 128) + kin * 32);
+                    umma_bf16(tmem_base + t * TCOL, a, b, idesc, kb > 0 ? 1u : 0u);
+                }
+            }
+        }
+        umma_commit(bar_mma);                 // arrives once every MMA issued above has finished
+    }
+    __syncwarp();
+    bool ok = mbar_wait(bar_mma, 0);
+    if (!ok) *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
+    ok = __syncthreads_and(ok) != 0;          // block-uniform from here on (aligned instructions follow)
+    tc_fence_after();
+
+    // ---- all logits of this thread's key(s) into registers, scaled to the log2 domain, masked
+    float L[CC];
+    if (any_live && ok) {
+        tmem_ld_cols<CC>(tmem_base + (static_cast<uint32_t>(warp * 32) << 16), L);
+    } else {
+#pragma unroll
+        for (int i = 0; i < CC; ++i) L[i] = 0.f;
+    }
+#pragma unroll
+    for (int t = 0; t < NTILE; ++t) {
+        const bool live = ok && tid < valid[t];
+#pragma unroll
+        for (int i = 0; i < TCOL; ++i) L[t * TCOL + i] = (live && i < npad) ? L[t * TCOL + i] * cscale : -CUDART_INF_F;
+    }
+
+    // ---- local maximum per query
+#pragma unroll
+    for (int qc = 0; qc < TCOL / 16; ++qc) {
+        if (qc * 16 >= npad) break;
+        float m[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            m[i] = L[qc * 16 + i];
+#pragma unroll
+            for (int t = 1; t < NTILE; ++t) m[i] = fmaxf(m[i], L[t * TCOL + qc * 16 + i]);
+        }
+        const float red = warp_reduce16<true>(m, lane);
+        if ((lane & 1) == 0) s_wred[warp][qc * 16 + col16(lane)] = red;
+    }
+    __syncthreads();
+    float m_raw = -CUDART_INF_F;
+    if (tid < npad) {
+        m_raw = fmaxf(fmaxf(s_wred[0][tid], s_wred[1][tid]), fmaxf(s_wred[2][tid], s_wred[3][tid]));
+        s_m[tid] = (m_raw == -CUDART_INF_F) ? 0.f : m_raw;
+    }
+    __syncthreads();
+
+    // ---- exponentials (kept in registers) and the local denominator per query
+#pragma unroll
+    for (int qc = 0; qc < TCOL / 16; ++qc) {
+        if (qc * 16 >= npad) break;
+        float sum[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float mm = s_m[qc * 16 + i];
+            sum[i] = 0.f;
+#pragma unroll
+            for (int t = 0; t < NTILE; ++t) {
+                const float e = ex2_approx(L[t * TCOL + qc * 16 + i] - mm);
+                L[t * TCOL + qc * 16 + i] = e;
+                sum[i] += e;
+            }
+        }
+        const float red = warp_reduce16<false>(sum, lane);
+        if ((lane & 1) == 0) s_wred[warp][qc * 16 + col16(lane)] = red;
+    }
+    __syncthreads();
+
+    // ---- exchange (max, sum) with the other key tiles of this (sample, head)
+    if (tid < npad)
+        s_loc[tid] = make_float2(m_raw, (s_wred[0][tid] + s_wred[1][tid]) + (s_wred[2][tid] + s_wred[3][tid]));
+    __syncthreads();
+    cluster_wait_acquire();                   // every peer is running and has initialised its barriers
+    for (int p = tid; p < npad * static_cast<int>(csize); p += kFastThreads) {
+        const int i = p % npad;
+        const uint32_t r = static_cast<uint32_t>(p / npad);
+        st_peer_f32x2(smem_u32(&s_peer[crank][i]), r, s_loc[i]);
+    }
+    __syncthreads();                          // all of this CTA's stores are ordered before the arrives below
+    if (tid < static_cast<int>(csize)) mbar_arrive_peer_release(bar_x, static_cast<uint32_t>(tid));
+    __syncwarp();
+    bool okx = mbar_wait_cluster(bar_x, 0);
+    if (!okx) *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
+    if (tid < npad) {
+        float gmax = -CUDART_INF_F;
+        for (uint32_t r = 0; r < csize; ++r) gmax = fmaxf(gmax, s_peer[r][tid].x);
+        float z = 0.f;
+        for (uint32_t r = 0; r < csize; ++r) {
+            const float2 pr = s_peer[r][tid];
+            if (pr.x > -CUDART_INF_F) z += pr.y * ex2_approx(pr.x - gmax);
+        }
+        const float inv_hn = 1.f / (static_cast<float>(n_heads) * static_cast<float>(s.n_txt));
+        s_w[tid] = (tid < s.n_txt && z > 0.f && okx) ? ex2_approx(s_m[tid] - gmax) / z * inv_hn : 0.f;
+    }
+    __syncthreads();
+
+    // ---- per key: sum over queries of the normalised probabilities (this head's contribution)
+#pragma unroll
+    for (int t = 0; t < NTILE; ++t) {
+        if (valid[t] <= 0) continue;
+        float acc = 0.f;
+#pragma unroll
+        for (int qc = 0; qc < TCOL / 16; ++qc) {
+            if (qc * 16 >= npad) break;       // columns past the padded query count were never exponentiated
+#pragma unroll
+            for (int i = 0; i < 16; ++i)      // s_w is 0 past the text queries
+                acc = fmaf(L[t * TCOL + qc * 16 + i], s_w[qc * 16 + i], acc);
+        }
+        if (tid < valid[t]) {
+            if (acc64)
+                atomicAdd(acc64 + s.vis_off + vis0[t] + tid, __float2ull_rn(acc * kFixScale));
+            else
+                part[static_cast<int64_t>(h) * part_stride + s.vis_off + vis0[t] + tid] = acc;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);    // the warp that allocated
+}
+
+template <int TCOL, int NTILE>
+cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int head_dim, const CUtensorMap* tq,
+                          const CUtensorMap* tk, int cluster, int npad, float* part, int64_t part_stride,
+                          unsigned long long* acc64, int* status, cudaStream_t stream)
+{
+    const size_t smem = 1024 + static_cast<size_t>(head_dim / 64) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
+    auto kern = salience_fast_kernel<TCOL, NTILE>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cluster, n_heads, bd.n);
+    cfg.blockDim = dim3(kFastThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, head_dim, npad, part, part_stride, acc64, status);
+}
+
+}  // namespace
+
+bool fast_salience_supported(int tiles_per_cta) { return tiles_per_cta >= 1 && tiles_per_cta <= 2; }
+
+cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int head_dim, const CUtensorMap* tmap_q,
+                                 const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
+                                 float* part, int64_t part_stride, unsigned long long* acc64, int* status,
+                                 cudaStream_t stream)
+{
+    const int tcol = npad <= 16 ? 16 : (npad <= 32 ? 32 : 64);
+#define MVLA_FAST(TC, NTL)                                                                                      \
+    if (tcol == TC && tiles_per_cta == NTL)                                                                     \
+        return launch_fast_t<TC, NTL>(bd, n_heads, head_dim, tmap_q, tmap_k, cluster, npad, part, part_stride, \
+                                      acc64, status, stream);
+    MVLA_FAST(16, 1) MVLA_FAST(32, 1) MVLA_FAST(64, 1) MVLA_FAST(16, 2) MVLA_FAST(32, 2) MVLA_FAST(64, 2)
+#undef MVLA_FAST
+    return cudaErrorInvalidConfiguration;
+}
+
+}  // namespace mvla

@@ -9,181 +9,12 @@
 // head's contribution  sum_i softmax(l[h,i,:])_j / (H n_t)  to part[h][j].  Heads are summed
 // later in a fixed order so that the result does not depend on scheduling.
 #include "common.cuh"
+#include "device_utils.cuh"
 
 #include <math_constants.h>
 
 namespace mvla {
 namespace {
-
-// ------------------------------------------------------------------ small PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p)
-{
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ uint32_t cluster_ctarank()
-{
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\t"
-                 "barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ float ld_peer_f32(uint32_t local_addr, uint32_t rank)
-{
-    uint32_t remote;
-    float v;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
-    return v;
-}
-__device__ __forceinline__ uint64_t global_ns()
-{
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Bounded wait: gives up after about one second and reports false.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
-{
-    const uint64_t t0 = global_ns();
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        uint32_t ok;
-        asm volatile("{\n\t.reg .pred p;\n\t"
-                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                     "selp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        if (ok) return true;
-        if (global_ns() - t0 > 1000000000ull) break;
-    }
-    return false;
-}
-// One box of a 3-D tiled tensor map -> this CTA's shared memory; completion counted on `bar`.
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
-                                            uint32_t bar)
-{
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
-                 " [%0], [%1, {%3, %4, %5}], [%2];"
-                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
-{
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
-{
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; issued by one thread.
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate)
-{
-    asm volatile("{\n\t.reg .pred p;\n\t"
-                 "setp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// 16 consecutive fp32 columns of this thread's tensor-memory lane.
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
-{
-    uint32_t r[16];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32"
-                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-                 : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-// Shared-memory matrix descriptor: K-major tile, 128-byte rows, 128-byte swizzle, groups of 8 rows
-// 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
-{
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);          // start address
-    d |= static_cast<uint64_t>(1) << 16;                         // leading byte offset (unused here)
-    d |= static_cast<uint64_t>(1024 >> 4) << 32;                 // stride byte offset
-    d |= static_cast<uint64_t>(1) << 46;                         // descriptor version
-    d |= static_cast<uint64_t>(2) << 61;                         // 128-byte swizzle
-    return d;
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t idesc_bf16_m128(int n)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | ((128u >> 4) << 24);
-}
-
-// Reduce 16 per-thread values across the 32 lanes of a warp in 16 shuffles.  On return lane L
-// holds the result of column col16(L); lanes L and L^1 hold the same column.
-template <bool IS_MAX>
-__device__ __forceinline__ float warp_reduce16(float (&v)[16], int lane)
-{
-#pragma unroll
-    for (int w = 8; w >= 1; w >>= 1) {
-        const int off = w * 2;
-        const bool up = (lane & off) != 0;
-#pragma unroll
-        for (int i = 0; i < w; ++i) {
-            const float send = up ? v[i] : v[i + w];
-            const float keep = up ? v[i + w] : v[i];
-            const float got = __shfl_xor_sync(0xffffffffu, send, off);
-            v[i] = IS_MAX ? fmaxf(keep, got) : keep + got;
-        }
-    }
-    const float got = __shfl_xor_sync(0xffffffffu, v[0], 1);
-    return IS_MAX ? fmaxf(v[0], got) : v[0] + got;
-}
-__device__ __forceinline__ int col16(int lane)
-{
-    return ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
-}
-
-struct TileInfo {
-    int valid;   // keys of this tile that exist (0: tile past the end)
-    int row0;    // first row in the packed tensors
-    int vis0;    // visual index of the first key
-};
-__device__ __forceinline__ TileInfo tile_info(const SampleDev& s, int tt)
-{
-    const int t2 = (s.n_2d + kKeyTile - 1) / kKeyTile;
-    const int t3 = (s.n_3d + kKeyTile - 1) / kKeyTile;
-    TileInfo ti{0, 0, 0};
-    if (tt < t2) {
-        const int st = tt * kKeyTile;
-        ti.valid = min(kKeyTile, s.n_2d - st);
-        ti.row0 = s.seq_off + s.off_2d + st;
-        ti.vis0 = st;
-    } else if (tt < t2 + t3) {
-        const int st = (tt - t2) * kKeyTile;
-        ti.valid = min(kKeyTile, s.n_3d - st);
-        ti.row0 = s.seq_off + s.off_3d + st;
-        ti.vis0 = s.n_2d + st;
-    }
-    return ti;
-}
-
-__device__ __forceinline__ float to_f32(float x) { return x; }
-__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
 
 constexpr int kThreads = 128;
 
@@ -201,11 +32,12 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
     uint8_t* dyn_smem = dyn_smem_raw + ((1024u - (smem_u32(dyn_smem_raw) & 1023u)) & 1023u);   // swizzle atoms are 1 KB
     __shared__ float s_m[kMaxText];          // local max per query (log2 domain), -inf replaced by 0
     __shared__ float s_w[kMaxText];          // final weight per query
-    __shared__ float s_stat[2][kMaxText];    // what peers read: raw local max, local sum
+    __shared__ float s_peer[kMaxCluster][2][kMaxText];   // (raw local max, local sum) pushed here by every CTA of the cluster
     __shared__ float s_wred[4][kMaxText];
     __shared__ __align__(8) uint64_t s_bar[2];
     __shared__ uint32_t s_tmem;
 
+    cluster_arrive_relaxed();                 // matched by the wait before the first remote store
     const SampleDev& s = bd.s[blockIdx.z];
     const int h = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -229,21 +61,12 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
         const uint32_t bar_full = smem_u32(&s_bar[0]), bar_mma = smem_u32(&s_bar[1]);
         tmem_cols = 32;
         while (tmem_cols < static_cast<uint32_t>(tiles_per_cta * tcol)) tmem_cols <<= 1;
-        if (tid == 0) {
+        if (tid == 0) {                       // the loads go out first; everything else overlaps with them
+            prefetch_tensormap(&tmap_q);
+            prefetch_tensormap(&tmap_k);
             mbar_init(bar_full, 1);
             mbar_init(bar_mma, 1);
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        }
-        if (warp == 0) {
-            __syncwarp();
-            tmem_alloc(smem_u32(&s_tmem), tmem_cols);
-        }
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-        tmem_base = s_tmem;
-
-        if (tid == 0) {
             int live = 0;
             for (int t = 0; t < tiles_per_cta; ++t) live += tile_info(s, tt0 + t).valid > 0;
             const uint32_t bytes = static_cast<uint32_t>(khalves) * (npad * 128 + live * 16384);
@@ -258,6 +81,14 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
                 for (int kh = 0; kh < khalves; ++kh)
                     tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * 64, h, ti.row0, bar_full);
             }
+        }
+        if (warp == 1) tmem_alloc(smem_u32(&s_tmem), tmem_cols);
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        tmem_base = s_tmem;
+
+        if (tid == 0) {
             bool got = mbar_wait(bar_full, 0);
             if (!got) {                       // report, then give the copies one more bounded chance to land
                 *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
@@ -362,10 +193,10 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
         if ((lane & 1) == 0) s_wred[warp][cb + col16(lane)] = red;
     }
     __syncthreads();
+    float m_raw = -CUDART_INF_F;
     if (tid < npad) {
-        const float m = fmaxf(fmaxf(s_wred[0][tid], s_wred[1][tid]), fmaxf(s_wred[2][tid], s_wred[3][tid]));
-        s_stat[0][tid] = m;
-        s_m[tid] = (m == -CUDART_INF_F) ? 0.f : m;
+        m_raw = fmaxf(fmaxf(s_wred[0][tid], s_wred[1][tid]), fmaxf(s_wred[2][tid], s_wred[3][tid]));
+        s_m[tid] = (m_raw == -CUDART_INF_F) ? 0.f : m_raw;
     }
     __syncthreads();
 
@@ -386,19 +217,27 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
         if ((lane & 1) == 0) s_wred[warp][cb + col16(lane)] = red;
     }
     __syncthreads();
-    if (tid < npad) s_stat[1][tid] = (s_wred[0][tid] + s_wred[1][tid]) + (s_wred[2][tid] + s_wred[3][tid]);
-    __syncthreads();
-
-    // ---- exchange (max, sum) with the other key tiles of this (sample, head)
-    cluster_sync_all();
+    // ---- exchange (max, sum) with the other key tiles of this (sample, head): every CTA pushes its
+    //      pair into every CTA's s_peer slot, then one release/acquire cluster barrier publishes them.
+    cluster_wait_acquire();                   // pairs with the arrive at kernel entry: all peers are running
     if (tid < npad) {
-        const uint32_t a_m = smem_u32(&s_stat[0][tid]), a_s = smem_u32(&s_stat[1][tid]);
+        const float ssum = (s_wred[0][tid] + s_wred[1][tid]) + (s_wred[2][tid] + s_wred[3][tid]);
+        const uint32_t a_m = smem_u32(&s_peer[crank][0][tid]), a_s = smem_u32(&s_peer[crank][1][tid]);
+        for (uint32_t r = 0; r < csize; ++r) {
+            st_peer_f32(a_m, r, m_raw);
+            st_peer_f32(a_s, r, ssum);
+        }
+    }
+    __syncwarp();
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    if (tid < npad) {
         float gmax = -CUDART_INF_F;
-        for (uint32_t r = 0; r < csize; ++r) gmax = fmaxf(gmax, ld_peer_f32(a_m, r));
+        for (uint32_t r = 0; r < csize; ++r) gmax = fmaxf(gmax, s_peer[r][0][tid]);
         float z = 0.f;
         for (uint32_t r = 0; r < csize; ++r) {
-            const float mr = ld_peer_f32(a_m, r);
-            if (mr > -CUDART_INF_F) z += ld_peer_f32(a_s, r) * exp2f(mr - gmax);
+            const float mr = s_peer[r][0][tid];
+            if (mr > -CUDART_INF_F) z += s_peer[r][1][tid] * exp2f(mr - gmax);
         }
         const float inv_hn = 1.f / (static_cast<float>(n_heads) * static_cast<float>(s.n_txt));
         s_w[tid] = (tid < s.n_txt && z > 0.f) ? exp2f(s_m[tid] - gmax) / z * inv_hn : 0.f;
@@ -425,13 +264,11 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
             part[static_cast<int64_t>(h) * part_stride + s.vis_off + ti.vis0 + tid] = acc;
     }
 
-    // peers may still be reading this CTA's statistics
-    __syncthreads();
-    cluster_sync_all();
+    // nothing touches a peer's shared memory after the barrier above, so CTAs may exit independently
     if constexpr (UMMA) {
         tc_fence_before();
         __syncthreads();
-        if (warp == 0) tmem_dealloc(tmem_base, tmem_cols);
+        if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);    // the warp that allocated
     }
 }
 
