@@ -68,6 +68,16 @@ struct SelectIO {
     int32_t n_in_launch;
 };
 
+// Launch attribute that lets a kernel begin before its stream predecessor has drained (the kernel
+// itself waits with griddepcontrol.wait before it touches anything the predecessor wrote).
+inline cudaLaunchAttribute pdl_attribute()
+{
+    cudaLaunchAttribute a = {};
+    a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    a.val.programmaticStreamSerializationAllowed = 1;
+    return a;
+}
+
 // ---- launchers (each enqueues on `stream` and returns the launch status) ----
 
 // bf16 tensor-core salience with logits held in registers (one or two key tiles per CTA).  With

@@ -38,6 +38,7 @@ compact_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ Com
                int32_t chunk_rows, int32_t chunk_row0, const int32_t* __restrict__ out_offsets,
                int32_t chunk_first, int32_t batch_total)
 {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = threadIdx.x & 31;
     const int64_t unit = static_cast<int64_t>(blockIdx.x) * kWarpsPerBlock + (threadIdx.x >> 5);
     const int per_row = a.seg_begin[3];
@@ -46,6 +47,7 @@ compact_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ Com
     const int u = static_cast<int>(unit - static_cast<int64_t>(r) * per_row);
     const int orow = chunk_row0 + r;
 
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // kept_idx comes from the kernel before this one
     // which sample owns output row `orow` (samples are few: linear scan)
     int b = 0;
     if (out_offsets) {            // offsets known only on the device: scan the whole batch
@@ -99,9 +101,15 @@ cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int
     if (total == 0 || chunk_rows <= 0) return cudaSuccess;
     const int64_t units = static_cast<int64_t>(chunk_rows) * total;
     const int64_t blocks = (units + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    compact_kernel<<<static_cast<unsigned>(blocks), kWarpsPerBlock * 32, 0, stream>>>(
-        bd, a, kept_idx, chunk_rows, chunk_row0, out_offsets, chunk_first, batch_total);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+    cfg.blockDim = dim3(kWarpsPerBlock * 32);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1] = {pdl_attribute()};
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, compact_kernel, bd, a, kept_idx, chunk_rows, chunk_row0, out_offsets, chunk_first,
+                              batch_total);
 }
 
 }  // namespace mvla

@@ -6,10 +6,9 @@
 //   * the loads are issued before anything else; tensor-memory allocation overlaps with them;
 //   * each thread reads ALL its logits from tensor memory once (one wide tcgen05.ld) and keeps them in
 //     registers through max -> exp2 -> sum -> weighted sum;
-//   * the per-query (max, sum) pairs travel between the CTAs of a cluster as plain remote shared-memory
-//     stores, spread over all threads, followed by ONE remote mbarrier arrive per peer (release /
-//     acquire at cluster scope): no cluster-wide hardware barrier and no chain of fences on the
-//     critical path;
+//   * the per-query (max, sum) pairs travel between the CTAs of a cluster as asynchronous remote
+//     shared-memory stores that credit the receiver's mbarrier when they land (st.async with
+//     complete_tx): one one-way trip, no cluster-wide hardware barrier and no fence on the critical path;
 //   * per-head contributions are added into one 64-bit fixed-point accumulator per token (scale 2^60):
 //     integer adds commute, so the sum over heads is exact and independent of scheduling.
 #include "common.cuh"
@@ -31,17 +30,16 @@ __device__ __forceinline__ float ex2_approx(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void st_peer_f32x2(uint32_t local_addr, uint32_t rank, float2 v)
+// Asynchronous 8-byte store into the shared memory of CTA `rank` (same offset as `local_addr`); on
+// landing it credits 8 bytes to that CTA's mbarrier at the offset of `local_bar`: the data and its
+// "ready" signal travel together, one way.
+__device__ __forceinline__ void st_async_peer_f32x2(uint32_t local_addr, uint32_t local_bar, uint32_t rank, float2 v)
 {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(remote), "f"(v.x), "f"(v.y) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_peer_release(uint32_t local_bar, uint32_t rank)
-{
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_bar), "r"(rank));
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+    uint32_t raddr, rbar;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(local_addr), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(local_bar), "r"(rank));
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
+                 ::"r"(raddr), "f"(v.x), "f"(v.y), "r"(rbar) : "memory");
 }
 // Bounded wait with acquire at cluster scope (the arrivals come from other CTAs).
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
@@ -102,13 +100,16 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         any_live |= ti.valid > 0;
     }
 
+    pdl_trigger();
     if (tid == 0) {                           // the loads go out first; everything else overlaps with them
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);
         mbar_init(bar_full, 1);
         mbar_init(bar_mma, 1);
-        mbar_init(bar_x, csize);
+        mbar_init(bar_x, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(bar_x, csize * static_cast<uint32_t>(npad) * 8u);     // every CTA of the cluster sends npad pairs
+        pdl_wait();                           // inputs may come from the kernel before this one
         int live = 0;
 #pragma unroll
         for (int t = 0; t < NTILE; ++t) live += valid[t] > 0;
@@ -230,10 +231,8 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     for (int p = tid; p < npad * static_cast<int>(csize); p += kFastThreads) {
         const int i = p % npad;
         const uint32_t r = static_cast<uint32_t>(p / npad);
-        st_peer_f32x2(smem_u32(&s_peer[crank][i]), r, s_loc[i]);
+        st_async_peer_f32x2(smem_u32(&s_peer[crank][i]), bar_x, r, s_loc[i]);
     }
-    __syncthreads();                          // all of this CTA's stores are ordered before the arrives below
-    if (tid < static_cast<int>(csize)) mbar_arrive_peer_release(bar_x, static_cast<uint32_t>(tid));
     __syncwarp();
     bool okx = mbar_wait_cluster(bar_x, 0);
     if (!okx) *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
@@ -251,6 +250,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     __syncthreads();
 
     // ---- per key: sum over queries of the normalised probabilities (this head's contribution)
+    pdl_wait();                               // the accumulators are read and cleared by the previous step's select
 #pragma unroll
     for (int t = 0; t < NTILE; ++t) {
         if (valid[t] <= 0) continue;
@@ -289,13 +289,14 @@ cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int head_dim, const 
     cfg.blockDim = dim3(kFastThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = cluster;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1] = pdl_attribute();
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, head_dim, npad, part, part_stride, acc64, status);
 }
 

@@ -18,8 +18,14 @@ select_kernel(const __grid_constant__ BatchDesc bd, const GateParams gp, const S
 
 cudaError_t launch_select(const BatchDesc& bd, const GateParams& gp, const SelectIO& io, cudaStream_t stream)
 {
-    select_kernel<<<bd.n, kSelThreads, 0, stream>>>(bd, gp, io);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(bd.n);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1] = {pdl_attribute()};
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, select_kernel, bd, gp, io);
 }
 
 }  // namespace mvla

@@ -34,6 +34,8 @@ struct SelectSmem {
     int krem[2];
     int k[2];
     int alltie[2];                // every element equal to the threshold key is kept: no tie ranking needed
+    int done[2];                  // the threshold is settled before all 32 bits were examined
+    uint32_t cmask[2];            // key bits that the threshold comparison looks at
 };
 
 // fp32 -> uint32 whose unsigned order is the float order; NaN sorts below everything.
@@ -118,6 +120,12 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
     const int b_glob = io.chunk_first + b_local;
     const bool carry = s.c_prev != 0.f;
 
+    // prologue that needs nothing from the previous kernel
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    for (int i = tid; i < 4 * 2 * 256; i += NT) (&sm.hist[0][0][0])[i] = 0;
+    if (tid < 2) { sm.prefix[tid] = 0u; sm.alltie[tid] = 1; sm.done[tid] = 0; sm.cmask[tid] = 0xFFFFFFFFu; }
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // scores come from the kernel before this one
+
     // ---- 1. all loads first
     float a[EPT], prev[EPT], nrm[EPT];
     unsigned long long fx[EPT];
@@ -132,8 +140,6 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
             if (gp.has_l1) nrm[e] = io.l1[s.vis_off + j];
         }
     }
-    for (int i = tid; i < 4 * 2 * 256; i += NT) (&sm.hist[0][0][0])[i] = 0;
-    if (tid < 2) { sm.prefix[tid] = 0u; sm.alltie[tid] = 1; }
     if (io.part && !io.acc64) {                            // per-head fp32 partials, summed in head order
 #pragma unroll
         for (int e = 0; e < EPT; ++e) {
@@ -184,7 +190,7 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
     }
 
     // One radix histogram pass over the keys that still match the prefix found so far.
-    auto histogram = [&](int pass, int shift, uint32_t p0, uint32_t p1) {
+    auto histogram = [&](int pass, int shift, uint32_t p0, uint32_t p1, bool skip0, bool skip1) {
         const uint32_t himask = shift == 24 ? 0u : (0xFFFFFFFFu << (shift + 8));
         int* hist = &sm.hist[pass][0][0];
 #pragma unroll
@@ -194,7 +200,8 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
             int bin = -1;                                  // -1: not a candidate (any more)
             if (j < nv) {
                 const int m = j >= n2;
-                if (((key[e] ^ (m ? p1 : p0)) & himask) == 0u) bin = (m << 8) | static_cast<int>((key[e] >> shift) & 255u);
+                if (!(m ? skip1 : skip0) && ((key[e] ^ (m ? p1 : p0)) & himask) == 0u)
+                    bin = (m << 8) | static_cast<int>((key[e] >> shift) & 255u);
             }
             // keys share their leading bytes most of the time: one atomic per warp instead of 32
             int same;
@@ -206,17 +213,17 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
             }
         }
     };
-    histogram(0, 24, 0u, 0u);                 // needs no budget yet: overlaps with the gate arithmetic
+    histogram(0, 24, 0u, 0u, false, false);   // needs no budget yet: overlaps with the gate arithmetic
 
-    // ---- 2. indicators, gates, budget (one thread; a few dozen flops)
-    if (tid == 0) {
+    // ---- 2. indicators, gates, budget (one thread of the last warp, which rarely owns elements; a few dozen flops)
+    if (tid == NT - 32) {
         float x[4];
-        x[3] = t1 / (t0 + t1);                                    // attention share of 3D (Eq. P2D / P3D)
+        x[3] = __fdividef(t1, t0 + t1);                                   // attention share of 3D (Eq. P2D / P3D)
         x[2] = 1.f - x[3];
         if (gp.has_l1) {                                          // feature-norm share (Eq. 3-1), mean norms
-            const float m2 = n2 > 0 ? t2 / static_cast<float>(n2) : 0.f;
-            const float m3 = n3 > 0 ? t3 / static_cast<float>(n3) : 0.f;
-            x[1] = m3 / (m2 + m3);
+            const float m2 = n2 > 0 ? __fdividef(t2, static_cast<float>(n2)) : 0.f;
+            const float m3 = n3 > 0 ? __fdividef(t3, static_cast<float>(n3)) : 0.f;
+            x[1] = __fdividef(m3, m2 + m3);
             x[0] = 1.f - x[1];
         } else {
             x[0] = x[1] = 0.5f;
@@ -262,16 +269,20 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
     }
     __syncthreads();
 
-    // ---- 3. radix select: after the four passes sm.prefix[m] is the key of the k_m-th largest
-    //         element of modality m and sm.krem[m] how many elements equal to it are kept.
-#pragma unroll
+    // ---- 3. radix select, 8 bits per pass, most significant first.  A modality is settled as soon as
+    //         the digit bin that holds its k-th largest element must be taken whole (then the bits seen
+    //         so far decide membership); otherwise after four passes sm.prefix[m] is the key of the k-th
+    //         largest element and sm.krem[m] how many elements equal to it are kept.
+#pragma unroll 1
     for (int pass = 0; pass < 4; ++pass) {
         const int shift = 24 - 8 * pass;
         if (pass > 0) {
-            histogram(pass, shift, sm.prefix[0], sm.prefix[1]);
+            const bool d0 = sm.done[0] || sm.k[0] == 0, d1 = sm.done[1] || sm.k[1] == 0;
+            if (d0 && d1) break;                            // block-uniform
+            histogram(pass, shift, sm.prefix[0], sm.prefix[1], d0, d1);
             __syncthreads();
         }
-        if (warp < 2 && sm.k[warp] > 0) {
+        if (warp < 2 && sm.k[warp] > 0 && !sm.done[warp]) {
             // lane L owns the 8 digits 255-8L .. 248-8L (descending); find the digit where the
             // count of elements with a larger digit first reaches k
             const int m = warp, krem = sm.krem[m];
@@ -291,7 +302,12 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
                     if (above < krem && krem <= above + cnt[i]) {
                         sm.prefix[m] |= static_cast<uint32_t>(255 - 8 * lane - i) << shift;
                         sm.krem[m] = krem - above;
-                        if (pass == 3) sm.alltie[m] = (krem - above == cnt[i]);
+                        if (krem - above == cnt[i]) {         // the whole bin is kept: settled
+                            sm.done[m] = 1;
+                            sm.cmask[m] = 0xFFFFFFFFu << shift;
+                        } else if (pass == 3) {
+                            sm.alltie[m] = 0;                 // equal keys straddle the budget: rank them by index
+                        }
                         break;
                     }
                     above += cnt[i];
@@ -306,6 +322,7 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
     const int P = (seq + NT - 1) / NT;
     const int pos0 = tid * P;
     const uint32_t th2 = sm.prefix[0], th3 = sm.prefix[1];
+    const uint32_t cm2 = sm.cmask[0], cm3 = sm.cmask[1];
     const bool any2 = sm.k[0] > 0, any3 = sm.k[1] > 0;
     const int need2 = any2 ? sm.krem[0] : 0, need3 = any3 ? sm.krem[1] : 0;
 
@@ -318,10 +335,10 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
         if (p < seq) {
             if (p >= s.off_txt && p < s.off_txt + s.n_txt) c = 1;
             else if (p >= s.off_2d && p < s.off_2d + n2) {
-                const uint32_t kk = sm.key[p - s.off_2d];
+                const uint32_t kk = sm.key[p - s.off_2d] & cm2;
                 c = !any2 ? 0 : (kk > th2 ? 1 : (kk == th2 ? 2 : 0));
             } else if (p >= s.off_3d && p < s.off_3d + n3) {
-                const uint32_t kk = sm.key[n2 + p - s.off_3d];
+                const uint32_t kk = sm.key[n2 + p - s.off_3d] & cm3;
                 c = !any3 ? 0 : (kk > th3 ? 1 : (kk == th3 ? 3 : 0));
             }
         }
