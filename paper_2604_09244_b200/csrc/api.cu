@@ -21,10 +21,26 @@ struct mvla_ctx {
     float* part;                 // [H][max_batch * max_vis] per-head partial scores
     int64_t part_stride;
     float* attn_ws;              // [max_batch * max_vis]
-    float* l1_ws;                // [max_batch * max_vis]
+    float* l1_ws;                // [2][max_batch * max_vis] feature norms, alternating between steps
     float* ahat_state;           // [n_prune_points][n_slots][max_vis]
     float* mhat_state;           // [n_prune_points][n_slots][4]
-    unsigned long long* acc64;   // [max_batch * max_vis] fixed-point score accumulators, zero between calls
+    unsigned long long* acc64;   // [2][max_batch * max_vis] fixed-point score accumulators, zero between calls,
+                                 // alternating between steps (a step's scoring may run beside the previous
+                                 // step's selection)
+    size_t vis_all;              // max_batch * max_vis
+    unsigned step_parity;
+    // Scoring of a step whose inputs are promised stable runs on a side stream, forked from and joined
+    // back into the caller's stream with events, so that it may run beside the previous step's
+    // selection and row copy.
+    cudaStream_t aux;
+    cudaEvent_t ev_fork, ev_sal, ev_sel[2];    // ev_sel[p]: after the selection that last used scratch set p
+    bool sel_valid[2];
+    // Buffers the previous prune step wrote or read after its selection (outputs, kept indices): the next
+    // step's selection may run beside that step's row copy only if it writes none of them.
+    struct Range { const char* lo; const char* hi; };
+    Range prev_out[10];
+    int n_prev_out;
+    unsigned long long sel_capture[2];         // capture sequence the event belongs to (0: none)
     std::vector<int32_t> t_host; // [n_prune_points][n_slots] steps absorbed so far
     int* status_host;            // mapped pinned word written by kernels whose bounded wait gave up
     int* status_dev;
@@ -218,7 +234,8 @@ int32_t check_sticky(mvla_ctx* ctx)
 // ctx->part, or, when `want_acc64` and the register-resident tensor-core kernel covers the shape, in the
 // fixed-point accumulators ctx->acc64 (*used_acc64 = true).
 int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, const void* k, int64_t rows,
-                           const void* hidden, float* l1, bool want_acc64, bool* used_acc64, cudaStream_t st)
+                           const void* hidden, float* l1, unsigned long long* acc64, bool* used_acc64,
+                           cudaStream_t st)
 {
     if (used_acc64) *used_acc64 = false;
     const mvla_config& c = ctx->cfg;
@@ -238,14 +255,15 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
         if (r != MVLA_OK) return r;
     }
     cudaError_t e;
+    const bool fast = ctx->use_umma && fast_salience_supported(tiles_per_cta);
     if (hidden && l1) {
         e = launch_l1norm(bd, c.dtype, c.d_model, hidden, l1, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
-    if (ctx->use_umma && fast_salience_supported(tiles_per_cta)) {
+    if (fast) {
         e = launch_salience_fast(bd, c.n_heads, c.head_dim, tq, tk, tiles_per_cta, cluster, npad, ctx->part,
-                                 ctx->part_stride, want_acc64 ? ctx->acc64 : nullptr, ctx->status_dev, st);
-        if (used_acc64) *used_acc64 = want_acc64;
+                                 ctx->part_stride, acc64, ctx->status_dev, st);
+        if (used_acc64) *used_acc64 = acc64 != nullptr;
     } else {
         e = launch_salience(bd, c.dtype, c.n_heads, c.head_dim, q, k, tq, tk, ctx->use_umma, tiles_per_cta,
                             cluster, npad, ctx->part, ctx->part_stride, ctx->status_dev, st);
@@ -253,6 +271,19 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
     if (e == cudaErrorInvalidConfiguration) return MVLA_ERR_UNSUPPORTED;
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     return MVLA_OK;
+}
+
+mvla_ctx::Range range_of(const void* p, size_t bytes)
+{
+    const char* c = static_cast<const char*>(p);
+    return {c, c ? c + bytes : c};
+}
+
+bool chunk_is_fast(const mvla_ctx* ctx, const BatchDesc& bd)
+{
+    int max_tiles = 1;
+    for (int b = 0; b < bd.n; ++b) max_tiles = std::max(max_tiles, tiles_of(bd.s[b]));
+    return ctx->use_umma && fast_salience_supported((max_tiles + kMaxCluster - 1) / kMaxCluster);
 }
 
 GateParams gate_params(const mvla_ctx* ctx, int32_t mode, bool has_l1)
@@ -309,6 +340,11 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (c.salience_path == MVLA_SALIENCE_FMA) ctx->use_umma = false;
     ctx->part = ctx->attn_ws = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
     ctx->acc64 = nullptr;
+    ctx->aux = nullptr;
+    ctx->ev_fork = ctx->ev_sal = ctx->ev_sel[0] = ctx->ev_sel[1] = nullptr;
+    ctx->sel_valid[0] = ctx->sel_valid[1] = false;
+    ctx->n_prev_out = -1;                            // unknown: no overlap
+    ctx->sel_capture[0] = ctx->sel_capture[1] = 0;
     ctx->status_host = ctx->status_dev = nullptr;
     ctx->last_cuda = cudaSuccess;
     ctx->tm_ptr[0] = ctx->tm_ptr[1] = nullptr;
@@ -326,11 +362,16 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     };
     alloc(&ctx->part, vis_all * c.n_heads);
     alloc(&ctx->attn_ws, vis_all);
-    alloc(&ctx->l1_ws, vis_all);
+    alloc(&ctx->l1_ws, 2 * vis_all);
+    ctx->vis_all = vis_all;
+    ctx->step_parity = 0;
     alloc(&ctx->ahat_state, n_state * ctx->max_vis);
     alloc(&ctx->mhat_state, n_state * 4);
-    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->acc64), vis_all * sizeof(unsigned long long));
-    if (e == cudaSuccess) e = cudaMemset(ctx->acc64, 0, vis_all * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->acc64), 2 * vis_all * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(ctx->acc64, 0, 2 * vis_all * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->aux, cudaStreamNonBlocking);
+    for (cudaEvent_t* ev : {&ctx->ev_fork, &ctx->ev_sal, &ctx->ev_sel[0], &ctx->ev_sel[1]})
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&ctx->status_host), sizeof(int), cudaHostAllocMapped);
     if (e == cudaSuccess) {
         *ctx->status_host = 0;
@@ -363,6 +404,12 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     cudaFree(ctx->ahat_state);
     cudaFree(ctx->mhat_state);
     cudaFree(ctx->acc64);
+    if (ctx->aux) {
+        cudaStreamSynchronize(ctx->aux);
+        cudaStreamDestroy(ctx->aux);
+    }
+    for (cudaEvent_t ev : {ctx->ev_fork, ctx->ev_sal, ctx->ev_sel[0], ctx->ev_sel[1]})
+        if (ev) cudaEventDestroy(ev);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     delete ctx;
 }
@@ -378,6 +425,7 @@ int32_t mvla_salience(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, 
     if (rc != MVLA_OK) return rc;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return MVLA_ERR_CUDA;
+    ctx->n_prev_out = -1;                            // what the stream ran last is no longer a known prune step
     Plan plan;
     rc = make_plan(ctx, 0, batch, samples, MVLA_MODE_FIXED, 0, false, &plan);
     if (rc != MVLA_OK) return rc;
@@ -385,7 +433,7 @@ int32_t mvla_salience(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, 
     const bool want_l1 = hidden && l1_out;
     for (int first = 0; first < batch; first += kMaxChunk) {
         const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
-        rc = run_salience_chunk(ctx, bd, q, k, rows, want_l1 ? hidden : nullptr, l1_out, false, nullptr, st);
+        rc = run_salience_chunk(ctx, bd, q, k, rows, want_l1 ? hidden : nullptr, l1_out, nullptr, nullptr, st);
         if (rc != MVLA_OK) return rc;
     }
     const cudaError_t e = launch_head_reduce(ctx->part, ctx->part_stride, ctx->cfg.n_heads, plan.total_vis, attn_out, st);
@@ -406,6 +454,7 @@ int32_t mvla_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvl
     if (mode == MVLA_MODE_ADAPTIVE && !l1) return MVLA_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return MVLA_ERR_CUDA;
+    ctx->n_prev_out = -1;                            // what the stream ran last is no longer a known prune step
     Plan plan;
     rc = make_plan(ctx, prune_point, batch, samples, mode, flags, true, &plan);
     if (rc != MVLA_OK) return rc;
@@ -446,6 +495,7 @@ int32_t mvla_compact(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, c
     if (rc != MVLA_OK) return rc;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return MVLA_ERR_CUDA;
+    ctx->n_prev_out = -1;                            // what the stream ran last is no longer a known prune step
     Plan plan;
     rc = make_plan(ctx, 0, batch, samples, MVLA_MODE_FIXED, 0, false, &plan);
     if (rc != MVLA_OK) return rc;
@@ -468,7 +518,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
 {
     if (!ctx || !in || !out || !in->q || !in->k || !out->kept_idx || !out->out_offsets || in->rows < 1)
         return MVLA_ERR_INVALID_ARG;
-    if (flags & ~(MVLA_FLAG_RESET_STATE | MVLA_FLAG_NO_STATE_UPDATE)) return MVLA_ERR_INVALID_ARG;
+    if (flags & ~(MVLA_FLAG_RESET_STATE | MVLA_FLAG_NO_STATE_UPDATE | MVLA_FLAG_INPUTS_STABLE)) return MVLA_ERR_INVALID_ARG;
     if (mode == MVLA_MODE_ADAPTIVE && !in->hidden) return MVLA_ERR_INVALID_ARG;
     const void* src[3] = {in->hidden, in->k, in->v};
     void* dst[3] = {out->out_hidden, out->out_k, out->out_v};
@@ -494,26 +544,83 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
     job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
 
+    // scratch set of this step
+    ctx->step_parity ^= 1u;
+    unsigned long long* acc64 = ctx->acc64 + ctx->step_parity * ctx->vis_all;
+    float* l1_ws = ctx->l1_ws + ctx->step_parity * ctx->vis_all;
+    // With stable inputs (and the fast scoring kernel, whose scratch alternates between two sets) the
+    // scoring goes to the side stream.  It must not start before the selection that last used this
+    // scratch set (two steps ago) has finished; nothing else of the earlier work concerns it.
+    bool forked = false;
+    unsigned long long cap_id = 0;
+    const unsigned par = ctx->step_parity;
+    if ((flags & MVLA_FLAG_INPUTS_STABLE) && batch <= kMaxChunk && chunk_is_fast(ctx, chunk_of(plan, 0, batch))) {
+        cudaStreamCaptureStatus cst = cudaStreamCaptureStatusNone;
+        if (cudaStreamGetCaptureInfo(st, &cst, &cap_id) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
+        if (cst != cudaStreamCaptureStatusActive) cap_id = 0;
+        cudaEvent_t dep = ctx->ev_sel[par];
+        if (!(ctx->sel_valid[par] && ctx->sel_capture[par] == cap_id)) {
+            dep = ctx->ev_fork;                      // no usable history: after everything enqueued so far
+            if (cudaEventRecord(dep, st) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
+        }
+        if (cudaStreamWaitEvent(ctx->aux, dep, 0) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
+        forked = true;
+    }
+    // May this step's selection run beside the previous step's row copy?  Only if that copy is known
+    // (the previous call on this context was a forked prune step) and touches nothing written here.
+    const size_t nvis_b = static_cast<size_t>(plan.total_vis), nout_b = static_cast<size_t>(plan.total_out);
+    const mvla_ctx::Range sel_w[7] = {
+        range_of(out->kept_idx, nout_b * 4), range_of(out->out_offsets, (batch + 1) * 4u),
+        range_of(out->budgets, batch * 8u), range_of(out->attn, nvis_b * 4), range_of(out->ahat, nvis_b * 4),
+        range_of(out->z, nvis_b * 4), range_of(out->diag, batch * sizeof(mvla_diag))};
+    bool sel_beside = forked && ctx->n_prev_out >= 0;
+    for (int i = 0; sel_beside && i < 7; ++i)
+        for (int j = 0; sel_beside && j < ctx->n_prev_out; ++j)
+            if (sel_w[i].lo && sel_w[i].lo < ctx->prev_out[j].hi && ctx->prev_out[j].lo < sel_w[i].hi) sel_beside = false;
+    if (forked) {                                    // remember what this step's copy touches
+        const size_t hb = static_cast<size_t>(ctx->cfg.d_model) * ctx->elem, kb = static_cast<size_t>(kv_bytes);
+        int m = 0;
+        for (int i = 0; i < 7; ++i) if (sel_w[i].lo) ctx->prev_out[m++] = sel_w[i];
+        if (out->out_hidden) ctx->prev_out[m++] = range_of(out->out_hidden, nout_b * hb);
+        if (out->out_k) ctx->prev_out[m++] = range_of(out->out_k, nout_b * kb);
+        if (out->out_v) ctx->prev_out[m++] = range_of(out->out_v, nout_b * kb);
+        ctx->n_prev_out = m;
+    } else {
+        ctx->n_prev_out = -1;
+    }
     for (int first = 0; first < batch; first += kMaxChunk) {
         const int n = std::min(kMaxChunk, batch - first);
         const BatchDesc bd = chunk_of(plan, first, n);
         bool used_acc64 = false;
-        rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, ctx->l1_ws, true,
-                                &used_acc64, st);
+        rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, l1_ws, acc64,
+                                &used_acc64, forked ? ctx->aux : st);
         if (rc != MVLA_OK) return rc;
+        if (forked) {                                // join: the selection needs the scores
+            if (cudaEventRecord(ctx->ev_sal, ctx->aux) != cudaSuccess ||
+                cudaStreamWaitEvent(st, ctx->ev_sal, 0) != cudaSuccess)
+                return fail_cuda(ctx, cudaGetLastError());
+        }
         SelectIO io;
         std::memset(&io, 0, sizeof io);
         io.n_heads = ctx->cfg.n_heads;
-        if (used_acc64) io.acc64 = ctx->acc64;
+        if (used_acc64) io.acc64 = acc64;
         else { io.part = ctx->part; io.part_stride = ctx->part_stride; }
-        io.l1 = adaptive ? ctx->l1_ws : nullptr;
+        io.l1 = adaptive ? l1_ws : nullptr;
         io.ahat_state = ctx->ahat_state; io.mhat_state = ctx->mhat_state;
         io.kept_idx = out->kept_idx; io.out_offsets = out->out_offsets; io.budgets = out->budgets;
         io.attn_out = out->attn; io.ahat_out = out->ahat; io.z_out = out->z; io.diag = out->diag;
         io.chunk_first = first; io.total_out = plan.total_out; io.write_total = first + n == batch;
         io.n_in_launch = n;
+        io.beside_previous = forked && sel_beside;
         cudaError_t e = launch_select(bd, gp, io, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
+        if (forked) {
+            if (cudaEventRecord(ctx->ev_sel[par], st) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
+            ctx->sel_valid[par] = true;
+            ctx->sel_capture[par] = cap_id;
+        } else {
+            ctx->sel_valid[par] = false;             // this set was used outside the event chain
+        }
         const int32_t row0 = bd.s[0].out_off;
         const int32_t nrows = bd.s[n - 1].out_off + bd.s[n - 1].n_out - row0;
         e = launch_compact(bd, job, out->kept_idx, nrows, row0, nullptr, first, batch, st);

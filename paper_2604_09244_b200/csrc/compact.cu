@@ -38,7 +38,6 @@ compact_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ Com
                int32_t chunk_rows, int32_t chunk_row0, const int32_t* __restrict__ out_offsets,
                int32_t chunk_first, int32_t batch_total)
 {
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = threadIdx.x & 31;
     const int64_t unit = static_cast<int64_t>(blockIdx.x) * kWarpsPerBlock + (threadIdx.x >> 5);
     const int per_row = a.seg_begin[3];
@@ -48,6 +47,9 @@ compact_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ Com
     const int orow = chunk_row0 + r;
 
     asm volatile("griddepcontrol.wait;" ::: "memory");      // kept_idx comes from the kernel before this one
+    // Only now may the next kernel start: a selection of the next step that runs beside this copy can
+    // rely on this step's selection (which owns the smoothed state) being complete.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // which sample owns output row `orow` (samples are few: linear scan)
     int b = 0;
     if (out_offsets) {            // offsets known only on the device: scan the whole batch

@@ -250,7 +250,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     __syncthreads();
 
     // ---- per key: sum over queries of the normalised probabilities (this head's contribution)
-    pdl_wait();                               // the accumulators are read and cleared by the previous step's select
+    pdl_wait();                               // the accumulators were read and cleared by an earlier selection
 #pragma unroll
     for (int t = 0; t < NTILE; ++t) {
         if (valid[t] <= 0) continue;

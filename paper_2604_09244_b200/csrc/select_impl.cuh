@@ -124,7 +124,10 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     for (int i = tid; i < 4 * 2 * 256; i += NT) (&sm.hist[0][0][0])[i] = 0;
     if (tid < 2) { sm.prefix[tid] = 0u; sm.alltie[tid] = 1; sm.done[tid] = 0; sm.cmask[tid] = 0xFFFFFFFFu; }
-    asm volatile("griddepcontrol.wait;" ::: "memory");      // scores come from the kernel before this one
+    // Scores normally come from the kernel before this one.  When the host has established that they
+    // do not (they arrive through an event dependency) and that no buffer written here is touched by
+    // that kernel, the wait moves to the end: completion still implies completion of all earlier work.
+    if (!io.beside_previous) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- 1. all loads first
     float a[EPT], prev[EPT], nrm[EPT];
@@ -363,6 +366,7 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
     int pos = block_exscan<NT>(kept, sm.scan);
     for (int i = 0; i < P; ++i)
         if ((mask >> i) & 1ull) io.kept_idx[s.out_off + pos++] = pos0 + i;
+    if (io.beside_previous) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 }  // namespace mvla

@@ -24,7 +24,7 @@ _ERR_NAMES = {-1: "MVLA_ERR_INVALID_ARG", -2: "MVLA_ERR_UNSUPPORTED", -3: "MVLA_
               -7: "MVLA_ERR_STATE"}
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 MODE_FIXED, MODE_ADAPTIVE = 0, 1
-FLAG_RESET_STATE, FLAG_NO_STATE_UPDATE = 1, 2
+FLAG_RESET_STATE, FLAG_NO_STATE_UPDATE, FLAG_INPUTS_STABLE = 1, 2, 4
 SALIENCE_AUTO, SALIENCE_FMA = 0, 1
 SET_2D, SET_3D = 1, 2
 

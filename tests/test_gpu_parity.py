@@ -282,3 +282,64 @@ def test_error_codes_never_fault():
         mvla.PruneContext(dtype=torch.bfloat16, n_heads=4, head_dim=96, d_model=256, max_batch=1, max_text=8,
                           max_2d=8, max_3d=8)
     assert e.value.code == mvla.ERR_UNSUPPORTED
+
+
+def test_inputs_stable_flag_changes_timing_only():
+    # back-to-back steps on rotating buffers, with and without the promise that the inputs are not
+    # produced by the preceding work: identical results, step after step
+    wls = [W.config2_single_frame(seed=s) for s in (31, 32, 33)]
+    wl = wls[0]
+    ctx = mvla.context_for(wl)
+    devs = [device_tensors(w) for w in wls]
+    ref = []
+    for d in devs:
+        o = ctx.prune_step(0, wl.samples, wl.mode, d["q"], d["k"], d["v"], d["hidden"], flags=mvla.FLAG_RESET_STATE)
+        torch.cuda.synchronize()
+        n = o.total_kept
+        ref.append((o.attn.clone(), o.kept_idx[:n].clone(), o.out_hidden[:n].clone(), o.out_v[:n].clone()))
+    outs = [ctx.alloc_outputs(wl.samples, extras=True) for _ in range(3)]
+    for rep in range(30):                                   # no synchronisation between the steps
+        i = rep % 3
+        d = devs[i]
+        ctx.prune_step(0, wl.samples, wl.mode, d["q"], d["k"], d["v"], d["hidden"],
+                       flags=mvla.FLAG_RESET_STATE | mvla.FLAG_INPUTS_STABLE, out=outs[i])
+    torch.cuda.synchronize()
+    for i in range(3):
+        o, n = outs[i], len(ref[i][1])
+        got = (o.attn, o.kept_idx[:n], o.out_hidden[:n], o.out_v[:n])
+        assert all(torch.equal(x, y) for x, y in zip(got, ref[i]))
+    ctx.close()
+
+
+def test_pipelined_steps_with_state_match_serial_steps():
+    # action steps with carry-over, enqueued back to back without synchronisation and with the
+    # stable-inputs promise (scoring, selection and row copy of neighbouring steps overlap), against the
+    # same steps run one at a time: identical bits, including when output buffers are reused
+    wl = W.small_workload(43, batch=3, D=256, H=4, d=128, dtype="bf16", n_txt=(5, 19, 33), n_2d=(70, 130, 260),
+                          n_3d=(150, 37, 300), keep=(0.4, 0.3, 0.55), steps=10, cold_start=1)
+    devs = [device_tensors(wl, t) for t in range(10)]
+
+    def run(flag, n_out, sync):
+        ctx = mvla.context_for(wl)
+        outs = [ctx.alloc_outputs(wl.samples, extras=True) for _ in range(n_out)]
+        res = []
+        for t, d in enumerate(devs):
+            o = ctx.prune_step(0, wl.samples, wl.mode, d["q"], d["k"], d["v"], d["hidden"],
+                               flags=flag | (mvla.FLAG_RESET_STATE if t == 0 else 0), out=outs[t % n_out])
+            if sync:
+                torch.cuda.synchronize()
+            res.append((o.total_kept, t % n_out))
+        torch.cuda.synchronize()
+        snap = [None] * 10
+        for t in range(10 - n_out, 10):                       # the last n_out steps are still in their buffers
+            o, n = outs[t % n_out], res[t][0]
+            snap[t] = (o.ahat.clone(), o.kept_idx[:n].clone(), o.budgets.clone(), o.out_hidden[:n].clone(),
+                       o.out_k[:n].clone())
+        ctx.close()
+        return snap
+
+    ref = run(0, 10, True)
+    for n_out in (10, 3, 1):                                  # 1: every step reuses the same output buffers
+        got = run(mvla.FLAG_INPUTS_STABLE, n_out, False)
+        for t in range(10 - n_out, 10):
+            assert all(torch.equal(x, y) for x, y in zip(got[t], ref[t])), (n_out, t)
