@@ -32,8 +32,8 @@ struct mvla_ctx {
     // Scoring of a step whose inputs are promised stable runs on a side stream, forked from and joined
     // back into the caller's stream with events, so that it may run beside the previous step's
     // selection and row copy.
-    cudaStream_t aux;
-    cudaEvent_t ev_fork, ev_sal, ev_sel[2];    // ev_sel[p]: after the selection that last used scratch set p
+    cudaStream_t aux[2];                       // one per scratch set, so that consecutive scorings do not serialise
+    cudaEvent_t ev_fork, ev_sal[2], ev_sel[2]; // ev_sel[p]: after the selection that last used scratch set p
     bool sel_valid[2];
     // Buffers the previous prune step wrote or read after its selection (outputs, kept indices): the next
     // step's selection may run beside that step's row copy only if it writes none of them.
@@ -235,7 +235,7 @@ int32_t check_sticky(mvla_ctx* ctx)
 // fixed-point accumulators ctx->acc64 (*used_acc64 = true).
 int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, const void* k, int64_t rows,
                            const void* hidden, float* l1, unsigned long long* acc64, bool* used_acc64,
-                           cudaStream_t st)
+                           bool free_running, cudaStream_t st)
 {
     if (used_acc64) *used_acc64 = false;
     const mvla_config& c = ctx->cfg;
@@ -262,7 +262,7 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
     }
     if (fast) {
         e = launch_salience_fast(bd, c.n_heads, c.head_dim, tq, tk, tiles_per_cta, cluster, npad, ctx->part,
-                                 ctx->part_stride, acc64, ctx->status_dev, st);
+                                 ctx->part_stride, acc64, ctx->status_dev, free_running, st);
         if (used_acc64) *used_acc64 = acc64 != nullptr;
     } else {
         e = launch_salience(bd, c.dtype, c.n_heads, c.head_dim, q, k, tq, tk, ctx->use_umma, tiles_per_cta,
@@ -340,8 +340,8 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (c.salience_path == MVLA_SALIENCE_FMA) ctx->use_umma = false;
     ctx->part = ctx->attn_ws = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
     ctx->acc64 = nullptr;
-    ctx->aux = nullptr;
-    ctx->ev_fork = ctx->ev_sal = ctx->ev_sel[0] = ctx->ev_sel[1] = nullptr;
+    ctx->aux[0] = ctx->aux[1] = nullptr;
+    ctx->ev_fork = ctx->ev_sal[0] = ctx->ev_sal[1] = ctx->ev_sel[0] = ctx->ev_sel[1] = nullptr;
     ctx->sel_valid[0] = ctx->sel_valid[1] = false;
     ctx->n_prev_out = -1;                            // unknown: no overlap
     ctx->sel_capture[0] = ctx->sel_capture[1] = 0;
@@ -369,8 +369,9 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     alloc(&ctx->mhat_state, n_state * 4);
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->acc64), 2 * vis_all * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(ctx->acc64, 0, 2 * vis_all * sizeof(unsigned long long));
-    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->aux, cudaStreamNonBlocking);
-    for (cudaEvent_t* ev : {&ctx->ev_fork, &ctx->ev_sal, &ctx->ev_sel[0], &ctx->ev_sel[1]})
+    for (cudaStream_t* sp : {&ctx->aux[0], &ctx->aux[1]})
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(sp, cudaStreamNonBlocking);
+    for (cudaEvent_t* ev : {&ctx->ev_fork, &ctx->ev_sal[0], &ctx->ev_sal[1], &ctx->ev_sel[0], &ctx->ev_sel[1]})
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&ctx->status_host), sizeof(int), cudaHostAllocMapped);
     if (e == cudaSuccess) {
@@ -404,11 +405,12 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     cudaFree(ctx->ahat_state);
     cudaFree(ctx->mhat_state);
     cudaFree(ctx->acc64);
-    if (ctx->aux) {
-        cudaStreamSynchronize(ctx->aux);
-        cudaStreamDestroy(ctx->aux);
-    }
-    for (cudaEvent_t ev : {ctx->ev_fork, ctx->ev_sal, ctx->ev_sel[0], ctx->ev_sel[1]})
+    for (cudaStream_t sp : {ctx->aux[0], ctx->aux[1]})
+        if (sp) {
+            cudaStreamSynchronize(sp);
+            cudaStreamDestroy(sp);
+        }
+    for (cudaEvent_t ev : {ctx->ev_fork, ctx->ev_sal[0], ctx->ev_sal[1], ctx->ev_sel[0], ctx->ev_sel[1]})
         if (ev) cudaEventDestroy(ev);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     delete ctx;
@@ -433,7 +435,7 @@ int32_t mvla_salience(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, 
     const bool want_l1 = hidden && l1_out;
     for (int first = 0; first < batch; first += kMaxChunk) {
         const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
-        rc = run_salience_chunk(ctx, bd, q, k, rows, want_l1 ? hidden : nullptr, l1_out, nullptr, nullptr, st);
+        rc = run_salience_chunk(ctx, bd, q, k, rows, want_l1 ? hidden : nullptr, l1_out, nullptr, nullptr, false, st);
         if (rc != MVLA_OK) return rc;
     }
     const cudaError_t e = launch_head_reduce(ctx->part, ctx->part_stride, ctx->cfg.n_heads, plan.total_vis, attn_out, st);
@@ -563,7 +565,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
             dep = ctx->ev_fork;                      // no usable history: after everything enqueued so far
             if (cudaEventRecord(dep, st) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
         }
-        if (cudaStreamWaitEvent(ctx->aux, dep, 0) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
+        if (cudaStreamWaitEvent(ctx->aux[par], dep, 0) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
         forked = true;
     }
     // May this step's selection run beside the previous step's row copy?  Only if that copy is known
@@ -593,11 +595,11 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         const BatchDesc bd = chunk_of(plan, first, n);
         bool used_acc64 = false;
         rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, l1_ws, acc64,
-                                &used_acc64, forked ? ctx->aux : st);
+                                &used_acc64, forked, forked ? ctx->aux[par] : st);
         if (rc != MVLA_OK) return rc;
         if (forked) {                                // join: the selection needs the scores
-            if (cudaEventRecord(ctx->ev_sal, ctx->aux) != cudaSuccess ||
-                cudaStreamWaitEvent(st, ctx->ev_sal, 0) != cudaSuccess)
+            if (cudaEventRecord(ctx->ev_sal[par], ctx->aux[par]) != cudaSuccess ||
+                cudaStreamWaitEvent(st, ctx->ev_sal[par], 0) != cudaSuccess)
                 return fail_cuda(ctx, cudaGetLastError());
         }
         SelectIO io;

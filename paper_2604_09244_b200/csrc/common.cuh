@@ -84,11 +84,13 @@ inline cudaLaunchAttribute pdl_attribute()
 // bf16 tensor-core salience with logits held in registers (one or two key tiles per CTA).  With
 // `acc64` the per-head contributions are added into 64-bit fixed-point accumulators (scale 2^60, one
 // per visual token, zero on entry); without it they go to part[h][vis] as in launch_salience.
+// `free_running`: the kernel does not wait for the kernel before it in its stream (the caller orders
+// everything it depends on with events).
 bool fast_salience_supported(int tiles_per_cta);
 cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int head_dim, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
-                                 cudaStream_t stream);
+                                 bool free_running, cudaStream_t stream);
 
 
 // Salience: per-head partial scores part[h][vis] (already scaled by 1/(H n_t)).

@@ -82,7 +82,7 @@ __device__ __forceinline__ void block_sum4(float (&x)[4], float (*scratch)[4], f
 
 // Exclusive block scan of one int per thread.
 template <int NT>
-__device__ __forceinline__ int block_exscan(int x, int* warp_tot)
+__device__ __forceinline__ int block_exscan(int x, int* warp_tot, int* total)
 {
     constexpr int NW = NT / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -104,8 +104,10 @@ __device__ __forceinline__ int block_exscan(int x, int* warp_tot)
             if (lane >= off) winc += n;
         }
         if (lane < NW) warp_tot[lane] = winc - t;          // exclusive prefix of the warp totals
+        if (lane == 31) warp_tot[NW] = winc;               // grand total
     }
     __syncthreads();
+    *total = warp_tot[NW];
     return warp_tot[warp] + inc - x;
 }
 
@@ -133,9 +135,11 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
     float a[EPT], prev[EPT], nrm[EPT];
     unsigned long long fx[EPT];
 #pragma unroll
+    for (int e = 0; e < EPT; ++e) { a[e] = 0.f; prev[e] = 0.f; nrm[e] = 0.f; fx[e] = 0ull; }
+#pragma unroll
     for (int e = 0; e < EPT; ++e) {
+        if (e * NT >= nv) break;                           // uniform: nobody owns an element in this slice
         const int j = tid + e * NT;
-        a[e] = 0.f; prev[e] = 0.f; nrm[e] = 0.f; fx[e] = 0ull;
         if (j < nv) {
             if (io.acc64) fx[e] = __ldcg(io.acc64 + s.vis_off + j);        // written by other CTAs' atomics
             else if (!io.part) a[e] = io.attn[s.vis_off + j];
@@ -146,6 +150,7 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
     if (io.part && !io.acc64) {                            // per-head fp32 partials, summed in head order
 #pragma unroll
         for (int e = 0; e < EPT; ++e) {
+            if (e * NT >= nv) break;
             const int j = tid + e * NT;
             if (j < nv) {
                 float acc = 0.f;
@@ -159,9 +164,11 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
     float sums[4] = {0.f, 0.f, 0.f, 0.f};     // sum a over 2D, over 3D, sum l1 over 2D, over 3D
     float ssm[4] = {0.f, 0.f, 0.f, 0.f};      // sums of the smoothed scores per modality (for z)
 #pragma unroll
+    for (int e = 0; e < EPT; ++e) key[e] = 0u;
+#pragma unroll
     for (int e = 0; e < EPT; ++e) {
+        if (e * NT >= nv) break;
         const int j = tid + e * NT;
-        key[e] = 0u;
         if (j < nv) {
             if (io.acc64) {
                 a[e] = static_cast<float>(__ull2double_rn(fx[e]) * kFixInv);
@@ -187,6 +194,7 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
         const float f2 = static_cast<float>(n2) / sm.tot[0], f3 = static_cast<float>(n3) / sm.tot[1];
 #pragma unroll
         for (int e = 0; e < EPT; ++e) {
+            if (e * NT >= nv) break;
             const int j = tid + e * NT;
             if (j < nv) io.z_out[s.vis_off + j] = key_to_float(key[e]) * (j < n2 ? f2 : f3);
         }
@@ -320,52 +328,53 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
         __syncthreads();
     }
 
-    // ---- 4. emission in sequence order.  Thread t owns positions [t*P, t*P + P), P <= 64.
-    const int seq = s.n_txt + nv;
-    const int P = (seq + NT - 1) / NT;
-    const int pos0 = tid * P;
+    // ---- 4. emission.  Each thread decides its own elements from the keys it holds in registers; one
+    //         block scan per slice of NT elements (in visual order: 2D first) ranks the kept ones.  The
+    //         three segments are contiguous, so a kept token's output row is the number of rows that the
+    //         segments lying before its own contribute plus its rank inside its modality.
     const uint32_t th2 = sm.prefix[0], th3 = sm.prefix[1];
     const uint32_t cm2 = sm.cmask[0], cm3 = sm.cmask[1];
-    const bool any2 = sm.k[0] > 0, any3 = sm.k[1] > 0;
-    const int need2 = any2 ? sm.krem[0] : 0, need3 = any3 ? sm.krem[1] : 0;
+    const int k2 = sm.k[0], k3 = sm.k[1];
+    const int need2 = k2 > 0 ? sm.krem[0] : 0, need3 = k3 > 0 ? sm.krem[1] : 0;
+    const bool rank_ties = !(sm.alltie[0] && sm.alltie[1]);          // block-uniform
+    const int base2 = (s.off_txt < s.off_2d ? s.n_txt : 0) + (s.off_3d < s.off_2d ? k3 : 0);
+    const int base3 = (s.off_txt < s.off_3d ? s.n_txt : 0) + (s.off_2d < s.off_3d ? k2 : 0);
+    const int baset = (s.off_2d < s.off_txt ? k2 : 0) + (s.off_3d < s.off_txt ? k3 : 0);
+    for (int i = tid; i < s.n_txt; i += NT) io.kept_idx[s.out_off + baset + i] = s.off_txt + i;
 
-    // per position 2 bits: 0 dropped, 1 kept, 2 tie in 2D, 3 tie in 3D
-    unsigned long long cls_lo = 0ull, cls_hi = 0ull;
-    int ties = 0;                                   // low 16 bits: 2D ties, high 16 bits: 3D ties
-    for (int i = 0; i < P; ++i) {
-        const int p = pos0 + i;
-        int c = 0;
-        if (p < seq) {
-            if (p >= s.off_txt && p < s.off_txt + s.n_txt) c = 1;
-            else if (p >= s.off_2d && p < s.off_2d + n2) {
-                const uint32_t kk = sm.key[p - s.off_2d] & cm2;
-                c = !any2 ? 0 : (kk > th2 ? 1 : (kk == th2 ? 2 : 0));
-            } else if (p >= s.off_3d && p < s.off_3d + n3) {
-                const uint32_t kk = sm.key[n2 + p - s.off_3d] & cm3;
-                c = !any3 ? 0 : (kk > th3 ? 1 : (kk == th3 ? 3 : 0));
+    int run_kept = 0, run_t2 = 0, run_t3 = 0;
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+        if (e * NT >= nv) break;                                      // uniform
+        const int j = tid + e * NT;
+        int c = 0;                                                    // 0 dropped, 1 kept, 2 tie in 2D, 3 tie in 3D
+        if (j < nv) {
+            if (j < n2) {
+                const uint32_t kk = key[e] & cm2;
+                c = k2 <= 0 ? 0 : (kk > th2 ? 1 : (kk == th2 ? 2 : 0));
+            } else {
+                const uint32_t kk = key[e] & cm3;
+                c = k3 <= 0 ? 0 : (kk > th3 ? 1 : (kk == th3 ? 3 : 0));
             }
         }
-        cls_lo |= static_cast<unsigned long long>(c & 1) << i;
-        cls_hi |= static_cast<unsigned long long>(c >> 1) << i;
-        ties += (c == 2) + ((c == 3) << 16);
+        if (rank_ties) {                                              // equal keys straddle a budget: lower index wins
+            int tot = 0;
+            const int tr = block_exscan<NT>((c == 2) + ((c == 3) << 16), sm.scan, &tot);
+            if (c == 2) c = (run_t2 + (tr & 0xFFFF)) < need2 ? 1 : 0;
+            else if (c == 3) c = (run_t3 + (tr >> 16)) < need3 ? 1 : 0;
+            run_t2 += tot & 0xFFFF;
+            run_t3 += tot >> 16;
+        } else if (c >= 2) {
+            c = 1;                                                    // every element equal to the threshold is kept
+        }
+        int tot = 0;
+        const int r = run_kept + block_exscan<NT>(c, sm.scan, &tot);
+        run_kept += tot;
+        if (c) {
+            if (j < n2) io.kept_idx[s.out_off + base2 + r] = s.off_2d + j;
+            else        io.kept_idx[s.out_off + base3 + (r - k2)] = s.off_3d + (j - n2);
+        }
     }
-    int r2 = 0, r3 = 0;
-    if (!(sm.alltie[0] && sm.alltie[1])) {           // ranks among equal keys, in index order (block-uniform branch)
-        const int tie_rank = block_exscan<NT>(ties, sm.scan);
-        r2 = tie_rank & 0xFFFF;
-        r3 = tie_rank >> 16;
-    }
-    unsigned long long mask = 0ull;
-    int kept = 0;
-    for (int i = 0; i < P; ++i) {
-        int c = static_cast<int>((cls_lo >> i) & 1ull) | (static_cast<int>((cls_hi >> i) & 1ull) << 1);
-        if (c == 2) c = (r2++ < need2) ? 1 : 0;                  // lower index wins
-        else if (c == 3) c = (r3++ < need3) ? 1 : 0;
-        if (c) { mask |= 1ull << i; ++kept; }
-    }
-    int pos = block_exscan<NT>(kept, sm.scan);
-    for (int i = 0; i < P; ++i)
-        if ((mask >> i) & 1ull) io.kept_idx[s.out_off + pos++] = pos0 + i;
     if (io.beside_previous) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
