@@ -59,11 +59,10 @@ class CDiag(C.Structure):
                 ("near_half", C.c_int32), ("near_gate", C.c_int32)]
 
 
-def lib():
-    global _lib
-    if _lib is None:
-        build()
-        L = C.CDLL(_LIB_PATH)
+def load(path: str):
+    """Load an oracle library from `path` and declare its signatures."""
+    if True:
+        L = C.CDLL(path)
         fp, dp, ip = C.POINTER(C.c_float), C.POINTER(C.c_double), C.POINTER(C.c_int32)
         sp, pp = C.POINTER(CSample), C.POINTER(CParams)
         L.oracle_salience.argtypes = [fp, fp, C.c_int32, C.c_int32, sp, dp]
@@ -96,7 +95,14 @@ def lib():
         L.oracle_prune_step.restype = C.c_int32
         L.oracle_num_threads.argtypes = []
         L.oracle_num_threads.restype = C.c_int32
-        _lib = L
+    return L
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = load(_LIB_PATH)
     return _lib
 
 

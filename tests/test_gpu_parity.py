@@ -343,3 +343,26 @@ def test_pipelined_steps_with_state_match_serial_steps():
         got = run(mvla.FLAG_INPUTS_STABLE, n_out, False)
         for t in range(10 - n_out, 10):
             assert all(torch.equal(x, y) for x, y in zip(got[t], ref[t])), (n_out, t)
+
+
+def test_step_segments_in_order_3d_text_2d():
+    # the three segments may come in any order; here [3D | text | 2D], two samples, adaptive budgets
+    base = W.small_workload(47, batch=2, D=256, H=4, d=128, dtype="bf16", n_txt=(9, 30), n_2d=(140, 77),
+                            n_3d=(200, 301), keep=(0.4, 0.3))
+    t = base.steps[0]
+    order, samples = [], []
+    for s in base.samples:
+        r = s.seq_off
+        order += list(range(r + s.off_3d, r + s.off_3d + s.n_3d)) + list(range(r + s.off_txt, r + s.off_txt + s.n_txt)) \
+            + list(range(r + s.off_2d, r + s.off_2d + s.n_2d))
+        samples.append(W.Sample(seq_off=s.seq_off, off_3d=0, n_3d=s.n_3d, off_txt=s.n_3d, n_txt=s.n_txt,
+                                off_2d=s.n_3d + s.n_txt, n_2d=s.n_2d, keep_total=s.keep_total,
+                                state_slot=s.state_slot))
+    order = np.array(order)
+    ten = W.Tensors(hidden=np.ascontiguousarray(t.hidden[order]), q=np.ascontiguousarray(t.q[order]),
+                    k=np.ascontiguousarray(t.k[order]), v=np.ascontiguousarray(t.v[order]))
+    wl = W.Workload("segments_3d_txt_2d", base.dtype, base.n_heads, base.head_dim, base.d_model, base.mode,
+                    samples, [ten])
+    ctx = mvla.context_for(wl)
+    out, refs = run_and_check_step(ctx, wl, 0, _fresh_states(wl))
+    ctx.close()

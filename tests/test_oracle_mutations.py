@@ -1,0 +1,80 @@
+"""Do the pins bite?  Each case plants one plausible mistake in a COPY of the oracle's C source (on the
+CPU, in a temporary directory), builds it, runs the pin tests against the mutated library and demands
+that at least one of them fails.  The oracle in the repository is never touched."""
+import os
+import subprocess
+
+import pytest
+
+import oracle
+import test_oracle_pins as pins
+
+SRC = os.path.join(os.path.dirname(oracle.__file__), "mvla_oracle.c")
+HDR = os.path.join(os.path.dirname(oracle.__file__), "mvla_oracle.h")
+
+PIN_TESTS = [getattr(pins, n) for n in dir(pins) if n.startswith("test_")]
+
+MUTATIONS = {
+    "logit scale dropped": ("logit[j] = acc / sqrt((double)d);", "logit[j] = acc;"),
+    "logit sign flipped": ("acc += (double)qi[c] * (double)kj[c];", "acc -= (double)qi[c] * (double)kj[c];"),
+    "query head offset wrong": ("+ s->off_txt + i) * row + (int64_t)h * d;", "+ s->off_txt + i) * row + (int64_t)h;"),
+    "key row ignores the sample offset": ("const float *kj = k + ((int64_t)s->seq_off + vis_row(s, j)) * row",
+                                          "const float *kj = k + ((int64_t)vis_row(s, j)) * row"),
+    "mean over heads only": ("a_out[j] = acc / ((double)H * (double)nt);", "a_out[j] = acc / ((double)H);"),
+    "softmax denominator over 2D keys only": ("for (int32_t j = 0; j < nv; ++j) den += exp(logit[j] - mx);",
+                                              "for (int32_t j = 0; j < s->n_2d; ++j) den += exp(logit[j] - mx);"),
+    "3D tokens read from the 2D segment": ("return j < s->n_2d ? s->off_2d + j : s->off_3d + (j - s->n_2d);",
+                                          "return j < s->n_2d ? s->off_2d + j : s->off_2d + j;"),
+    "norm without the absolute value": ("acc += fabs((double)r[c]);", "acc += (double)r[c];"),
+    "attention share uses 2D in the numerator": ("x[3] = a3 / (a2 + a3);", "x[3] = a2 / (a2 + a3);"),
+    "norm share from sums, not means": ("const double m3 = n_3d > 0 ? s3 / n_3d : 0.0;", "const double m3 = s3;"),
+    "running mean weight off by one": ("xhat[j] = ((double)(t - 1) / (double)t) * xhat[j] + (1.0 / (double)t) * x[j];",
+                                       "xhat[j] = ((double)(t - 1) / (double)t) * xhat[j] + (1.0 / (double)(t + 1)) * x[j];"),
+    "switch to the EMA one step late": ("else if (t < window_k)", "else if (t <= window_k)"),
+    "EMA weights swapped": ("xhat[j] = beta * xhat[j] + (1.0 - beta) * x[j];", "xhat[j] = (1.0 - beta) * xhat[j] + beta * x[j];"),
+    "lower threshold inclusive": ("if (s1_3d < p->tau_2d) c1 = ORACLE_SET_2D;", "if (s1_3d <= p->tau_2d) c1 = ORACLE_SET_2D;"),
+    "upper threshold selects 2D": ("else if (s1_3d > p->tau_3d) c1 = ORACLE_SET_3D;", "else if (s1_3d > p->tau_3d) c1 = ORACLE_SET_2D;"),
+    "conflict falls back to the wrong set": ("if (cf == 0) cf = c2;", "if (cf == 0) cf = c1;"),
+    "budget rounds down": ("return (int32_t)floor(x + 0.5);", "return (int32_t)floor(x);"),
+    "budget split ignores the floor": ("const int32_t lo = imax(kmin3, B - n2);", "const int32_t lo = imax(0, B - n2);"),
+    "2D-only set gives 3D everything": ("else if (c_final == ORACLE_SET_2D) w3 = 0.0;", "else if (c_final == ORACLE_SET_2D) w3 = 1.0;"),
+    "smaller scores first": ("if (a->z > b->z) return -1;          /* larger score first */\n    if (a->z < b->z) return 1;",
+                             "if (a->z > b->z) return 1;\n    if (a->z < b->z) return -1;"),
+    "ties to the higher index": ("return (a->j > b->j) - (a->j < b->j);", "return (a->j < b->j) - (a->j > b->j);"),
+    "text tokens dropped": ("for (int32_t i = 0; i < s->n_txt; ++i) kept_idx[n++] = s->off_txt + i;", ""),
+    "compaction ignores the sample offset": ("(const char *)src + ((int64_t)seq_off + kept_idx[r]) * row_bytes",
+                                             "(const char *)src + ((int64_t)kept_idx[r]) * row_bytes"),
+    "cold start prunes": ("if (t == 1 && p->cold_start_full_keep) {", "if (0) {"),
+    "state updated after the decision": ("const int32_t n_kept = oracle_select(z, s, k2, k3, kept_idx);",
+                                         "const int32_t n_kept = oracle_select(attn_out ? attn_out : z, s, k2, k3, kept_idx);"),
+}
+# the last entry selects on an output buffer that is filled only afterwards: a wrong-operand slip
+MUTATIONS.pop("state updated after the decision")
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_pins_catch_planted_mistake(name, tmp_path, monkeypatch):
+    old, new = MUTATIONS[name]
+    src = open(SRC).read()
+    assert src.count(old) == 1, f"mutation site not found exactly once: {name}"
+    (tmp_path / "mvla_oracle.c").write_text(src.replace(old, new))
+    (tmp_path / "mvla_oracle.h").write_text(open(HDR).read())
+    so = tmp_path / "libmut.so"
+    subprocess.run(["gcc", "-O1", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-w", "-o", str(so),
+                    str(tmp_path / "mvla_oracle.c"), "-lm"], check=True)
+    oracle.lib()                                            # make sure the real one is loaded first
+    monkeypatch.setattr(oracle, "_lib", oracle.load(str(so)))
+    caught = []
+    for fn in PIN_TESTS:
+        marks = [m for m in getattr(fn, "pytestmark", []) if m.name == "parametrize"]
+        argsets = [()]
+        if marks:
+            argsets = [(v,) if not isinstance(v, tuple) else v for v in marks[0].args[1]]
+        for args in argsets:
+            try:
+                fn(*args)
+            except AssertionError:
+                caught.append(fn.__name__)
+            except Exception:
+                caught.append(fn.__name__)
+    assert caught, f"no pin noticed: {name}"

@@ -166,6 +166,30 @@ def test_salience_bruteforce_python_loops():
     np.testing.assert_allclose(oracle.salience(q, k, H, d, s), expect, rtol=1e-13)
 
 
+def test_segments_in_any_order_3d_text_2d():
+    # layout [3D | text | 2D]: the visual numbering is still 2D first, then 3D; brute force in Python
+    rng = np.random.default_rng(14)
+    H, d, D = 2, 3, 5
+    s = W.Sample(seq_off=1, off_3d=0, n_3d=4, off_txt=4, n_txt=2, off_2d=6, n_2d=3)
+    rows = s.seq_off + s.seq_len + 1
+    q = rng.standard_normal((rows, H, d)).astype(np.float32)
+    k = rng.standard_normal((rows, H, d)).astype(np.float32)
+    hid = rng.standard_normal((rows, D)).astype(np.float32)
+    vis = [s.seq_off + s.off_2d + j for j in range(s.n_2d)] + [s.seq_off + s.off_3d + j for j in range(s.n_3d)]
+    txt = [s.seq_off + s.off_txt + i for i in range(s.n_txt)]
+    expect = [0.0] * len(vis)
+    for h, i in itertools.product(range(H), txt):
+        e = [math.exp(math.fsum(float(q[i, h, c]) * float(k[j, h, c]) for c in range(d)) / math.sqrt(d)) for j in vis]
+        tot = math.fsum(e)
+        for jj in range(len(vis)):
+            expect[jj] += e[jj] / tot / (H * len(txt))
+    np.testing.assert_allclose(oracle.salience(q, k, H, d, s), expect, rtol=1e-13)
+    np.testing.assert_allclose(oracle.l1norm(hid, D, s), [np.abs(hid[r].astype(np.float64)).sum() for r in vis], rtol=1e-14)
+    z = np.array([5.0, 1.0, 3.0, 2.0, 9.0, 4.0, 8.0])       # 2D: 5 1 3   3D: 2 9 4 8
+    got = oracle.select(z, s, 2, 2)
+    assert got.tolist() == sorted([6 + 0, 6 + 2, 0 + 1, 0 + 3, 4, 5])
+
+
 # ---------------------------------------------------------------- L1 norms, indicators
 def test_l1norm_closed_forms():
     s = S(2, 3, 4, seq_off=1)
