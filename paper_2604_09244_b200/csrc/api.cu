@@ -12,6 +12,8 @@
 
 using namespace mvla;
 
+namespace { constexpr int kSets = 4; }   // scratch sets = prune steps that may be in flight at once
+
 struct mvla_ctx {
     mvla_config cfg;
     int n_slots;
@@ -21,26 +23,26 @@ struct mvla_ctx {
     float* part;                 // [H][max_batch * max_vis] per-head partial scores
     int64_t part_stride;
     float* attn_ws;              // [max_batch * max_vis]
-    float* l1_ws;                // [2][max_batch * max_vis] feature norms, alternating between steps
+    float* l1_ws;                // [kSets][max_batch * max_vis] feature norms, one set per step in flight
     float* ahat_state;           // [n_prune_points][n_slots][max_vis]
     float* mhat_state;           // [n_prune_points][n_slots][4]
-    unsigned long long* acc64;   // [2][max_batch * max_vis] fixed-point score accumulators, zero between calls,
-                                 // alternating between steps (a step's scoring may run beside the previous
-                                 // step's selection)
+    unsigned long long* acc64;   // [kSets][max_batch * max_vis] fixed-point score accumulators, zero between
+                                 // calls; the sets rotate from step to step (a step's scoring may run beside
+                                 // the selections of the steps before it)
     size_t vis_all;              // max_batch * max_vis
-    unsigned step_parity;
+    unsigned step_parity;        // index of the scratch set of the current step
     // Scoring of a step whose inputs are promised stable runs on a side stream, forked from and joined
     // back into the caller's stream with events, so that it may run beside the previous step's
     // selection and row copy.
-    cudaStream_t aux[2];                       // one per scratch set, so that consecutive scorings do not serialise
-    cudaEvent_t ev_fork, ev_sal[2], ev_sel[2]; // ev_sel[p]: after the selection that last used scratch set p
-    bool sel_valid[2];
+    cudaStream_t aux[kSets];                   // one per scratch set, so that consecutive steps do not serialise
+    cudaEvent_t ev_fork, ev_sel[kSets];        // ev_sel[p]: after the selection that last used scratch set p
+    bool sel_valid[kSets];
     // Buffers the previous prune step wrote or read after its selection (outputs, kept indices): the next
     // step's selection may run beside that step's row copy only if it writes none of them.
     struct Range { const char* lo; const char* hi; };
     Range prev_out[10];
     int n_prev_out;
-    unsigned long long sel_capture[2];         // capture sequence the event belongs to (0: none)
+    unsigned long long sel_capture[kSets];         // capture sequence the event belongs to (0: none)
     std::vector<int32_t> t_host; // [n_prune_points][n_slots] steps absorbed so far
     int* status_host;            // mapped pinned word written by kernels whose bounded wait gave up
     int* status_dev;
@@ -340,11 +342,14 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (c.salience_path == MVLA_SALIENCE_FMA) ctx->use_umma = false;
     ctx->part = ctx->attn_ws = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
     ctx->acc64 = nullptr;
-    ctx->aux[0] = ctx->aux[1] = nullptr;
-    ctx->ev_fork = ctx->ev_sal[0] = ctx->ev_sal[1] = ctx->ev_sel[0] = ctx->ev_sel[1] = nullptr;
-    ctx->sel_valid[0] = ctx->sel_valid[1] = false;
+    ctx->ev_fork = nullptr;
+    for (int i = 0; i < kSets; ++i) {
+        ctx->aux[i] = nullptr;
+        ctx->ev_sel[i] = nullptr;
+        ctx->sel_valid[i] = false;
+        ctx->sel_capture[i] = 0;
+    }
     ctx->n_prev_out = -1;                            // unknown: no overlap
-    ctx->sel_capture[0] = ctx->sel_capture[1] = 0;
     ctx->status_host = ctx->status_dev = nullptr;
     ctx->last_cuda = cudaSuccess;
     ctx->tm_ptr[0] = ctx->tm_ptr[1] = nullptr;
@@ -362,16 +367,17 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     };
     alloc(&ctx->part, vis_all * c.n_heads);
     alloc(&ctx->attn_ws, vis_all);
-    alloc(&ctx->l1_ws, 2 * vis_all);
+    alloc(&ctx->l1_ws, kSets * vis_all);
     ctx->vis_all = vis_all;
     ctx->step_parity = 0;
     alloc(&ctx->ahat_state, n_state * ctx->max_vis);
     alloc(&ctx->mhat_state, n_state * 4);
-    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->acc64), 2 * vis_all * sizeof(unsigned long long));
-    if (e == cudaSuccess) e = cudaMemset(ctx->acc64, 0, 2 * vis_all * sizeof(unsigned long long));
-    for (cudaStream_t* sp : {&ctx->aux[0], &ctx->aux[1]})
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->acc64), kSets * vis_all * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(ctx->acc64, 0, kSets * vis_all * sizeof(unsigned long long));
+    for (cudaStream_t* sp = ctx->aux; sp != ctx->aux + kSets; ++sp)
         if (e == cudaSuccess) e = cudaStreamCreateWithFlags(sp, cudaStreamNonBlocking);
-    for (cudaEvent_t* ev : {&ctx->ev_fork, &ctx->ev_sal[0], &ctx->ev_sal[1], &ctx->ev_sel[0], &ctx->ev_sel[1]})
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
+    for (cudaEvent_t* ev = ctx->ev_sel; ev != ctx->ev_sel + kSets; ++ev)
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&ctx->status_host), sizeof(int), cudaHostAllocMapped);
     if (e == cudaSuccess) {
@@ -405,12 +411,13 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     cudaFree(ctx->ahat_state);
     cudaFree(ctx->mhat_state);
     cudaFree(ctx->acc64);
-    for (cudaStream_t sp : {ctx->aux[0], ctx->aux[1]})
+    for (cudaStream_t sp : ctx->aux)
         if (sp) {
             cudaStreamSynchronize(sp);
             cudaStreamDestroy(sp);
         }
-    for (cudaEvent_t ev : {ctx->ev_fork, ctx->ev_sal[0], ctx->ev_sal[1], ctx->ev_sel[0], ctx->ev_sel[1]})
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    for (cudaEvent_t ev : ctx->ev_sel)
         if (ev) cudaEventDestroy(ev);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     delete ctx;
@@ -547,12 +554,13 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
 
     // scratch set of this step
-    ctx->step_parity ^= 1u;
+    ctx->step_parity = (ctx->step_parity + 1u) % kSets;
     unsigned long long* acc64 = ctx->acc64 + ctx->step_parity * ctx->vis_all;
     float* l1_ws = ctx->l1_ws + ctx->step_parity * ctx->vis_all;
-    // With stable inputs (and the fast scoring kernel, whose scratch alternates between two sets) the
-    // scoring goes to the side stream.  It must not start before the selection that last used this
-    // scratch set (two steps ago) has finished; nothing else of the earlier work concerns it.
+    // With stable inputs (and the fast scoring kernel, whose scratch rotates over kSets sets) scoring
+    // and selection go to the side stream of this step's scratch set; only the row copy stays on the
+    // caller's stream.  Scoring must not start before the selection that last used the set (kSets steps
+    // ago, on the same side stream) has finished; nothing else of the earlier work concerns it.
     bool forked = false;
     unsigned long long cap_id = 0;
     const unsigned par = ctx->step_parity;
@@ -560,12 +568,14 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         cudaStreamCaptureStatus cst = cudaStreamCaptureStatusNone;
         if (cudaStreamGetCaptureInfo(st, &cst, &cap_id) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
         if (cst != cudaStreamCaptureStatusActive) cap_id = 0;
-        cudaEvent_t dep = ctx->ev_sel[par];
+        // The side stream of this scratch set last ran the selection of kSets steps ago, so its own order
+        // already protects the set.  Without such history (first steps, another capture) it starts
+        // after everything enqueued so far.
         if (!(ctx->sel_valid[par] && ctx->sel_capture[par] == cap_id)) {
-            dep = ctx->ev_fork;                      // no usable history: after everything enqueued so far
-            if (cudaEventRecord(dep, st) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
+            if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess ||
+                cudaStreamWaitEvent(ctx->aux[par], ctx->ev_fork, 0) != cudaSuccess)
+                return fail_cuda(ctx, cudaGetLastError());
         }
-        if (cudaStreamWaitEvent(ctx->aux[par], dep, 0) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
         forked = true;
     }
     // May this step's selection run beside the previous step's row copy?  Only if that copy is known
@@ -595,12 +605,24 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         const BatchDesc bd = chunk_of(plan, first, n);
         bool used_acc64 = false;
         rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, l1_ws, acc64,
-                                &used_acc64, forked, forked ? ctx->aux[par] : st);
+                                &used_acc64, false, forked ? ctx->aux[par] : st);
         if (rc != MVLA_OK) return rc;
-        if (forked) {                                // join: the selection needs the scores
-            if (cudaEventRecord(ctx->ev_sal[par], ctx->aux[par]) != cudaSuccess ||
-                cudaStreamWaitEvent(st, ctx->ev_sal[par], 0) != cudaSuccess)
-                return fail_cuda(ctx, cudaGetLastError());
+        cudaStream_t sel_stream = st;
+        if (forked) {
+            // The selection follows its scoring on the side stream.  It must also follow the previous
+            // selection (the smoothed state is updated in call order): an event if that one ran on the
+            // other side stream, else everything enqueued on the caller's stream so far.  The same
+            // conservative order is taken when an output of this selection coincides with a buffer
+            // that the previous step's row copy may still be using, or when that step is unknown.
+            sel_stream = ctx->aux[par];
+            const unsigned prv = (par + kSets - 1u) % kSets;     // the set of the previous step
+            const bool chained = ctx->sel_valid[prv] && ctx->sel_capture[prv] == cap_id;
+            cudaEvent_t dep = ctx->ev_sel[prv];
+            if (!chained || !sel_beside) {
+                dep = ctx->ev_fork;
+                if (cudaEventRecord(dep, st) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
+            }
+            if (cudaStreamWaitEvent(sel_stream, dep, 0) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
         }
         SelectIO io;
         std::memset(&io, 0, sizeof io);
@@ -613,11 +635,13 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         io.attn_out = out->attn; io.ahat_out = out->ahat; io.z_out = out->z; io.diag = out->diag;
         io.chunk_first = first; io.total_out = plan.total_out; io.write_total = first + n == batch;
         io.n_in_launch = n;
-        io.beside_previous = forked && sel_beside;
-        cudaError_t e = launch_select(bd, gp, io, st);
+        io.beside_previous = 0;
+        cudaError_t e = launch_select(bd, gp, io, sel_stream);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
-        if (forked) {
-            if (cudaEventRecord(ctx->ev_sel[par], st) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
+        if (forked) {                                // join: the row copy, and whatever the caller enqueues next
+            if (cudaEventRecord(ctx->ev_sel[par], sel_stream) != cudaSuccess ||
+                cudaStreamWaitEvent(st, ctx->ev_sel[par], 0) != cudaSuccess)
+                return fail_cuda(ctx, cudaGetLastError());
             ctx->sel_valid[par] = true;
             ctx->sel_capture[par] = cap_id;
         } else {

@@ -8,10 +8,12 @@
 //   2. modality sums -> the four indicators, smoothed too; dual threshold (Sec. 4.1), target-object
 //      rule (Sec. 4.2), fusion (Sec. 4.4), budget split.  One thread does this while the others
 //      already build the first radix histogram;
-//   3. radix select of the k-th largest key of each modality: 4 passes of 8 bits, both modalities at
-//      once, one warp-aggregated shared-memory histogram per pass (all cleared up front);
-//   4. emission in sequence order merged with all text positions: elements above the threshold plus
-//      the first (lowest-index) elements equal to it, with two block-wide prefix scans.
+//   3. radix select of the k-th largest key of each modality: up to 4 passes of 8 bits, both
+//      modalities at once, one warp-aggregated shared-memory histogram per pass (all cleared up
+//      front); a modality is settled early when a digit bin must be taken whole;
+//   4. emission merged with all text positions: elements above the threshold plus the first
+//      (lowest-index) elements equal to it; one block-wide prefix scan per NT elements ranks the kept
+//      ones (one more only when equal keys straddle a budget).
 #pragma once
 
 #include "common.cuh"
