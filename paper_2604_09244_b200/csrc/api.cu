@@ -635,7 +635,6 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         io.attn_out = out->attn; io.ahat_out = out->ahat; io.z_out = out->z; io.diag = out->diag;
         io.chunk_first = first; io.total_out = plan.total_out; io.write_total = first + n == batch;
         io.n_in_launch = n;
-        io.beside_previous = 0;
         cudaError_t e = launch_select(bd, gp, io, sel_stream);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
         if (forked) {                                // join: the row copy, and whatever the caller enqueues next

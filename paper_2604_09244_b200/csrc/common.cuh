@@ -66,7 +66,6 @@ struct SelectIO {
     int32_t total_out;
     int32_t write_total;     // this launch holds the batch's last sample
     int32_t n_in_launch;
-    int32_t beside_previous;  // 1: may run beside the kernel before it in the stream; waits for it only before completing
 };
 
 // Launch attribute that lets a kernel begin before its stream predecessor has drained (the kernel

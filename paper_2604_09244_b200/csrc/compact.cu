@@ -47,8 +47,7 @@ compact_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ Com
     const int orow = chunk_row0 + r;
 
     asm volatile("griddepcontrol.wait;" ::: "memory");      // kept_idx comes from the kernel before this one
-    // Only now may the next kernel start: a selection of the next step that runs beside this copy can
-    // rely on this step's selection (which owns the smoothed state) being complete.
+    // Only now may the next kernel become resident: by then this step's selection is complete.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // which sample owns output row `orow` (samples are few: linear scan)
     int b = 0;

@@ -29,7 +29,8 @@ template <int NT>
 struct SelectSmem {
     uint32_t key[kMaxVis];
     int hist[4][2][256];          // one histogram per radix pass and modality
-    float red[NT / 32][4];
+    float red[NT / 32][4];        // per-warp partial sums of the instantaneous scores and norms
+    float red2[NT / 32][4];       // scratch of the optional normalisation
     float tot[4];
     int scan[NT / 32 + 1];
     uint32_t prefix[2];
@@ -127,11 +128,13 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
     // prologue that needs nothing from the previous kernel
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     for (int i = tid; i < 4 * 2 * 256; i += NT) (&sm.hist[0][0][0])[i] = 0;
-    if (tid < 2) { sm.prefix[tid] = 0u; sm.alltie[tid] = 1; sm.done[tid] = 0; sm.cmask[tid] = 0xFFFFFFFFu; }
-    // Scores normally come from the kernel before this one.  When the host has established that they
-    // do not (they arrive through an event dependency) and that no buffer written here is touched by
-    // that kernel, the wait moves to the end: completion still implies completion of all earlier work.
-    if (!io.beside_previous) asm volatile("griddepcontrol.wait;" ::: "memory");
+    const bool k_fixed = s.k_2d_fixed >= 0;               // budgets decided on the host (FIXED mode, cold start)
+    if (tid < 2) {
+        sm.prefix[tid] = 0u; sm.alltie[tid] = 1; sm.done[tid] = 0; sm.cmask[tid] = 0xFFFFFFFFu;
+        if (k_fixed) sm.k[tid] = sm.krem[tid] = tid == 0 ? s.k_2d_fixed : s.budget - s.k_2d_fixed;
+    }
+    __syncthreads();                                        // histograms are clear before anyone adds to them
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // scores come from the kernel before this one
 
     // ---- 1. all loads first
     float a[EPT], prev[EPT], nrm[EPT];
@@ -186,13 +189,20 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
             else        { sums[1] += a[e]; sums[3] += nrm[e]; ssm[1] += smo; }
         }
     }
-    block_sum4<NT>(sums, sm.red, sm.tot);     // also orders the histogram clearing before the atomics below
-    const float t0 = sm.tot[0], t1 = sm.tot[1], t2 = sm.tot[2], t3 = sm.tot[3];
+    // Per-warp partial sums (fixed shuffle tree).  The sum over warps is taken later by the one warp that
+    // needs it, so that with host-decided budgets nothing below waits for the indicator arithmetic.
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) sums[c] += __shfl_xor_sync(0xffffffffu, sums[c], off);
+    if (lane == 0)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) sm.red[warp][c] = sums[c];
 
     // optional: the smoothed scores normalised to mean one inside each modality.  The ranking below
     // uses the smoothed scores themselves; a positive per-modality factor cannot change it.
     if (io.z_out) {
-        block_sum4<NT>(ssm, sm.red, sm.tot);
+        block_sum4<NT>(ssm, sm.red2, sm.tot);
         const float f2 = static_cast<float>(n2) / sm.tot[0], f3 = static_cast<float>(n3) / sm.tot[1];
 #pragma unroll
         for (int e = 0; e < EPT; ++e) {
@@ -226,10 +236,25 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
             }
         }
     };
-    histogram(0, 24, 0u, 0u, false, false);   // needs no budget yet: overlaps with the gate arithmetic
+    histogram(0, 24, 0u, 0u, false, false);   // needs no budget yet
+    __syncthreads();                          // first histogram and the per-warp sums are complete
 
-    // ---- 2. indicators, gates, budget (one thread of the last warp, which rarely owns elements; a few dozen flops)
-    if (tid == NT - 32) {
+    // ---- 2. indicators, gates, budget: the last warp (which rarely owns elements) adds the per-warp sums
+    //         with the same fixed tree, its first lane does the few dozen flops.  With host-decided budgets
+    //         the other warps go straight on to the digit search and meet this warp at the next barrier.
+    if (warp == NT / 32 - 1) {
+        float t0, t1, t2, t3;
+        {
+            float y[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                y[c] = lane < NT / 32 ? sm.red[lane][c] : 0.f;
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) y[c] += __shfl_xor_sync(0xffffffffu, y[c], off);
+            }
+            t0 = y[0]; t1 = y[1]; t2 = y[2]; t3 = y[3];
+        }
+      if (lane == 0) {
         float x[4];
         x[3] = __fdividef(t1, t0 + t1);                                   // attention share of 3D (Eq. P2D / P3D)
         x[2] = 1.f - x[3];
@@ -263,8 +288,10 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
             k3 = min(max(k3, lo), hi);
             k2 = s.budget - k3;
         }
-        sm.k[0] = k2; sm.k[1] = k3;
-        sm.krem[0] = k2; sm.krem[1] = k3;
+        if (!k_fixed) {
+            sm.k[0] = k2; sm.k[1] = k3;
+            sm.krem[0] = k2; sm.krem[1] = k3;
+        }
         if (io.budgets) {
             io.budgets[b_glob * 2 + 0] = k2;
             io.budgets[b_glob * 2 + 1] = k3;
@@ -279,8 +306,9 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
         }
         io.out_offsets[b_glob] = s.out_off;
         if (io.write_total && b_local == io.n_in_launch - 1) io.out_offsets[b_glob + 1] = io.total_out;
+      }
     }
-    __syncthreads();
+    if (!k_fixed) __syncthreads();            // the digit search needs the budgets (block-uniform branch)
 
     // ---- 3. radix select, 8 bits per pass, most significant first.  A modality is settled as soon as
     //         the digit bin that holds its k-th largest element must be taken whole (then the bits seen
@@ -377,7 +405,6 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
             else        io.kept_idx[s.out_off + base3 + (r - k2)] = s.off_3d + (j - n2);
         }
     }
-    if (io.beside_previous) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 }  // namespace mvla
