@@ -23,7 +23,7 @@
 namespace mvla {
 
 constexpr float kFixScale = 1152921504606846976.f;          // 2^60
-constexpr double kFixInv = 1.0 / 1152921504606846976.0;
+constexpr float kFixInv = 1.f / 1152921504606846976.f;      // 2^-60, exact
 
 template <int NT>
 struct SelectSmem {
@@ -176,7 +176,7 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
         const int j = tid + e * NT;
         if (j < nv) {
             if (io.acc64) {
-                a[e] = static_cast<float>(__ull2double_rn(fx[e]) * kFixInv);
+                a[e] = __ull2float_rn(fx[e]) * kFixInv;   // one rounding: the exact head sum to fp32
                 io.acc64[s.vis_off + j] = 0ull;            // ready for the next call
             }
             const float smo = carry ? fmaf(s.c_prev, prev[e], s.c_new * a[e]) : a[e];
