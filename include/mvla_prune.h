@@ -58,15 +58,17 @@ extern "C" {
 
 #define MVLA_FLAG_RESET_STATE     1u  /* restart the episode: this call is action step t = 1 */
 #define MVLA_FLAG_NO_STATE_UPDATE 2u  /* dry run: decide as usual but leave the smoothed state and t untouched */
-#define MVLA_FLAG_INPUTS_STABLE   4u  /* mvla_prune_step only.  The caller promises that the work enqueued on the stream just
-                                         before this call neither writes q, k, hidden nor touches this call's output
-                                         buffers (the library checks the latter itself against its own previous prune
-                                         step and falls back to waiting where they coincide).  Scoring then runs on a
-                                         side stream owned by the context, forked from and joined into `stream` with
-                                         events, beside the previous step's selection and row copy, and the selection
-                                         may run beside the previous row copy.  Every result of the call is still
-                                         complete, in stream order, only after all earlier work; the smoothed state is
-                                         updated in call order.  Without the flag every kernel waits for all earlier work. */
+#define MVLA_FLAG_INPUTS_STABLE   4u  /* mvla_prune_step only.  The caller promises that none of ITS OWN work enqueued on
+                                         `stream` before this call and possibly still running writes q, k, hidden or
+                                         touches this call's output buffers.  (Earlier prune steps of this context
+                                         need no promise: where one of them writes a buffer that this call reads or
+                                         writes, the library orders this call after everything enqueued so far.)
+                                         Scoring and selection then run on one of a small ring of streams owned by the
+                                         context, beside the selection and row copy of the steps before; the row copy
+                                         stays on `stream` and waits for the step's selection.  Every result of the
+                                         call is complete in the order of `stream`, as without the flag, and the
+                                         smoothed state is updated in call order.  Without the flag every kernel waits
+                                         for all earlier work of `stream`. */
 
 #define MVLA_SET_2D 1   /* candidate sets are bit sets */
 #define MVLA_SET_3D 2

@@ -12,7 +12,7 @@
 
 using namespace mvla;
 
-namespace { constexpr int kSets = 4; }   // scratch sets = prune steps that may be in flight at once
+namespace { constexpr int kSets = 6; }   // scratch sets = prune steps that may be in flight at once
 
 struct mvla_ctx {
     mvla_config cfg;
@@ -31,17 +31,20 @@ struct mvla_ctx {
                                  // the selections of the steps before it)
     size_t vis_all;              // max_batch * max_vis
     unsigned step_parity;        // index of the scratch set of the current step
-    // Scoring of a step whose inputs are promised stable runs on a side stream, forked from and joined
-    // back into the caller's stream with events, so that it may run beside the previous step's
-    // selection and row copy.
+    // Scoring and selection of a step whose inputs are promised stable run on the side stream of the
+    // step's scratch set, beside the selection and row copy of the steps before; the row copy stays
+    // on the caller's stream and waits for ev_sel of the step.
     cudaStream_t aux[kSets];                   // one per scratch set, so that consecutive steps do not serialise
     cudaEvent_t ev_fork, ev_sel[kSets];        // ev_sel[p]: after the selection that last used scratch set p
+    cudaEvent_t ev_copy[kSets];                // ev_copy[p]: after the row copy of that same step
     bool sel_valid[kSets];
-    // Buffers the previous prune step wrote or read after its selection (outputs, kept indices): the next
-    // step's selection may run beside that step's row copy only if it writes none of them.
+    // Buffers that the side-stream steps still possibly in flight write (selection outputs, copied rows),
+    // one entry per scratch set.  A step whose side-stream work reads or writes any of them (its inputs,
+    // its selection outputs) is ordered after everything enqueued on the caller's stream instead.
     struct Range { const char* lo; const char* hi; };
-    Range prev_out[10];
-    int n_prev_out;
+    Range hist[kSets][10];
+    int n_hist[kSets];
+    bool hist_unknown;                         // the stream ran other work of this context since: order after it
     unsigned long long sel_capture[kSets];         // capture sequence the event belongs to (0: none)
     std::vector<int32_t> t_host; // [n_prune_points][n_slots] steps absorbed so far
     int* status_host;            // mapped pinned word written by kernels whose bounded wait gave up
@@ -345,11 +348,12 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     ctx->ev_fork = nullptr;
     for (int i = 0; i < kSets; ++i) {
         ctx->aux[i] = nullptr;
-        ctx->ev_sel[i] = nullptr;
+        ctx->ev_sel[i] = ctx->ev_copy[i] = nullptr;
+        ctx->n_hist[i] = 0;
         ctx->sel_valid[i] = false;
         ctx->sel_capture[i] = 0;
     }
-    ctx->n_prev_out = -1;                            // unknown: no overlap
+    ctx->hist_unknown = true;
     ctx->status_host = ctx->status_dev = nullptr;
     ctx->last_cuda = cudaSuccess;
     ctx->tm_ptr[0] = ctx->tm_ptr[1] = nullptr;
@@ -378,6 +382,8 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
         if (e == cudaSuccess) e = cudaStreamCreateWithFlags(sp, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
     for (cudaEvent_t* ev = ctx->ev_sel; ev != ctx->ev_sel + kSets; ++ev)
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
+    for (cudaEvent_t* ev = ctx->ev_copy; ev != ctx->ev_copy + kSets; ++ev)
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&ctx->status_host), sizeof(int), cudaHostAllocMapped);
     if (e == cudaSuccess) {
@@ -419,6 +425,8 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     for (cudaEvent_t ev : ctx->ev_sel)
         if (ev) cudaEventDestroy(ev);
+    for (cudaEvent_t ev : ctx->ev_copy)
+        if (ev) cudaEventDestroy(ev);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     delete ctx;
 }
@@ -434,7 +442,7 @@ int32_t mvla_salience(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, 
     if (rc != MVLA_OK) return rc;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return MVLA_ERR_CUDA;
-    ctx->n_prev_out = -1;                            // what the stream ran last is no longer a known prune step
+    ctx->hist_unknown = true;                        // what the stream ran last is no longer a known prune step
     Plan plan;
     rc = make_plan(ctx, 0, batch, samples, MVLA_MODE_FIXED, 0, false, &plan);
     if (rc != MVLA_OK) return rc;
@@ -463,7 +471,7 @@ int32_t mvla_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvl
     if (mode == MVLA_MODE_ADAPTIVE && !l1) return MVLA_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return MVLA_ERR_CUDA;
-    ctx->n_prev_out = -1;                            // what the stream ran last is no longer a known prune step
+    ctx->hist_unknown = true;                        // what the stream ran last is no longer a known prune step
     Plan plan;
     rc = make_plan(ctx, prune_point, batch, samples, mode, flags, true, &plan);
     if (rc != MVLA_OK) return rc;
@@ -504,7 +512,7 @@ int32_t mvla_compact(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, c
     if (rc != MVLA_OK) return rc;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return MVLA_ERR_CUDA;
-    ctx->n_prev_out = -1;                            // what the stream ran last is no longer a known prune step
+    ctx->hist_unknown = true;                        // what the stream ran last is no longer a known prune step
     Plan plan;
     rc = make_plan(ctx, 0, batch, samples, MVLA_MODE_FIXED, 0, false, &plan);
     if (rc != MVLA_OK) return rc;
@@ -559,46 +567,63 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     float* l1_ws = ctx->l1_ws + ctx->step_parity * ctx->vis_all;
     // With stable inputs (and the fast scoring kernel, whose scratch rotates over kSets sets) scoring
     // and selection go to the side stream of this step's scratch set; only the row copy stays on the
-    // caller's stream.  Scoring must not start before the selection that last used the set (kSets steps
-    // ago, on the same side stream) has finished; nothing else of the earlier work concerns it.
-    bool forked = false;
+    // caller's stream.  What the side-stream work of step k must follow:
+    //   * selection and row copy of step k - kSets (same scratch set; the copy also frees that step's
+    //     output buffers, so at most kSets - 1 earlier copies can still be running);
+    //   * selection of step k - 1 (the smoothed state is updated in call order);
+    //   * if it reads or writes a buffer that one of those kSets - 1 steps writes, or if the stream has
+    //     run other work of this context since: everything enqueued on the caller's stream so far.
+    // Events recorded under another stream capture cannot be waited on; then, too, the step starts
+    // after everything enqueued so far.
+    bool forked = false, ordered_after_all = false;
     unsigned long long cap_id = 0;
     const unsigned par = ctx->step_parity;
+    const unsigned prv = (par + kSets - 1u) % kSets;     // the set of the previous step
+    const size_t nvis_b = static_cast<size_t>(plan.total_vis), nout_b = static_cast<size_t>(plan.total_out);
+    const size_t hb = static_cast<size_t>(ctx->cfg.d_model) * ctx->elem, kb = static_cast<size_t>(kv_bytes);
     if ((flags & MVLA_FLAG_INPUTS_STABLE) && batch <= kMaxChunk && chunk_is_fast(ctx, chunk_of(plan, 0, batch))) {
         cudaStreamCaptureStatus cst = cudaStreamCaptureStatusNone;
         if (cudaStreamGetCaptureInfo(st, &cst, &cap_id) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
         if (cst != cudaStreamCaptureStatusActive) cap_id = 0;
-        // The side stream of this scratch set last ran the selection of kSets steps ago, so its own order
-        // already protects the set.  Without such history (first steps, another capture) it starts
-        // after everything enqueued so far.
-        if (!(ctx->sel_valid[par] && ctx->sel_capture[par] == cap_id)) {
-            if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess ||
-                cudaStreamWaitEvent(ctx->aux[par], ctx->ev_fork, 0) != cudaSuccess)
-                return fail_cuda(ctx, cudaGetLastError());
-        }
         forked = true;
-    }
-    // May this step's selection run beside the previous step's row copy?  Only if that copy is known
-    // (the previous call on this context was a forked prune step) and touches nothing written here.
-    const size_t nvis_b = static_cast<size_t>(plan.total_vis), nout_b = static_cast<size_t>(plan.total_out);
-    const mvla_ctx::Range sel_w[7] = {
-        range_of(out->kept_idx, nout_b * 4), range_of(out->out_offsets, (batch + 1) * 4u),
-        range_of(out->budgets, batch * 8u), range_of(out->attn, nvis_b * 4), range_of(out->ahat, nvis_b * 4),
-        range_of(out->z, nvis_b * 4), range_of(out->diag, batch * sizeof(mvla_diag))};
-    bool sel_beside = forked && ctx->n_prev_out >= 0;
-    for (int i = 0; sel_beside && i < 7; ++i)
-        for (int j = 0; sel_beside && j < ctx->n_prev_out; ++j)
-            if (sel_w[i].lo && sel_w[i].lo < ctx->prev_out[j].hi && ctx->prev_out[j].lo < sel_w[i].hi) sel_beside = false;
-    if (forked) {                                    // remember what this step's copy touches
-        const size_t hb = static_cast<size_t>(ctx->cfg.d_model) * ctx->elem, kb = static_cast<size_t>(kv_bytes);
+        // buffers the side-stream work touches: selection outputs, and the inputs of scoring
+        const size_t in_rows = static_cast<size_t>(in->rows);
+        const mvla_ctx::Range side[10] = {
+            range_of(out->kept_idx, nout_b * 4), range_of(out->out_offsets, (batch + 1) * 4u),
+            range_of(out->budgets, batch * 8u), range_of(out->attn, nvis_b * 4), range_of(out->ahat, nvis_b * 4),
+            range_of(out->z, nvis_b * 4), range_of(out->diag, batch * sizeof(mvla_diag)),
+            range_of(in->q, in_rows * kb), range_of(in->k, in_rows * kb),
+            range_of(adaptive ? in->hidden : nullptr, in_rows * hb)};
+        bool clash = ctx->hist_unknown;
+        for (unsigned s = 0; !clash && s < kSets; ++s) {
+            if (s == par) continue;
+            for (int i = 0; !clash && i < 10; ++i)
+                for (int j = 0; !clash && j < ctx->n_hist[s]; ++j)
+                    clash = side[i].lo && side[i].lo < ctx->hist[s][j].hi && ctx->hist[s][j].lo < side[i].hi;
+        }
+        const bool own_ok = ctx->sel_valid[par] && ctx->sel_capture[par] == cap_id;
+        const bool chained = ctx->sel_valid[prv] && ctx->sel_capture[prv] == cap_id;
+        ordered_after_all = clash || !own_ok || !chained;
+        cudaError_t e;
+        if (ordered_after_all) {
+            e = cudaEventRecord(ctx->ev_fork, st);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->aux[par], ctx->ev_fork, 0);
+            if (ctx->hist_unknown)
+                for (int& n : ctx->n_hist) n = 0;
+        } else {
+            e = cudaStreamWaitEvent(ctx->aux[par], ctx->ev_copy[par], 0);
+        }
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        // remember what this step writes
         int m = 0;
-        for (int i = 0; i < 7; ++i) if (sel_w[i].lo) ctx->prev_out[m++] = sel_w[i];
-        if (out->out_hidden) ctx->prev_out[m++] = range_of(out->out_hidden, nout_b * hb);
-        if (out->out_k) ctx->prev_out[m++] = range_of(out->out_k, nout_b * kb);
-        if (out->out_v) ctx->prev_out[m++] = range_of(out->out_v, nout_b * kb);
-        ctx->n_prev_out = m;
+        for (int i = 0; i < 7; ++i) if (side[i].lo) ctx->hist[par][m++] = side[i];
+        if (out->out_hidden) ctx->hist[par][m++] = range_of(out->out_hidden, nout_b * hb);
+        if (out->out_k) ctx->hist[par][m++] = range_of(out->out_k, nout_b * kb);
+        if (out->out_v) ctx->hist[par][m++] = range_of(out->out_v, nout_b * kb);
+        ctx->n_hist[par] = m;
+        ctx->hist_unknown = false;
     } else {
-        ctx->n_prev_out = -1;
+        ctx->hist_unknown = true;
     }
     for (int first = 0; first < batch; first += kMaxChunk) {
         const int n = std::min(kMaxChunk, batch - first);
@@ -609,20 +634,9 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         if (rc != MVLA_OK) return rc;
         cudaStream_t sel_stream = st;
         if (forked) {
-            // The selection follows its scoring on the side stream.  It must also follow the previous
-            // selection (the smoothed state is updated in call order): an event if that one ran on the
-            // other side stream, else everything enqueued on the caller's stream so far.  The same
-            // conservative order is taken when an output of this selection coincides with a buffer
-            // that the previous step's row copy may still be using, or when that step is unknown.
             sel_stream = ctx->aux[par];
-            const unsigned prv = (par + kSets - 1u) % kSets;     // the set of the previous step
-            const bool chained = ctx->sel_valid[prv] && ctx->sel_capture[prv] == cap_id;
-            cudaEvent_t dep = ctx->ev_sel[prv];
-            if (!chained || !sel_beside) {
-                dep = ctx->ev_fork;
-                if (cudaEventRecord(dep, st) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
-            }
-            if (cudaStreamWaitEvent(sel_stream, dep, 0) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
+            if (!ordered_after_all && cudaStreamWaitEvent(sel_stream, ctx->ev_sel[prv], 0) != cudaSuccess)
+                return fail_cuda(ctx, cudaGetLastError());
         }
         SelectIO io;
         std::memset(&io, 0, sizeof io);
@@ -650,6 +664,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         const int32_t nrows = bd.s[n - 1].out_off + bd.s[n - 1].n_out - row0;
         e = launch_compact(bd, job, out->kept_idx, nrows, row0, nullptr, first, batch, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
+        if (forked && cudaEventRecord(ctx->ev_copy[par], st) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
     }
     commit_steps(ctx, prune_point, plan, samples);
     if (total_kept_out) *total_kept_out = plan.total_out;

@@ -339,10 +339,44 @@ def test_pipelined_steps_with_state_match_serial_steps():
         return snap
 
     ref = run(0, 10, True)
-    for n_out in (10, 3, 1):                                  # 1: every step reuses the same output buffers
+    for n_out in (10, 3, 2, 1):                                # 1: every step reuses the same output buffers
         got = run(mvla.FLAG_INPUTS_STABLE, n_out, False)
         for t in range(10 - n_out, 10):
             assert all(torch.equal(x, y) for x, y in zip(got[t], ref[t])), (n_out, t)
+
+
+def test_pipelined_steps_sharing_an_index_buffer_two_steps_apart():
+    # Every step has its own row buffers, but steps t and t + 2 share kept_idx, and the caller's stream is
+    # kept busy between the steps so that the row copies lag behind the selections running ahead on the
+    # library's own streams.  A selection must not overwrite indices that an earlier copy has yet to read.
+    import dataclasses
+    wl = W.small_workload(47, batch=2, D=256, H=4, d=128, dtype="bf16", n_txt=(7, 21), n_2d=(90, 200),
+                          n_3d=(160, 310), keep=(0.45, 0.35), steps=12, cold_start=0)
+    devs = [device_tensors(wl, t) for t in range(12)]
+
+    def run(flag, share, delay):
+        ctx = mvla.context_for(wl)
+        outs = [ctx.alloc_outputs(wl.samples, extras=True) for _ in range(12)]
+        if share:
+            outs = [dataclasses.replace(o, kept_idx=outs[t % 2].kept_idx) for t, o in enumerate(outs)]
+        kept = []
+        for t, d in enumerate(devs):
+            if delay:
+                torch.cuda._sleep(300000)                     # touches none of the step's buffers
+            o = ctx.prune_step(0, wl.samples, wl.mode, d["q"], d["k"], d["v"], d["hidden"],
+                               flags=flag | (mvla.FLAG_RESET_STATE if t == 0 else 0), out=outs[t])
+            kept.append(o.total_kept)
+            if not flag:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        res = [(o.out_hidden[:n].clone(), o.out_k[:n].clone(), o.budgets.clone()) for o, n in zip(outs, kept)]
+        ctx.close()
+        return res
+
+    ref = run(0, False, False)
+    got = run(mvla.FLAG_INPUTS_STABLE, True, True)
+    for t in range(12):
+        assert all(torch.equal(x, y) for x, y in zip(got[t], ref[t])), t
 
 
 def test_step_segments_in_order_3d_text_2d():
