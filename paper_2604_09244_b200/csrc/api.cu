@@ -45,6 +45,10 @@ struct mvla_ctx {
     Range hist[kSets][10];
     int n_hist[kSets];
     bool hist_unknown;                         // the stream ran other work of this context since: order after it
+    // Smoothed states (prune point x slot) that the step last run on each scratch set reads and writes:
+    // a later selection touching one of them waits for that selection, others need not.
+    int32_t state_of[kSets][kMaxChunk];
+    int n_state_of[kSets];
     unsigned long long sel_capture[kSets];         // capture sequence the event belongs to (0: none)
     std::vector<int32_t> t_host; // [n_prune_points][n_slots] steps absorbed so far
     int* status_host;            // mapped pinned word written by kernels whose bounded wait gave up
@@ -350,6 +354,7 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
         ctx->aux[i] = nullptr;
         ctx->ev_sel[i] = ctx->ev_copy[i] = nullptr;
         ctx->n_hist[i] = 0;
+        ctx->n_state_of[i] = 0;
         ctx->sel_valid[i] = false;
         ctx->sel_capture[i] = 0;
     }
@@ -570,15 +575,17 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     // caller's stream.  What the side-stream work of step k must follow:
     //   * selection and row copy of step k - kSets (same scratch set; the copy also frees that step's
     //     output buffers, so at most kSets - 1 earlier copies can still be running);
-    //   * selection of step k - 1 (the smoothed state is updated in call order);
+    //   * every selection of the kSets - 1 steps before that touches a smoothed state (prune point,
+    //     slot) this step touches: a state is updated in call order.  Steps on other slots -- independent
+    //     requests -- are not waited for;
     //   * if it reads or writes a buffer that one of those kSets - 1 steps writes, or if the stream has
     //     run other work of this context since: everything enqueued on the caller's stream so far.
     // Events recorded under another stream capture cannot be waited on; then, too, the step starts
     // after everything enqueued so far.
     bool forked = false, ordered_after_all = false;
+    unsigned dep_mask = 0;
     unsigned long long cap_id = 0;
     const unsigned par = ctx->step_parity;
-    const unsigned prv = (par + kSets - 1u) % kSets;     // the set of the previous step
     const size_t nvis_b = static_cast<size_t>(plan.total_vis), nout_b = static_cast<size_t>(plan.total_out);
     const size_t hb = static_cast<size_t>(ctx->cfg.d_model) * ctx->elem, kb = static_cast<size_t>(kv_bytes);
     if ((flags & MVLA_FLAG_INPUTS_STABLE) && batch <= kMaxChunk && chunk_is_fast(ctx, chunk_of(plan, 0, batch))) {
@@ -601,15 +608,35 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
                 for (int j = 0; !clash && j < ctx->n_hist[s]; ++j)
                     clash = side[i].lo && side[i].lo < ctx->hist[s][j].hi && ctx->hist[s][j].lo < side[i].hi;
         }
+        // earlier selections still possibly in flight that touch a smoothed state this step touches: the
+        // state is updated in call order, so this step's selection waits for the most recent one per
+        // state (dep_mask; that one has in turn waited for those before it).  Steps older than
+        // kSets - 1 calls are ordered through the row-copy event or the stream itself.
         const bool own_ok = ctx->sel_valid[par] && ctx->sel_capture[par] == cap_id;
-        const bool chained = ctx->sel_valid[prv] && ctx->sel_capture[prv] == cap_id;
-        ordered_after_all = clash || !own_ok || !chained;
+        bool stale = false;
+        bool covered[kMaxChunk] = {};            // per sample of this step: most recent toucher of its state found
+        for (unsigned back = 1; back < kSets; ++back) {          // most recent step first
+            const unsigned s = (par + kSets - back) % kSets;
+            bool hit = false;
+            for (int b = 0; b < batch; ++b) {
+                if (covered[b]) continue;        // an even later step touches it and has waited for this one
+                const int32_t mine = prune_point * ctx->n_slots + samples[b].state_slot;
+                for (int i = 0; i < ctx->n_state_of[s]; ++i)
+                    if (ctx->state_of[s][i] == mine) { covered[b] = hit = true; break; }
+            }
+            if (!hit) continue;
+            if (ctx->sel_valid[s] && ctx->sel_capture[s] == cap_id) dep_mask |= 1u << s;
+            else stale = true;                   // its event cannot be waited on from here
+        }
+        ordered_after_all = clash || !own_ok || stale;
         cudaError_t e;
         if (ordered_after_all) {
             e = cudaEventRecord(ctx->ev_fork, st);
             if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->aux[par], ctx->ev_fork, 0);
-            if (ctx->hist_unknown)
+            if (ctx->hist_unknown) {
                 for (int& n : ctx->n_hist) n = 0;
+                for (int& n : ctx->n_state_of) n = 0;
+            }
         } else {
             e = cudaStreamWaitEvent(ctx->aux[par], ctx->ev_copy[par], 0);
         }
@@ -622,6 +649,8 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         if (out->out_v) ctx->hist[par][m++] = range_of(out->out_v, nout_b * kb);
         ctx->n_hist[par] = m;
         ctx->hist_unknown = false;
+        for (int b = 0; b < batch; ++b) ctx->state_of[par][b] = prune_point * ctx->n_slots + samples[b].state_slot;
+        ctx->n_state_of[par] = batch;
     } else {
         ctx->hist_unknown = true;
     }
@@ -635,8 +664,9 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         cudaStream_t sel_stream = st;
         if (forked) {
             sel_stream = ctx->aux[par];
-            if (!ordered_after_all && cudaStreamWaitEvent(sel_stream, ctx->ev_sel[prv], 0) != cudaSuccess)
-                return fail_cuda(ctx, cudaGetLastError());
+            for (unsigned s = 0; !ordered_after_all && s < kSets; ++s)
+                if ((dep_mask >> s & 1u) && cudaStreamWaitEvent(sel_stream, ctx->ev_sel[s], 0) != cudaSuccess)
+                    return fail_cuda(ctx, cudaGetLastError());
         }
         SelectIO io;
         std::memset(&io, 0, sizeof io);

@@ -256,7 +256,7 @@ class PruneContext:
         return out
 
 
-def context_for(wl, *, max_batch=None, n_prune_points=1, salience_path=SALIENCE_AUTO,
+def context_for(wl, *, max_batch=None, n_prune_points=1, n_state_slots=0, salience_path=SALIENCE_AUTO,
                 device=None) -> PruneContext:
     """A context sized for a synthetic workload (see ``workloads``)."""
     dt = {"bf16": torch.bfloat16, "fp32": torch.float32}[wl.dtype]
@@ -265,7 +265,7 @@ def context_for(wl, *, max_batch=None, n_prune_points=1, salience_path=SALIENCE_
                         max_text=max(s.n_txt for s in wl.samples),
                         max_2d=max(max(s.n_2d for s in wl.samples), 1),
                         max_3d=max(max(s.n_3d for s in wl.samples), 1),
-                        n_prune_points=n_prune_points, tau_2d=wl.tau_2d, tau_3d=wl.tau_3d,
+                        n_prune_points=n_prune_points, n_state_slots=n_state_slots, tau_2d=wl.tau_2d, tau_3d=wl.tau_3d,
                         beta=wl.beta, window_k=wl.window_k, eps_3d=wl.eps_3d,
                         floor_ratio=wl.floor_ratio, cold_start_full_keep=wl.cold_start_full_keep,
                         salience_path=salience_path, device=device)

@@ -379,6 +379,39 @@ def test_pipelined_steps_sharing_an_index_buffer_two_steps_apart():
         assert all(torch.equal(x, y) for x, y in zip(got[t], ref[t])), t
 
 
+def test_pipelined_steps_of_interleaved_episodes_keep_their_states_apart():
+    # three episodes (state slots) take turns; inside an episode the carry-over must see the steps in
+    # call order although selections of different episodes are free to run beside one another
+    import dataclasses
+    wl = W.small_workload(53, batch=2, D=256, H=4, d=128, dtype="bf16", n_txt=(9, 30), n_2d=(100, 180),
+                          n_3d=(140, 333), keep=(0.5, 0.3), steps=12, cold_start=1)
+    devs = [device_tensors(wl, t) for t in range(12)]
+    episodes = [[dataclasses.replace(s, state_slot=s.state_slot + 2 * e) for s in wl.samples] for e in range(3)]
+    order = [0, 1, 2, 0, 0, 1, 2, 2, 1, 0, 2, 1]              # which episode each call belongs to
+
+    def run(flag):
+        ctx = mvla.context_for(wl, n_state_slots=6)
+        outs = [ctx.alloc_outputs(wl.samples, extras=True) for _ in range(12)]
+        seen, kept = set(), []
+        for t, e in enumerate(order):
+            d = devs[t]
+            o = ctx.prune_step(0, episodes[e], wl.mode, d["q"], d["k"], d["v"], d["hidden"],
+                               flags=flag | (0 if e in seen else mvla.FLAG_RESET_STATE), out=outs[t])
+            seen.add(e)
+            kept.append(o.total_kept)
+            if not flag:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        res = [(o.ahat.clone(), o.kept_idx[:n].clone(), o.budgets.clone(), o.out_v[:n].clone())
+               for o, n in zip(outs, kept)]
+        ctx.close()
+        return res
+
+    ref, got = run(0), run(mvla.FLAG_INPUTS_STABLE)
+    for t in range(12):
+        assert all(torch.equal(x, y) for x, y in zip(got[t], ref[t])), t
+
+
 def test_step_segments_in_order_3d_text_2d():
     # the three segments may come in any order; here [3D | text | 2D], two samples, adaptive budgets
     base = W.small_workload(47, batch=2, D=256, H=4, d=128, dtype="bf16", n_txt=(9, 30), n_2d=(140, 77),
