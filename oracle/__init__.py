@@ -24,13 +24,13 @@ MODE_FIXED, MODE_ADAPTIVE = 0, 1
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (-O2, OpenMP over heads only)."""
-    src = os.path.join(_HERE, "mvla_oracle.c")
-    hdr = os.path.join(_HERE, "mvla_oracle.h")
+    srcs = [os.path.join(_HERE, f) for f in ("mvla_oracle.c", "mvla_patch_oracle.c")]
+    deps = srcs + [os.path.join(_HERE, f) for f in ("mvla_oracle.h", "mvla_patch_oracle.h")]
     if (not force and os.path.exists(_LIB_PATH)
-            and os.path.getmtime(_LIB_PATH) >= max(os.path.getmtime(src), os.path.getmtime(hdr))):
+            and os.path.getmtime(_LIB_PATH) >= max(os.path.getmtime(d) for d in deps)):
         return _LIB_PATH
     cmd = ["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
-           "-o", _LIB_PATH, src, "-lm"]
+           "-o", _LIB_PATH] + srcs + ["-lm"]
     subprocess.run(cmd, check=True)
     return _LIB_PATH
 
@@ -57,6 +57,23 @@ class CDiag(C.Structure):
                 ("c_s1", C.c_int32), ("c_s2", C.c_int32), ("c_final", C.c_int32),
                 ("budget", C.c_int32), ("k_2d", C.c_int32), ("k_3d", C.c_int32),
                 ("near_half", C.c_int32), ("near_gate", C.c_int32)]
+
+
+class CPatchParams(C.Structure):
+    _fields_ = [("tau_2d", C.c_double), ("tau_3d", C.c_double), ("beta", C.c_double),
+                ("window_k", C.c_int32), ("eps_3d", C.c_double), ("obj_2d_min", C.c_double),
+                ("bg_prune_prob", C.c_double), ("kmeans_max_iter", C.c_int32),
+                ("cold_start_full_keep", C.c_int32)]
+
+
+class CPatchState(C.Structure):
+    _fields_ = [("t", C.c_int32), ("xhat", C.POINTER(C.c_double))]
+
+
+class CPatchDiag(C.Structure):
+    _fields_ = [("t", C.c_int32), ("iters", C.c_int32), ("n_label", C.c_int32 * 3),
+                ("k_2d", C.c_int32), ("k_3d", C.c_int32), ("centre", C.c_double * 3),
+                ("mu_2d", C.c_double), ("mu_3d", C.c_double), ("kmeans_margin", C.c_double)]
 
 
 def load(path: str):
@@ -95,6 +112,28 @@ def load(path: str):
         L.oracle_prune_step.restype = C.c_int32
         L.oracle_num_threads.argtypes = []
         L.oracle_num_threads.restype = C.c_int32
+        # Alg. 1 patch by patch
+        ppp, psp, pdp = C.POINTER(CPatchParams), C.POINTER(CPatchState), C.POINTER(CPatchDiag)
+        L.oracle_attention.argtypes = [fp, fp, C.c_int32, C.c_int32, sp, dp]
+        L.oracle_attention.restype = None
+        L.oracle_ortho_decompose.argtypes = [dp, dp, C.c_int32, dp, dp]
+        L.oracle_ortho_decompose.restype = None
+        L.oracle_patch_indicators.argtypes = [dp, C.c_int32, C.c_int32, dp, dp]
+        L.oracle_patch_indicators.restype = None
+        L.oracle_kmeans1d.argtypes = [dp, C.c_int32, C.c_int32, ip, dp, dp]
+        L.oracle_kmeans1d.restype = C.c_int32
+        L.oracle_patch_c_s1.argtypes = [C.c_double, C.c_double, C.c_double]
+        L.oracle_patch_c_s1.restype = C.c_int32
+        L.oracle_patch_c_s2.argtypes = [C.c_int32, C.c_double, C.c_double, C.c_double, C.c_double,
+                                        C.c_double, ppp]
+        L.oracle_patch_c_s2.restype = C.c_int32
+        L.oracle_patch_fuse.argtypes = [C.c_int32, C.c_int32]
+        L.oracle_patch_fuse.restype = C.c_int32
+        L.oracle_patch_select.argtypes = [dp, dp, dp, sp, ppp, psp, ip, ip, ip, pdp]
+        L.oracle_patch_select.restype = C.c_int32
+        L.oracle_patch_step.argtypes = [fp, fp, fp, C.c_int32, C.c_int32, C.c_int32, sp, dp, ppp, psp,
+                                        ip, ip, ip, pdp, dp, dp]
+        L.oracle_patch_step.restype = C.c_int32
     return L
 
 
@@ -288,3 +327,150 @@ def run_workload_step(wl, step: int, states: List[State]) -> List[StepResult]:
     return [prune_step(ten.q, ten.k, ten.hidden if wl.mode == MODE_ADAPTIVE else None,
                        wl.n_heads, wl.head_dim, wl.d_model, s, p, wl.mode, states[b])
             for b, s in enumerate(wl.samples)]
+
+
+# --------------------------------------------------------------------------
+# Alg. 1 patch by patch (mvla_patch_oracle.c)
+# --------------------------------------------------------------------------
+LABEL_BG, LABEL_ROB, LABEL_OBJ = 0, 1, 2
+
+
+def c_patch_params(tau_2d=0.08, tau_3d=0.20, beta=0.85, window_k=7, eps_3d=0.02, obj_2d_min=0.5,
+                   bg_prune_prob=0.9, kmeans_max_iter=32, cold_start_full_keep=1) -> CPatchParams:
+    return CPatchParams(float(tau_2d), float(tau_3d), float(beta), int(window_k), float(eps_3d),
+                        float(obj_2d_min), float(bg_prune_prob), int(kmeans_max_iter),
+                        int(cold_start_full_keep))
+
+
+def patch_params_of(wl) -> CPatchParams:
+    return c_patch_params(wl.tau_2d, wl.tau_3d, wl.beta, wl.window_k, wl.eps_3d,
+                          wl.extra.get("obj_2d_min", 0.5), 1.0 - wl.floor_ratio,
+                          wl.extra.get("kmeans_max_iter", 32), wl.cold_start_full_keep)
+
+
+def attention(q, k, n_heads, head_dim, s) -> np.ndarray:
+    """alpha[h, i, j]: [H, n_txt, n_vis]."""
+    q, qp = _f32(q)
+    k, kp = _f32(k)
+    cs = c_sample(s)
+    out = np.zeros((n_heads, cs.n_txt, cs.n_2d + cs.n_3d), dtype=np.float64)
+    lib().oracle_attention(qp, kp, n_heads, head_dim, C.byref(cs), out.ctypes.data_as(C.POINTER(C.c_double)))
+    return out
+
+
+def ortho_decompose(a2, a3):
+    a2, p2 = _f64(a2)
+    a3, p3 = _f64(a3)
+    para, ortho = np.zeros_like(a2), np.zeros_like(a2)
+    dp = lambda a: a.ctypes.data_as(C.POINTER(C.c_double))
+    lib().oracle_ortho_decompose(p2, p3, len(a2), dp(para), dp(ortho))
+    return para, ortho
+
+
+def patch_indicators(alpha, l1) -> np.ndarray:
+    """alpha: [rows, 2P]; l1: [2P] -> x [P, 4]."""
+    alpha, ap = _f64(alpha)
+    l1, lp = _f64(l1)
+    rows, nv = alpha.shape
+    x = np.zeros((nv // 2, 4), dtype=np.float64)
+    lib().oracle_patch_indicators(ap, rows, nv // 2, lp, x.ctypes.data_as(C.POINTER(C.c_double)))
+    return x
+
+
+def kmeans1d(v, max_iter=32):
+    v, vp = _f64(v)
+    labels = np.zeros(len(v), dtype=np.int32)
+    centre = np.zeros(3, dtype=np.float64)
+    margin = C.c_double()
+    it = lib().oracle_kmeans1d(vp, len(v), max_iter, labels.ctypes.data_as(C.POINTER(C.c_int32)),
+                               centre.ctypes.data_as(C.POINTER(C.c_double)), C.byref(margin))
+    return labels, centre, it, margin.value
+
+
+def patch_c_s1(m, tau_2d, tau_3d) -> int:
+    return lib().oracle_patch_c_s1(float(m), float(tau_2d), float(tau_3d))
+
+
+def patch_c_s2(label, m2, m3, mu_2d, mu_3d, u, params: CPatchParams) -> int:
+    return lib().oracle_patch_c_s2(int(label), float(m2), float(m3), float(mu_2d), float(mu_3d),
+                                   float(u), C.byref(params))
+
+
+def patch_fuse(c_s1, c_s2) -> int:
+    return lib().oracle_patch_fuse(int(c_s1), int(c_s2))
+
+
+class PatchState:
+    """Smoothed per-patch indicators of one (prune point, sample)."""
+
+    def __init__(self, n_patch: int):
+        self.xhat = np.zeros((n_patch, 4), dtype=np.float64)
+        self.c = CPatchState(0, self.xhat.ctypes.data_as(C.POINTER(C.c_double)))
+
+    @property
+    def t(self) -> int:
+        return self.c.t
+
+
+@dataclass
+class PatchResult:
+    kept_idx: np.ndarray
+    labels: np.ndarray
+    cand: np.ndarray          # [P, 3] = (C_S1, C_S2, C_final)
+    attn: Optional[np.ndarray]
+    x: Optional[np.ndarray]
+    xhat: np.ndarray
+    t: int
+    iters: int
+    n_label: np.ndarray
+    k_2d: int
+    k_3d: int
+    centre: np.ndarray
+    mu_2d: float
+    mu_3d: float
+    kmeans_margin: float
+
+
+def _patch_result(n, kept, labels, cand, attn, x, state, dg) -> PatchResult:
+    return PatchResult(kept[:n].copy(), labels, cand, attn, x, state.xhat.copy(), dg.t, dg.iters,
+                       np.array(dg.n_label[:]), dg.k_2d, dg.k_3d, np.array(dg.centre[:]), dg.mu_2d,
+                       dg.mu_3d, dg.kmeans_margin)
+
+
+def patch_select(a, x, u, s, params: CPatchParams, state: PatchState) -> PatchResult:
+    a, ap = _f64(a)
+    x, xp = _f64(x)
+    u, up = _f64(u)
+    cs = c_sample(s)
+    P = cs.n_2d
+    kept = np.zeros(cs.n_txt + 2 * P, dtype=np.int32)
+    labels = np.zeros(P, dtype=np.int32)
+    cand = np.zeros((P, 3), dtype=np.int32)
+    dg = CPatchDiag()
+    ip = lambda v: v.ctypes.data_as(C.POINTER(C.c_int32))
+    n = lib().oracle_patch_select(ap, xp, up, C.byref(cs), C.byref(params), C.byref(state.c), ip(labels),
+                                  ip(cand), ip(kept), C.byref(dg))
+    return _patch_result(n, kept, labels, cand, None, None, state, dg)
+
+
+def patch_step(q, k, hidden, n_heads, head_dim, d_model, s, u, params: CPatchParams,
+               state: PatchState) -> PatchResult:
+    q, qp = _f32(q)
+    k, kp = _f32(k)
+    hidden, hp = _f32(hidden)
+    u, up = _f64(u)
+    cs = c_sample(s)
+    P = cs.n_2d
+    assert cs.n_3d == P, "a patch owns one 2D and one 3D token"
+    kept = np.zeros(cs.n_txt + 2 * P, dtype=np.int32)
+    labels = np.zeros(P, dtype=np.int32)
+    cand = np.zeros((P, 3), dtype=np.int32)
+    attn = np.zeros(2 * P)
+    x = np.zeros((P, 4))
+    dg = CPatchDiag()
+    ip = lambda v: v.ctypes.data_as(C.POINTER(C.c_int32))
+    dp = lambda v: v.ctypes.data_as(C.POINTER(C.c_double))
+    n = lib().oracle_patch_step(qp, kp, hp, n_heads, head_dim, d_model, C.byref(cs), up, C.byref(params),
+                                C.byref(state.c), ip(labels), ip(cand), ip(kept), C.byref(dg), dp(attn), dp(x))
+    assert n >= 0
+    return _patch_result(n, kept, labels, cand, attn, x, state, dg)

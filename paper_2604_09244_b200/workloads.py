@@ -30,6 +30,7 @@ import numpy as np
 
 MODE_FIXED = 0
 MODE_ADAPTIVE = 1
+MODE_PATCH = 2
 
 
 # --------------------------------------------------------------------------
@@ -103,7 +104,7 @@ class Workload:
     n_heads: int
     head_dim: int
     d_model: int
-    mode: int                  # MODE_FIXED | MODE_ADAPTIVE
+    mode: int                  # MODE_FIXED | MODE_ADAPTIVE | MODE_PATCH
     samples: List[Sample]
     steps: List[Tensors]       # one entry per action step (len 1 unless config 5)
     cold_start_full_keep: int = 0
@@ -349,10 +350,67 @@ def small_workload(seed: int, *, batch=2, D=256, H=4, d=64, dtype="bf16", mode=M
     return Workload(f"small_{seed}", dtype, H, d, D, mode, samples, out,
                     cold_start_full_keep=cold_start, seed=seed)
 
+def patch_workload(seed: int = 5, *, batch: int = 1, D=4096, H=32, d=128, dtype="bf16", n_txt=(32,),
+                   n_patch=(256,), steps: int = 1, cold_start: int = 0, text_first: bool = False) -> Workload:
+    """Paired-patch workload in the shape of the paper's host model (App. "MVLA Models": 256 image
+    tokens from 16x16 patches + 256 point tokens): patch p owns 2D token p and 3D token p of its
+    sample.  Per sample about 4 % of the patches are "target object" patches (both hidden rows x4),
+    12 % "robot" patches (both rows x2), the rest background; one object patch has its 3D row
+    scaled by 0.05 (a 3D response near zero); of the other patches 20 % have the 3D row scaled by 0.4
+    and 20 % by 2.5, which moves the patch's 3D feature share across both synthetic thresholds.
+    ``extra["rand_u"][t]`` holds, per action step, one uniform float32 in [0, 1) per patch (samples
+    back to back): the random numbers of the background rule, drawn here and handed to whoever runs
+    the method.  Later steps drift like the action-iteration workload."""
+    rng = np.random.default_rng(seed)
+    samples, off = [], 0
+    for b in range(batch):
+        nt, P = n_txt[b % len(n_txt)], n_patch[b % len(n_patch)]
+        if text_first:
+            smp = Sample(seq_off=off, off_txt=0, n_txt=nt, off_2d=nt, n_2d=P, off_3d=nt + P, n_3d=P,
+                         state_slot=b)
+        else:
+            smp = layout_2d_3d_txt(off, nt, P, P, state_slot=b)
+        samples.append(smp)
+        off += smp.seq_len
+    hidden = rng.standard_normal((off, D), dtype=np.float32)
+    w = _draw_weights(rng, D, H * d)
+    roles = []
+    for smp in samples:
+        P = smp.n_2d
+        perm = rng.permutation(P)
+        n_obj, n_rob = max(1, _rhu(0.04 * P)), max(1, _rhu(0.12 * P))
+        obj, rob, rest = perm[:n_obj], perm[n_obj:n_obj + n_rob], perm[n_obj + n_rob:]
+        r2, r3 = smp.seq_off + smp.off_2d, smp.seq_off + smp.off_3d
+        for idx, g in ((obj, 4.0), (rob, 2.0)):
+            hidden[r2 + idx] *= np.float32(g)
+            hidden[r3 + idx] *= np.float32(g)
+        hidden[r3 + obj[0]] *= np.float32(0.05)
+        others = np.concatenate([obj[1:], rob, rest])
+        sel = rng.permutation(len(others))
+        n20 = _rhu(0.2 * len(others))
+        hidden[r3 + others[sel[:n20]]] *= np.float32(0.4)
+        hidden[r3 + others[sel[n20:2 * n20]]] *= np.float32(2.5)
+        roles.append({"obj": np.sort(obj), "rob": np.sort(rob)})
+    n_pat = sum(smp.n_2d for smp in samples)
+    out, us = [], []
+    for t in range(steps):
+        if t > 0:
+            rows = np.sort(rng.choice(off, size=max(1, _rhu(0.10 * off)), replace=False))
+            hidden[rows] += rng.standard_normal((len(rows), D), dtype=np.float32) * np.float32(0.1)
+        out.append(_project(hidden.copy(), w, H, d, dtype))
+        us.append(rng.random(n_pat, dtype=np.float32))
+    return Workload(f"patch_{seed}", dtype, H, d, D, MODE_PATCH, samples, out,
+                    cold_start_full_keep=cold_start, seed=seed, extra={"rand_u": us, "roles": roles})
+
+
+def patch_mla(seed: int = 5, batch: int = 1) -> Workload:
+    """The paper's host-model shape: 32 text + 256 image + 256 point tokens, D = 4096, 32 x 128, bf16."""
+    return patch_workload(seed, batch=batch)
+
 
 def by_name(name: str, seed: Optional[int] = None) -> Workload:
     table = {"config1": config1_tiny, "config2": config2_single_frame,
              "config3": config3_multi_view, "config4": config4_batched,
-             "config5": config5_action_iteration}
+             "config5": config5_action_iteration, "patch_mla": patch_mla}
     fn = table[name]
     return fn() if seed is None else fn(seed=seed)

@@ -9,10 +9,13 @@ import pytest
 import oracle
 import test_oracle_pins as pins
 
-SRC = os.path.join(os.path.dirname(oracle.__file__), "mvla_oracle.c")
-HDR = os.path.join(os.path.dirname(oracle.__file__), "mvla_oracle.h")
+import test_patch_oracle_pins as patch_pins
+
+ODIR = os.path.dirname(oracle.__file__)
+FILES = ("mvla_oracle.c", "mvla_oracle.h", "mvla_patch_oracle.c", "mvla_patch_oracle.h")
 
 PIN_TESTS = [getattr(pins, n) for n in dir(pins) if n.startswith("test_")]
+PATCH_PIN_TESTS = [getattr(patch_pins, n) for n in dir(patch_pins) if n.startswith("test_")]
 
 MUTATIONS = {
     "logit scale dropped": ("logit[j] = acc / sqrt((double)d);", "logit[j] = acc;"),
@@ -52,20 +55,65 @@ MUTATIONS = {
 MUTATIONS.pop("state updated after the decision")
 
 
+# Mistakes planted in the patch-by-patch statement of Alg. 1 (mvla_patch_oracle.c).
+PATCH_MUTATIONS = {
+    "projection on the wrong vector": ("d22 += a2[r] * a2[r];", "d22 += a3[r] * a3[r];"),
+    "orthogonal part keeps the parallel part": ("ortho[r] = a3[r] - para[r];", "ortho[r] = a3[r];"),
+    "3D share uses the whole vector": ("x[4 * p + 3] = no / (n2 + n3);", "x[4 * p + 3] = n3 / (n2 + n3);"),
+    "2D attention share inverted": ("x[4 * p + 2] = n2 / (n2 + n3);", "x[4 * p + 2] = n3 / (n2 + n3);"),
+    "feature shares swapped": ("x[4 * p + 1] = f3 / (f2 + f3);", "x[4 * p + 1] = f2 / (f2 + f3);"),
+    "3D token of the patch read from the wrong column": ("a3[r] = alpha[(size_t)r * nv + P + p];",
+                                                         "a3[r] = alpha[(size_t)r * nv + p];"),
+    "attention not normalised": ("for (int32_t j = 0; j < nv; ++j) out[j] = exp(out[j] - mx) / den;",
+                                 "for (int32_t j = 0; j < nv; ++j) out[j] = exp(out[j] - mx);"),
+    "k-means ties go up": ("if (dc < bd) { second = bd; bd = dc; best = c; }", "if (dc <= bd) { second = bd; bd = dc; best = c; }"),
+    "k-means centre is a sum": ("if (cnt > 0) centre[c] = acc / cnt;", "if (cnt > 0) centre[c] = acc;"),
+    "k-means starts from the maximum twice": ("centre[1] = n > 0 ? sum / n : 0.0;", "centre[1] = mx;"),
+    "patch threshold inclusive": ("if (mhat_s1_3d < tau_2d) return ORACLE_SET_2D;", "if (mhat_s1_3d <= tau_2d) return ORACLE_SET_2D;"),
+    "background kept when it should go": ("return u < p->bg_prune_prob ? 0 : both;", "return u < p->bg_prune_prob ? both : 0;"),
+    "robot rule compares 2D first": ("if (m3 > mu_3d) return both;                    /* pure 3D reliance above the baseline */\n        if (m2 > mu_2d) return ORACLE_SET_2D;",
+                                     "if (m2 > mu_2d) return ORACLE_SET_2D;\n        if (m3 > mu_3d) return both;"),
+    "object rule is an or": ("if (m2 > p->obj_2d_min && m3 < p->eps_3d) return ORACLE_SET_2D;",
+                             "if (m2 > p->obj_2d_min || m3 < p->eps_3d) return ORACLE_SET_2D;"),
+    "empty semantic set falls back to the modality set": ("if (c_s2 == 0) return 0;", "if (c_s2 == 0) return c_s1;"),
+    "patch conflict keeps the modality set": ("return cf != 0 ? cf : c_s2;", "return cf != 0 ? cf : c_s1;"),
+    "3D mask emits the 2D token": ("kept_idx[n] = s->off_3d + q; ++n; ++dg.k_3d;", "kept_idx[n] = s->off_2d + q; ++n; ++dg.k_3d;"),
+    "baseline from the instantaneous shares": ("s3 += st->xhat[4 * q + 3];", "s3 += x[4 * q + 3];"),
+    "clusters the 2D mass only": ("mass[q] = a[q] + a[P + q];", "mass[q] = a[q];"),
+    "patch cold start prunes": ("if (cold) cf = ORACLE_SET_2D | ORACLE_SET_3D;", "if (0) cf = 0;"),
+}
+
+
+def _run_mutant(which, old, new, tests, tmp_path, monkeypatch, name):
+    for f in FILES:
+        src = open(os.path.join(ODIR, f)).read()
+        if f == which:
+            assert src.count(old) == 1, f"mutation site not found exactly once: {name}"
+            src = src.replace(old, new)
+        (tmp_path / f).write_text(src)
+    so = tmp_path / "libmut.so"
+    subprocess.run(["gcc", "-O1", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-w", "-o", str(so),
+                    str(tmp_path / "mvla_oracle.c"), str(tmp_path / "mvla_patch_oracle.c"), "-lm"], check=True)
+    oracle.lib()                                            # make sure the real one is loaded first
+    monkeypatch.setattr(oracle, "_lib", oracle.load(str(so)))
+    return _caught(tests)
+
+
+@pytest.mark.parametrize("name", sorted(PATCH_MUTATIONS))
+def test_patch_pins_catch_planted_mistake(name, tmp_path, monkeypatch):
+    old, new = PATCH_MUTATIONS[name]
+    assert _run_mutant("mvla_patch_oracle.c", old, new, PATCH_PIN_TESTS, tmp_path, monkeypatch, name), f"no pin noticed: {name}"
+
+
 @pytest.mark.parametrize("name", sorted(MUTATIONS))
 def test_pins_catch_planted_mistake(name, tmp_path, monkeypatch):
     old, new = MUTATIONS[name]
-    src = open(SRC).read()
-    assert src.count(old) == 1, f"mutation site not found exactly once: {name}"
-    (tmp_path / "mvla_oracle.c").write_text(src.replace(old, new))
-    (tmp_path / "mvla_oracle.h").write_text(open(HDR).read())
-    so = tmp_path / "libmut.so"
-    subprocess.run(["gcc", "-O1", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-w", "-o", str(so),
-                    str(tmp_path / "mvla_oracle.c"), "-lm"], check=True)
-    oracle.lib()                                            # make sure the real one is loaded first
-    monkeypatch.setattr(oracle, "_lib", oracle.load(str(so)))
+    assert _run_mutant("mvla_oracle.c", old, new, PIN_TESTS, tmp_path, monkeypatch, name), f"no pin noticed: {name}"
+
+
+def _caught(tests):
     caught = []
-    for fn in PIN_TESTS:
+    for fn in tests:
         marks = [m for m in getattr(fn, "pytestmark", []) if m.name == "parametrize"]
         argsets = [()]
         if marks:
@@ -77,4 +125,4 @@ def test_pins_catch_planted_mistake(name, tmp_path, monkeypatch):
                 caught.append(fn.__name__)
             except Exception:
                 caught.append(fn.__name__)
-    assert caught, f"no pin noticed: {name}"
+    return caught
