@@ -55,6 +55,11 @@ def make_workload(name: str):
         return W.config4_batched(), "configs[3]: batched serving, batch 16, adaptive per-sample keep"
     if name == "config5":
         return W.config5_action_iteration(T=2), "configs[4]: action iteration, one step (t=2), adaptive keep 30 %"
+    if name == "patch_mla":
+        return W.patch_mla(), "paired patches in the paper's host-model shape (App. MVLA Models): batch 1, D=4096, " \
+                              "32 heads x 128, 32 text + 256 2D + 256 3D tokens, bf16, Alg. 1 patch by patch (masks, no budget)"
+    if name == "patch_mla_b16":
+        return W.patch_mla(batch=16), "paired patches, host-model shape, batch 16"
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -66,7 +71,7 @@ def algorithmic_bytes(wl, kept_rows: int):
     nv = wl.total_vis
     nt = sum(s.n_txt for s in wl.samples)
     sal = (nv + nt) * hd * e
-    l1 = nv * wl.d_model * e if wl.mode == 1 else 0
+    l1 = nv * wl.d_model * e if wl.mode in (1, 2) else 0
     comp = 2 * kept_rows * (wl.d_model + 2 * hd) * e
     return {"salience": sal, "l1": l1, "compact": comp, "scores": 12 * nv,
             "total": sal + l1 + comp + 12 * nv}
@@ -131,14 +136,21 @@ def time_oracle(wl, max_steps: int, max_seconds: float):
     import numpy as np
     import oracle
     t = wl.steps[-1]
-    p = oracle.params_of(wl)
+    patch = wl.mode == 2
+    p = oracle.patch_params_of(wl) if patch else oracle.params_of(wl)
     n = 0
     t0 = time.perf_counter()
     while True:
+        pat = 0
         for s in wl.samples:
-            st = oracle.State(s.n_vis)
-            r = oracle.prune_step(t.q, t.k, t.hidden if wl.mode == 1 else None, wl.n_heads, wl.head_dim,
-                                  wl.d_model, s, p, wl.mode, st)
+            if patch:
+                r = oracle.patch_step(t.q, t.k, t.hidden, wl.n_heads, wl.head_dim, wl.d_model, s,
+                                      wl.extra["rand_u"][-1][pat:pat + s.n_2d], p, oracle.PatchState(s.n_2d))
+                pat += s.n_2d
+            else:
+                st = oracle.State(s.n_vis)
+                r = oracle.prune_step(t.q, t.k, t.hidden if wl.mode == 1 else None, wl.n_heads, wl.head_dim,
+                                      wl.d_model, s, p, wl.mode, st)
             for src in (t.hidden, t.k, t.v):
                 oracle.compact(src, s.seq_off, r.kept_idx)
         n += 1
@@ -188,6 +200,8 @@ def run_ours(args, rank, local, world):
     # A single-frame workload is a stream of independent requests: each step starts a fresh smoothed
     # state, and requests in flight at the same time hold distinct state slots, as the concurrent
     # requests of a server do.  A workload with carry-over keeps its one episode (one slot per sample).
+    is_patch = wl.mode == 2
+    u_dev = torch.from_numpy(wl.extra["rand_u"][-1]).to(dev) if is_patch else None
     n_req = 8 if not wl.cold_start_full_keep else 1
     ctx = mvla.context_for(wl, n_state_slots=n_req * len(wl.samples))
     probe = ctx.alloc_outputs(wl.samples, extras=False)
@@ -212,12 +226,14 @@ def run_ours(args, rank, local, world):
     def step(i, extra=0):
         s, o = sets[i % n_sets], outs[i % n_sets]
         return ctx.prune_step(0, cs_req[i % n_req], wl.mode, s["q"], s["k"], s["v"], s["hidden"],
-                              flags=flags | extra, out=o)
+                              flags=flags | extra, out=o, rand_u=u_dev)
 
     o0 = step(0)
     torch.cuda.synchronize()
-    kept_rows = o0.total_kept
-    launches_per_step = 3 + (1 if wl.mode == 1 else 0)
+    # the patch-by-patch path decides its row count on the device (total_kept is then the capacity bound)
+    kept_rows = int(o0.out_offsets[-1]) if is_patch else o0.total_kept
+    # patch path: norms, scoring, head sum, indicators, decide, emit, row copy
+    launches_per_step = 7 if is_patch else 3 + (1 if wl.mode == 1 else 0)
 
     # ---- device-resident timing: CUDA graphs of back-to-back steps over the rotating sets
     per_graph = -(-200 // n_sets) * n_sets   # ~200 steps per graph: the pipeline of overlapping steps fills once per replay
@@ -284,19 +300,26 @@ def run_ours(args, rank, local, world):
     attn_b = [torch.empty(wl.total_vis, dtype=torch.float32, device=dev) for _ in range(n_sets)]
     l1_b = [torch.empty(wl.total_vis, dtype=torch.float32, device=dev) for _ in range(n_sets)]
     adaptive = wl.mode == 1
+    x_b = [torch.empty(wl.total_vis // 2, 4, dtype=torch.float32, device=dev) for _ in range(n_sets)] if is_patch else None
 
     def st_salience(i):
         s = sets[i % n_sets]
+        if is_patch:
+            ctx.patch_indicators(cs, s["q"], s["k"], s["hidden"], attn_out=attn_b[i % n_sets], x_out=x_b[i % n_sets])
+            return
         ctx.salience(cs, s["q"], s["k"], s["hidden"] if adaptive else None, attn_out=attn_b[i % n_sets],
                      l1_out=l1_b[i % n_sets] if adaptive else None)
 
     def st_select(i):
+        if is_patch:
+            ctx.patch_select(0, cs, attn_b[i % n_sets], x_b[i % n_sets], u_dev, flags=flags, out=outs[i % n_sets])
+            return
         ctx.select(0, cs, wl.mode, attn_b[i % n_sets], l1_b[i % n_sets] if adaptive else None, flags=flags,
                    out=outs[i % n_sets])
 
     def st_compact(i):
         s, o = sets[i % n_sets], outs[i % n_sets]
-        ctx.compact(cs, o.kept_idx, o.out_offsets, kept_rows, s["hidden"], s["k"], s["v"],
+        ctx.compact(cs, o.kept_idx, o.out_offsets, probe_rows if is_patch else kept_rows, s["hidden"], s["k"], s["v"],
                     out_hidden=o.out_hidden, out_k=o.out_k, out_v=o.out_v)
 
     stage_us = {}
@@ -327,14 +350,18 @@ def run_ours(args, rank, local, world):
     res_dev = [o.out_hidden[:kept_rows], o.out_k[:kept_rows], o.out_v[:kept_rows], o.kept_idx[:kept_rows],
                o.out_offsets, o.budgets]
     res_host = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in res_dev]
-    h2d = in_bytes
+    u_pin = torch.from_numpy(wl.extra["rand_u"][-1]).pin_memory() if is_patch else None
+    u_stage = torch.empty_like(u_dev) if is_patch else None
+    h2d = in_bytes + (u_pin.numel() * 4 if is_patch else 0)
     d2h = sum(t.numel() * t.element_size() for t in res_dev)
 
     def e2e_step():
         for n in names:
             stage_in[n].copy_(pin_in[n], non_blocking=True)
+        if is_patch:
+            u_stage.copy_(u_pin, non_blocking=True)
         ctx.prune_step(0, cs, wl.mode, stage_in["q"], stage_in["k"], stage_in["v"], stage_in["hidden"],
-                       flags=flags, out=o)
+                       flags=flags, out=o, rand_u=u_stage)
         for dst, src in zip(res_host, res_dev):
             dst.copy_(src, non_blocking=True)
 

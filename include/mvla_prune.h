@@ -55,6 +55,8 @@ extern "C" {
 
 #define MVLA_MODE_FIXED    0   /* per-modality keep ratios keep_2d / keep_3d */
 #define MVLA_MODE_ADAPTIVE 1   /* one total keep ratio, split by the stage rules */
+#define MVLA_MODE_PATCH    2   /* Alg. 1 taken literally, patch by patch: no budget, the masks decide (mvla_prune_step;
+                                  needs patch_path = 1 at create and n_2d == n_3d: patch p owns 2D token p and 3D token p) */
 
 #define MVLA_FLAG_RESET_STATE     1u  /* restart the episode: this call is action step t = 1 */
 #define MVLA_FLAG_NO_STATE_UPDATE 2u  /* dry run: decide as usual but leave the smoothed state and t untouched */
@@ -99,6 +101,12 @@ typedef struct mvla_config {
     double beta;               /* Eq. 9 */
     double eps_3d;
     double floor_ratio;
+    /* patch-by-patch path (MVLA_MODE_PATCH) */
+    double obj_2d_min;         /* target-object rule (Sec. 4.2): {2D} only when M^S2_2D,p > obj_2d_min and
+                                  M^S2_3D,p < eps_3d; 0 -> 0.5 */
+    int32_t patch_path;        /* 1: allocate the per-patch state and the attention scratch
+                                  (n_heads x max_text x max_batch x (max_2d + max_3d) floats) */
+    int32_t kmeans_max_iter;   /* rounds of the 1-D K-Means (Sec. 4.2); 0 -> 32 */
 } mvla_config;
 
 /* One batch element (host array).  Offsets are rows relative to seq_off; the three segments
@@ -123,12 +131,29 @@ typedef struct mvla_diag {
     float mhat[4];             /* the same, smoothed (Eqs. 8, 9) */
 } mvla_diag;
 
+/* Per-sample record of the patch-by-patch path (device array, optional). */
+#define MVLA_LABEL_BG  0       /* K-Means classes by ascending centre (Sec. 4.2) */
+#define MVLA_LABEL_ROB 1
+#define MVLA_LABEL_OBJ 2
+typedef struct mvla_patch_diag {
+    int32_t t;                 /* 1-based action step this call was */
+    int32_t iters;             /* K-Means rounds run */
+    int32_t n_label[3];        /* patches per class */
+    int32_t k_2d, k_3d;        /* kept tokens per modality */
+    int32_t n_out;             /* kept rows of the sample = n_txt + k_2d + k_3d */
+    float centre[3];           /* class centres, ascending */
+    float mu_2d, mu_3d;        /* baselines of Sec. 4.2 */
+    float reserved[3];
+} mvla_patch_diag;
+
 /* Inputs of the fused step (device pointers). hidden may be NULL in FIXED mode when
  * out_hidden is NULL too. */
 typedef struct mvla_tensors {
     const void *q, *k, *v;     /* [rows, H, d] */
     const void *hidden;        /* [rows, D] */
     int64_t rows;              /* rows allocated in each tensor (bounds the TMA descriptors) */
+    const float *rand_u;       /* MVLA_MODE_PATCH: one uniform number in [0, 1) per patch, samples back to back
+                                  (the draws of the background rule); NULL otherwise */
 } mvla_tensors;
 
 /* Outputs of the fused step (device pointers, caller-owned). */
@@ -142,6 +167,11 @@ typedef struct mvla_outputs {
     float *ahat;               /* [sum n_vis] smoothed scores used for ranking  nullable */
     float *z;                  /* [sum n_vis] smoothed scores normalised to mean 1 per modality  nullable */
     mvla_diag *diag;           /* [batch]  nullable */
+    /* MVLA_MODE_PATCH only, all nullable: */
+    float *patch_x;            /* [sum P][4] instantaneous [M^S1_2D, M^S1_3D, M^S2_2D, M^S2_3D] of every patch */
+    float *patch_xhat;         /* [sum P][4] the same, smoothed */
+    int32_t *patch_info;       /* [sum P] label | C_S1 << 2 | C_S2 << 4 | C_final << 6 */
+    struct mvla_patch_diag *patch_diag;   /* [batch] */
 } mvla_outputs;
 
 /* Kept rows of a sample: n_txt + B where B = n_2d + n_3d on a cold-start step (t = 1 with
@@ -203,7 +233,10 @@ int32_t mvla_compact(mvla_ctx *ctx, int32_t batch, const mvla_sample *samples,
  * The whole prune point (Alg. 1) as one submission: salience (+ L1 norms in
  * ADAPTIVE mode), carry-over, budget, select, compact.  Equivalent to the three
  * calls above on the same arguments.  `total_kept_out` (host, nullable) receives
- * the number of output rows.
+ * the number of output rows.  In MVLA_MODE_PATCH the chain is mvla_patch_indicators, mvla_patch_select,
+ * mvla_compact; the row count is then known only on the device (out_offsets[batch]) and
+ * `total_kept_out` receives the capacity bound sum(n_txt + n_2d + n_3d); `budgets` receives the kept
+ * counts per modality; MVLA_FLAG_INPUTS_STABLE is accepted and ignored.
  */
 int32_t mvla_prune_step(mvla_ctx *ctx, int32_t prune_point, int32_t batch,
                         const mvla_sample *samples, int32_t mode, uint32_t flags,
@@ -236,6 +269,40 @@ int32_t mvla_prune_step(mvla_ctx *ctx, int32_t prune_point, int32_t batch,
 int32_t mvla_salience_noalloc(int32_t device, int32_t dtype, int32_t n_heads, int32_t head_dim,
                               int32_t batch, const mvla_sample *samples, const void *q, const void *k,
                               int64_t rows, float *attn_out, void *stream);
+
+/*
+ * Per-patch indicators X_t of Alg. 1 (needs patch_path = 1; every sample has n_2d == n_3d = P):
+ *   M^S1_{2D,3D},p = share of the L1 feature norm of the patch's 2D / 3D token (Eq. 3-1, the term of patch p);
+ *   M^S2_2D,p      = ||a2||_1 / (||a2||_1 + ||a3||_1) with a2, a3 the attention vectors (one entry per head and
+ *                    text query) of the patch's 2D and 3D token (Eq. P2D);
+ *   M^S2_3D,p      = ||a3 - <a3,a2>/<a2,a2> a2||_1 / (||a2||_1 + ||a3||_1), the part of a3 orthogonal to a2
+ *                    (Eq. 3-4, Eq. P3D).
+ * attn_out: device, sum(2P) floats, the per-token scores a_j as mvla_salience writes them.
+ * x_out: device, [sum P][4] floats = [M^S1_2D, M^S1_3D, M^S2_2D, M^S2_3D], samples back to back.  Stateless.
+ */
+int32_t mvla_patch_indicators(mvla_ctx *ctx, int32_t batch, const mvla_sample *samples, const void *q,
+                              const void *k, const void *hidden, int64_t rows, float *attn_out,
+                              float *x_out, void *stream);
+
+/*
+ * Alg. 1 stages 1-4 patch by patch: temporal predictor of the four indicators of every patch (Eqs. 8, 9),
+ * dual threshold (Sec. 4.1), 1-D K-Means with K = 3 on the patches' attention mass attn[p] + attn[P + p] and
+ * the rules for background / robot / target-object patches (Sec. 4.2), candidate fusion (Sec. 4.4), masks
+ * (Eq. 10) written as kept positions in ascending order merged with all text positions.
+ *   K-Means: centres start at (min, mean, max); a round assigns every patch to its nearest centre (ties to
+ *   the lower one) and, unless no label changed, moves each non-empty class's centre to its mean; at most
+ *   kmeans_max_iter rounds; classes by ascending centre are background, robot, target object.
+ *   Background patch: discarded when rand_u[p] < 1 - floor_ratio.  Baselines mu: means over the sample's
+ *   patches of the smoothed M^S2 shares.  Action step t = 1 with cold_start_full_keep keeps everything.
+ * The number of kept rows is data dependent: out_offsets [batch + 1] and counts [batch][2] = kept 2D / 3D
+ * tokens are written on the device; kept_idx needs capacity sum(n_txt + 2P).  keep_* of the samples are
+ * ignored.  Advances the slots' step counters like mvla_select.  flags: RESET_STATE, NO_STATE_UPDATE.
+ * xhat_out [sum P][4], info_out [sum P] (label | C_S1 << 2 | C_S2 << 4 | C_final << 6), diag [batch]: nullable.
+ */
+int32_t mvla_patch_select(mvla_ctx *ctx, int32_t prune_point, int32_t batch, const mvla_sample *samples,
+                          uint32_t flags, const float *attn, const float *x, const float *rand_u,
+                          int32_t *kept_idx, int32_t *out_offsets, int32_t *counts, float *xhat_out,
+                          int32_t *info_out, mvla_patch_diag *diag, void *stream);
 
 /* Free everything the context owns.  NULL is accepted.  The caller must have
  * synchronised any stream that still runs work enqueued through the context. */

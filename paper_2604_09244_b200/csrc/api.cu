@@ -30,6 +30,14 @@ struct mvla_ctx {
                                  // calls; the sets rotate from step to step (a step's scoring may run beside
                                  // the selections of the steps before it)
     size_t vis_all;              // max_batch * max_vis
+    // patch-by-patch path (cfg.patch_path): attention copy [H][max_text][vis_all], per-patch smoothed
+    // indicators [n_prune_points][n_slots][max_patch][4], and the scratch between its kernels
+    float* alpha_ws;
+    float* xhat_patch;
+    float* patch_x_ws;           // [vis_all / 2][4]
+    uint8_t* mask_ws;            // [vis_all]
+    int32_t* nout_ws;            // [max_batch][4]
+    int max_patch;
     unsigned step_parity;        // index of the scratch set of the current step
     // Scoring and selection of a step whose inputs are promised stable run on the side stream of the
     // step's scratch set, beside the selection and row copy of the steps before; the row copy stays
@@ -244,7 +252,7 @@ int32_t check_sticky(mvla_ctx* ctx)
 // fixed-point accumulators ctx->acc64 (*used_acc64 = true).
 int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, const void* k, int64_t rows,
                            const void* hidden, float* l1, unsigned long long* acc64, bool* used_acc64,
-                           bool free_running, cudaStream_t st)
+                           bool free_running, cudaStream_t st, AlphaOut alpha = AlphaOut{nullptr, 0, 0})
 {
     if (used_acc64) *used_acc64 = false;
     const mvla_config& c = ctx->cfg;
@@ -271,11 +279,11 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
     }
     if (fast) {
         e = launch_salience_fast(bd, c.n_heads, c.head_dim, tq, tk, tiles_per_cta, cluster, npad, ctx->part,
-                                 ctx->part_stride, acc64, ctx->status_dev, free_running, st);
+                                 ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, st);
         if (used_acc64) *used_acc64 = acc64 != nullptr;
     } else {
         e = launch_salience(bd, c.dtype, c.n_heads, c.head_dim, q, k, tq, tk, ctx->use_umma, tiles_per_cta,
-                            cluster, npad, ctx->part, ctx->part_stride, ctx->status_dev, st);
+                            cluster, npad, ctx->part, ctx->part_stride, ctx->status_dev, alpha, st);
     }
     if (e == cudaErrorInvalidConfiguration) return MVLA_ERR_UNSUPPORTED;
     if (e != cudaSuccess) return fail_cuda(ctx, e);
@@ -306,6 +314,123 @@ GateParams gate_params(const mvla_ctx* ctx, int32_t mode, bool has_l1)
     return gp;
 }
 
+// ---- patch-by-patch path ----
+int32_t validate_patch(const mvla_ctx* ctx, int32_t batch, const mvla_sample* samples)
+{
+    if (!ctx->cfg.patch_path) return MVLA_ERR_UNSUPPORTED;        // its state and scratch were not allocated
+    for (int b = 0; b < batch; ++b)
+        if (samples[b].n_2d != samples[b].n_3d || samples[b].n_2d < 1) return MVLA_ERR_INVALID_ARG;   // a patch owns one token of each
+    return MVLA_OK;
+}
+
+AlphaOut alpha_of(const mvla_ctx* ctx)
+{
+    return AlphaOut{ctx->alpha_ws, static_cast<int64_t>(ctx->cfg.max_text) * static_cast<int64_t>(ctx->vis_all),
+                    static_cast<int64_t>(ctx->vis_all)};
+}
+
+PatchParams patch_params(const mvla_ctx* ctx)
+{
+    const mvla_config& c = ctx->cfg;
+    PatchParams pp;
+    pp.tau_2d = c.tau_2d; pp.tau_3d = c.tau_3d; pp.eps_3d = c.eps_3d;
+    pp.obj_2d_min = c.obj_2d_min > 0.0 ? c.obj_2d_min : 0.5;
+    pp.bg_prune_prob = 1.0 - c.floor_ratio;
+    pp.kmeans_max_iter = c.kmeans_max_iter > 0 ? c.kmeans_max_iter : 32;
+    pp.cold_start_full_keep = c.cold_start_full_keep;
+    pp.max_patch = std::max(ctx->max_patch, 1);
+    return pp;
+}
+
+// Salience with the attention copy, feature norms, head sum, per-patch indicators.
+int32_t run_patch_indicators(mvla_ctx* ctx, const Plan& plan, int32_t batch, const void* q, const void* k,
+                             const void* hidden, int64_t rows, float* attn_out, float* x_out, cudaStream_t st)
+{
+    const AlphaOut alpha = alpha_of(ctx);
+    for (int first = 0; first < batch; first += kMaxChunk) {
+        const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
+        const int32_t rc = run_salience_chunk(ctx, bd, q, k, rows, hidden, ctx->l1_ws, nullptr, nullptr, false, st, alpha);
+        if (rc != MVLA_OK) return rc;
+    }
+    cudaError_t e = launch_head_reduce(ctx->part, ctx->part_stride, ctx->cfg.n_heads, plan.total_vis, attn_out, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    for (int first = 0; first < batch; first += kMaxChunk) {
+        const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
+        e = launch_patch_indicators(bd, ctx->cfg.n_heads, alpha, ctx->l1_ws, x_out, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
+    return MVLA_OK;
+}
+
+int32_t run_patch_select(mvla_ctx* ctx, const Plan& plan, int32_t batch, const float* attn, const float* x,
+                         const float* rand_u, int32_t* kept_idx, int32_t* out_offsets, int32_t* counts,
+                         float* xhat_out, int32_t* info_out, mvla_patch_diag* diag, cudaStream_t st)
+{
+    const PatchParams pp = patch_params(ctx);
+    PatchIO io;
+    std::memset(&io, 0, sizeof io);
+    io.attn = attn; io.x = x; io.rand_u = rand_u;
+    io.xhat_state = ctx->xhat_patch; io.xhat_out = xhat_out; io.info_out = info_out; io.diag = diag;
+    io.counts = counts; io.mask_ws = ctx->mask_ws; io.nout_ws = ctx->nout_ws;
+    io.kept_idx = kept_idx; io.out_offsets = out_offsets; io.batch_total = batch;
+    for (int pass = 0; pass < 2; ++pass)          // every sample's count is known before any list is placed
+        for (int first = 0; first < batch; first += kMaxChunk) {
+            const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
+            io.chunk_first = first;
+            const cudaError_t e = pass == 0 ? launch_patch_decide(bd, pp, io, st) : launch_patch_emit(bd, io, st);
+            if (e != cudaSuccess) return fail_cuda(ctx, e);
+        }
+    return MVLA_OK;
+}
+
+int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, uint32_t flags,
+                         const mvla_tensors* in, const mvla_outputs* out, int32_t* total_kept_out, void* stream)
+{
+    if (!in->hidden || !in->rand_u) return MVLA_ERR_INVALID_ARG;
+    if (flags & ~(MVLA_FLAG_RESET_STATE | MVLA_FLAG_NO_STATE_UPDATE | MVLA_FLAG_INPUTS_STABLE)) return MVLA_ERR_INVALID_ARG;
+    const void* src[3] = {in->hidden, in->k, in->v};
+    void* dst[3] = {out->out_hidden, out->out_k, out->out_v};
+    if (!aligned16(in->q) || !aligned16(out->patch_x) || !aligned16(out->patch_xhat)) return MVLA_ERR_INVALID_ARG;
+    for (int i = 0; i < 3; ++i) {
+        if (!aligned16(src[i]) || !aligned16(dst[i])) return MVLA_ERR_INVALID_ARG;
+        if (dst[i] && (!src[i] || src[i] == dst[i])) return MVLA_ERR_INVALID_ARG;
+    }
+    int32_t rc = check_sticky(ctx);
+    if (rc != MVLA_OK) return rc;
+    rc = validate_samples(ctx, batch, samples, MVLA_MODE_ADAPTIVE, in->rows);
+    if (rc != MVLA_OK) return rc;
+    rc = validate_patch(ctx, batch, samples);
+    if (rc != MVLA_OK) return rc;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return MVLA_ERR_CUDA;
+    ctx->hist_unknown = true;
+    Plan plan;
+    rc = make_plan(ctx, prune_point, batch, samples, MVLA_MODE_ADAPTIVE, flags, true, &plan);
+    if (rc != MVLA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* attn = out->attn ? out->attn : ctx->attn_ws;
+    float* x = out->patch_x ? out->patch_x : ctx->patch_x_ws;
+    rc = run_patch_indicators(ctx, plan, batch, in->q, in->k, in->hidden, in->rows, attn, x, st);
+    if (rc != MVLA_OK) return rc;
+    rc = run_patch_select(ctx, plan, batch, attn, x, in->rand_u, out->kept_idx, out->out_offsets, out->budgets,
+                          out->patch_xhat, out->patch_info, out->patch_diag, st);
+    if (rc != MVLA_OK) return rc;
+    int64_t cap = 0;                               // the row count is known only on the device: cover the capacity
+    for (int b = 0; b < batch; ++b) cap += samples[b].n_txt + samples[b].n_2d + samples[b].n_3d;
+    CompactJob job;
+    const int32_t kv_bytes = static_cast<int32_t>(ctx->cfg.n_heads * ctx->cfg.head_dim * ctx->elem);
+    for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
+    job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
+    for (int first = 0; first < batch; first += kMaxChunk) {
+        const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
+        const cudaError_t e = launch_compact(bd, job, out->kept_idx, static_cast<int32_t>(cap), 0, out->out_offsets, first, batch, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
+    commit_steps(ctx, prune_point, plan, samples);
+    if (total_kept_out) *total_kept_out = static_cast<int32_t>(cap);
+    return MVLA_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -323,6 +448,8 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
         return MVLA_ERR_INVALID_ARG;
     if (c.dtype != MVLA_DTYPE_BF16 && c.dtype != MVLA_DTYPE_FP32) return MVLA_ERR_UNSUPPORTED;
     if (c.salience_path != MVLA_SALIENCE_AUTO && c.salience_path != MVLA_SALIENCE_FMA) return MVLA_ERR_INVALID_ARG;
+    if ((c.patch_path != 0 && c.patch_path != 1) || c.kmeans_max_iter < 0 || !(c.obj_2d_min >= 0.0 && c.obj_2d_min <= 1.0))
+        return MVLA_ERR_INVALID_ARG;
     if (c.head_dim != 64 && c.head_dim != 128) return MVLA_ERR_UNSUPPORTED;
     if (c.max_text > kMaxText || c.max_2d + c.max_3d > kMaxVis || c.max_batch > 64) return MVLA_ERR_UNSUPPORTED;
     const size_t elem = c.dtype == MVLA_DTYPE_BF16 ? 2 : 4;
@@ -349,6 +476,10 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (c.salience_path == MVLA_SALIENCE_FMA) ctx->use_umma = false;
     ctx->part = ctx->attn_ws = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
     ctx->acc64 = nullptr;
+    ctx->alpha_ws = ctx->xhat_patch = ctx->patch_x_ws = nullptr;
+    ctx->mask_ws = nullptr;
+    ctx->nout_ws = nullptr;
+    ctx->max_patch = std::min(c.max_2d, c.max_3d);
     ctx->ev_fork = nullptr;
     for (int i = 0; i < kSets; ++i) {
         ctx->aux[i] = nullptr;
@@ -383,6 +514,13 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     alloc(&ctx->mhat_state, n_state * 4);
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->acc64), kSets * vis_all * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(ctx->acc64, 0, kSets * vis_all * sizeof(unsigned long long));
+    if (c.patch_path) {
+        alloc(&ctx->alpha_ws, static_cast<size_t>(c.n_heads) * c.max_text * vis_all);
+        alloc(&ctx->xhat_patch, n_state * std::max(ctx->max_patch, 1) * 4);
+        alloc(&ctx->patch_x_ws, (vis_all / 2 + 1) * 4);
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->mask_ws), vis_all);
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->nout_ws), static_cast<size_t>(c.max_batch) * 4 * sizeof(int32_t));
+    }
     for (cudaStream_t* sp = ctx->aux; sp != ctx->aux + kSets; ++sp)
         if (e == cudaSuccess) e = cudaStreamCreateWithFlags(sp, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
@@ -422,6 +560,11 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     cudaFree(ctx->ahat_state);
     cudaFree(ctx->mhat_state);
     cudaFree(ctx->acc64);
+    cudaFree(ctx->alpha_ws);
+    cudaFree(ctx->xhat_patch);
+    cudaFree(ctx->patch_x_ws);
+    cudaFree(ctx->mask_ws);
+    cudaFree(ctx->nout_ws);
     for (cudaStream_t sp : ctx->aux)
         if (sp) {
             cudaStreamSynchronize(sp);
@@ -534,12 +677,61 @@ int32_t mvla_compact(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, c
     return MVLA_OK;
 }
 
+int32_t mvla_patch_indicators(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const void* q, const void* k,
+                              const void* hidden, int64_t rows, float* attn_out, float* x_out, void* stream)
+{
+    if (!ctx || !q || !k || !hidden || !attn_out || !x_out || rows < 1) return MVLA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(hidden) || !aligned16(x_out)) return MVLA_ERR_INVALID_ARG;
+    int32_t rc = check_sticky(ctx);
+    if (rc != MVLA_OK) return rc;
+    rc = validate_samples(ctx, batch, samples, MVLA_MODE_FIXED, rows);
+    if (rc != MVLA_OK) return rc;
+    rc = validate_patch(ctx, batch, samples);
+    if (rc != MVLA_OK) return rc;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return MVLA_ERR_CUDA;
+    ctx->hist_unknown = true;
+    Plan plan;
+    rc = make_plan(ctx, 0, batch, samples, MVLA_MODE_FIXED, 0, false, &plan);
+    if (rc != MVLA_OK) return rc;
+    return run_patch_indicators(ctx, plan, batch, q, k, hidden, rows, attn_out, x_out, static_cast<cudaStream_t>(stream));
+}
+
+int32_t mvla_patch_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, uint32_t flags,
+                          const float* attn, const float* x, const float* rand_u, int32_t* kept_idx,
+                          int32_t* out_offsets, int32_t* counts, float* xhat_out, int32_t* info_out,
+                          mvla_patch_diag* diag, void* stream)
+{
+    if (!ctx || !attn || !x || !rand_u || !kept_idx || !out_offsets) return MVLA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(xhat_out)) return MVLA_ERR_INVALID_ARG;
+    if (flags & ~(MVLA_FLAG_RESET_STATE | MVLA_FLAG_NO_STATE_UPDATE)) return MVLA_ERR_INVALID_ARG;
+    int32_t rc = check_sticky(ctx);
+    if (rc != MVLA_OK) return rc;
+    rc = validate_samples(ctx, batch, samples, MVLA_MODE_ADAPTIVE, -1);
+    if (rc != MVLA_OK) return rc;
+    rc = validate_patch(ctx, batch, samples);
+    if (rc != MVLA_OK) return rc;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return MVLA_ERR_CUDA;
+    ctx->hist_unknown = true;
+    Plan plan;
+    rc = make_plan(ctx, prune_point, batch, samples, MVLA_MODE_ADAPTIVE, flags, true, &plan);
+    if (rc != MVLA_OK) return rc;
+    rc = run_patch_select(ctx, plan, batch, attn, x, rand_u, kept_idx, out_offsets, counts, xhat_out, info_out, diag,
+                          static_cast<cudaStream_t>(stream));
+    if (rc != MVLA_OK) return rc;
+    commit_steps(ctx, prune_point, plan, samples);
+    return MVLA_OK;
+}
+
 int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples,
                         int32_t mode, uint32_t flags, const mvla_tensors* in, const mvla_outputs* out,
                         int32_t* total_kept_out, void* stream)
 {
     if (!ctx || !in || !out || !in->q || !in->k || !out->kept_idx || !out->out_offsets || in->rows < 1)
         return MVLA_ERR_INVALID_ARG;
+    if (mode == MVLA_MODE_PATCH)
+        return prune_step_patch(ctx, prune_point, batch, samples, flags, in, out, total_kept_out, stream);
     if (flags & ~(MVLA_FLAG_RESET_STATE | MVLA_FLAG_NO_STATE_UPDATE | MVLA_FLAG_INPUTS_STABLE)) return MVLA_ERR_INVALID_ARG;
     if (mode == MVLA_MODE_ADAPTIVE && !in->hidden) return MVLA_ERR_INVALID_ARG;
     const void* src[3] = {in->hidden, in->k, in->v};

@@ -85,11 +85,18 @@ inline cudaLaunchAttribute pdl_attribute()
 // per visual token, zero on entry); without it they go to part[h][vis] as in launch_salience.
 // `free_running`: the kernel does not wait for the kernel before it in its stream (the caller orders
 // everything it depends on with events).
+// Optional copy of the attention itself for the patch-by-patch path:
+// ptr[(h * stride_h) + (i * stride_i) + vis_off + j] = alpha[h, i, j]   (null: not written).
+struct AlphaOut {
+    float* ptr;
+    int64_t stride_h, stride_i;
+};
+
 bool fast_salience_supported(int tiles_per_cta);
 cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int head_dim, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
-                                 bool free_running, cudaStream_t stream);
+                                 bool free_running, AlphaOut alpha, cudaStream_t stream);
 
 
 // Salience: per-head partial scores part[h][vis] (already scaled by 1/(H n_t)).
@@ -98,7 +105,7 @@ cudaError_t launch_salience(const BatchDesc& bd, int dtype, int n_heads, int hea
                             const void* q, const void* k, const CUtensorMap* tmap_q,
                             const CUtensorMap* tmap_k, bool use_umma, int tiles_per_cta,
                             int cluster, int npad, float* part, int64_t part_stride,
-                            int* status, cudaStream_t stream);
+                            int* status, AlphaOut alpha, cudaStream_t stream);
 
 // attn[j] = sum_h part[h][j]  (fixed head order).
 cudaError_t launch_head_reduce(const float* part, int64_t part_stride, int n_heads, int total_vis,
@@ -123,5 +130,35 @@ struct CompactJob {
 cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int32_t* kept_idx,
                            int32_t chunk_rows, int32_t chunk_row0, const int32_t* out_offsets,
                            int32_t chunk_first, int32_t batch_total, cudaStream_t stream);
+
+// ---- patch-by-patch path (Alg. 1 taken literally) ----
+struct PatchParams {
+    double tau_2d, tau_3d, eps_3d, obj_2d_min, bg_prune_prob;
+    int32_t kmeans_max_iter;
+    int32_t cold_start_full_keep;
+    int32_t max_patch;       // stride (in patches) of one (prune point, slot) in the per-patch state
+};
+struct PatchIO {
+    const float* attn;       // [sum 2P] per-token scores
+    const float* x;          // [sum P][4] instantaneous indicators
+    const float* rand_u;     // [sum P]
+    float* xhat_state;       // [points * slots][max_patch][4]
+    float* xhat_out;         // nullable
+    int32_t* info_out;       // nullable
+    mvla_patch_diag* diag;   // nullable
+    int32_t* counts;         // [batch][2] nullable
+    uint8_t* mask_ws;        // [sum 2P] keep flags in visual order (scratch between the two kernels)
+    int32_t* nout_ws;        // [batch] kept rows per sample (scratch)
+    int32_t* kept_idx;
+    int32_t* out_offsets;
+    int32_t chunk_first, batch_total;
+};
+// x[p] = per-patch indicators from the attention copy and the feature norms.
+cudaError_t launch_patch_indicators(const BatchDesc& bd, int n_heads, AlphaOut alpha, const float* l1,
+                                    float* x_out, cudaStream_t stream);
+// Stages 1-4 of Alg. 1 for every patch; leaves keep flags and row counts in the scratch of `io`.
+cudaError_t launch_patch_decide(const BatchDesc& bd, const PatchParams& pp, const PatchIO& io, cudaStream_t stream);
+// Offsets over the whole batch and the ordered kept-position lists.
+cudaError_t launch_patch_emit(const BatchDesc& bd, const PatchIO& io, cudaStream_t stream);
 
 }  // namespace mvla

@@ -52,6 +52,7 @@ compact_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ Com
     // which sample owns output row `orow` (samples are few: linear scan)
     int b = 0;
     if (out_offsets) {            // offsets known only on the device: scan the whole batch
+        if (orow >= out_offsets[batch_total]) return;      // the launch covered a capacity bound, not the row count
         while (b + 1 < batch_total && orow >= out_offsets[b + 1]) ++b;
         b -= chunk_first;
         if (b < 0 || b >= bd.n) return;      // row belongs to another launch's samples

@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(kFastThreads, 1)
 salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
                      const __grid_constant__ CUtensorMap tmap_k, int n_heads, int head_dim, int npad,
                      float* __restrict__ part, int64_t part_stride, unsigned long long* __restrict__ acc64,
-                     int* status, int free_running)
+                     int* status, int free_running, const AlphaOut alpha)
 {
     constexpr int CC = TCOL * NTILE;
     extern __shared__ uint8_t dyn_smem_raw[];
@@ -269,6 +269,13 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
                 atomicAdd(acc64 + s.vis_off + vis0[t] + tid, __float2ull_rn(acc * kFixScale));
             else
                 part[static_cast<int64_t>(h) * part_stride + s.vis_off + vis0[t] + tid] = acc;
+            if (alpha.ptr) {              // the attention itself, for the per-patch indicators (coalesced over keys)
+                float* ap = alpha.ptr + static_cast<int64_t>(h) * alpha.stride_h + s.vis_off + vis0[t] + tid;
+                const float hn = static_cast<float>(n_heads) * static_cast<float>(s.n_txt);   // s_w carries 1 / (H n_t)
+#pragma unroll
+                for (int i = 0; i < TCOL; ++i)
+                    if (i < s.n_txt) ap[static_cast<int64_t>(i) * alpha.stride_i] = L[t * TCOL + i] * s_w[i] * hn;
+            }
         }
     }
 
@@ -280,7 +287,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
 template <int TCOL, int NTILE>
 cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int head_dim, const CUtensorMap* tq,
                           const CUtensorMap* tk, int cluster, int npad, float* part, int64_t part_stride,
-                          unsigned long long* acc64, int* status, int free_running, cudaStream_t stream)
+                          unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, cudaStream_t stream)
 {
     const size_t smem = 1024 + static_cast<size_t>(head_dim / 64) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
     auto kern = salience_fast_kernel<TCOL, NTILE>;
@@ -299,7 +306,7 @@ cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int head_dim, const 
     attr[1] = pdl_attribute();
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, head_dim, npad, part, part_stride, acc64, status, free_running);
+    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, head_dim, npad, part, part_stride, acc64, status, free_running, alpha);
 }
 
 }  // namespace
@@ -309,13 +316,13 @@ bool fast_salience_supported(int tiles_per_cta) { return tiles_per_cta >= 1 && t
 cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int head_dim, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
-                                 bool free_running, cudaStream_t stream)
+                                 bool free_running, AlphaOut alpha, cudaStream_t stream)
 {
     const int tcol = npad <= 16 ? 16 : (npad <= 32 ? 32 : 64);
 #define MVLA_FAST(TC, NTL)                                                                                      \
     if (tcol == TC && tiles_per_cta == NTL)                                                                     \
         return launch_fast_t<TC, NTL>(bd, n_heads, head_dim, tmap_q, tmap_k, cluster, npad, part, part_stride, \
-                                      acc64, status, free_running ? 1 : 0, stream);
+                                      acc64, status, free_running ? 1 : 0, alpha, stream);
     MVLA_FAST(16, 1) MVLA_FAST(32, 1) MVLA_FAST(64, 1) MVLA_FAST(16, 2) MVLA_FAST(32, 2) MVLA_FAST(64, 2)
 #undef MVLA_FAST
     return cudaErrorInvalidConfiguration;

@@ -26,7 +26,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
                 const __grid_constant__ CUtensorMap tmap_k, const T* __restrict__ q,
                 const T* __restrict__ k, int n_heads, int head_dim, int tiles_per_cta, int npad,
-                float* __restrict__ part, int64_t part_stride, int* status)
+                float* __restrict__ part, int64_t part_stride, int* status, const AlphaOut alpha)
 {
     extern __shared__ uint8_t dyn_smem_raw[];
     uint8_t* dyn_smem = dyn_smem_raw + ((1024u - (smem_u32(dyn_smem_raw) & 1023u)) & 1023u);   // swizzle atoms are 1 KB
@@ -256,7 +256,11 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const float e = exp2f(v[i] - s_m[cb + i]);
-                    acc += (cb + i < s.n_txt) ? e * s_w[cb + i] : 0.f;
+                    const float pr = (cb + i < s.n_txt) ? e * s_w[cb + i] : 0.f;
+                    acc += pr;
+                    if (alpha.ptr && cb + i < s.n_txt && tid < ti.valid)   // the attention itself (per-patch indicators)
+                        alpha.ptr[static_cast<int64_t>(h) * alpha.stride_h + static_cast<int64_t>(cb + i) * alpha.stride_i +
+                                  s.vis_off + ti.vis0 + tid] = pr * (static_cast<float>(n_heads) * static_cast<float>(s.n_txt));
                 }
             }
         }
@@ -321,7 +325,8 @@ l1norm_kernel(const __grid_constant__ BatchDesc bd, int d_model, const T* __rest
 template <typename T, bool UMMA>
 cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int head_dim, const void* q, const void* k,
                               const CUtensorMap* tq, const CUtensorMap* tk, int tiles_per_cta, int cluster,
-                              int npad, float* part, int64_t part_stride, int* status, cudaStream_t stream)
+                              int npad, float* part, int64_t part_stride, int* status, AlphaOut alpha,
+                              cudaStream_t stream)
 {
     size_t smem;
     if (UMMA)
@@ -348,7 +353,7 @@ cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int head_dim, co
     static const CUtensorMap zero_map = {};
     return cudaLaunchKernelEx(&cfg, kern, bd, tq ? *tq : zero_map, tk ? *tk : zero_map,
                               static_cast<const T*>(q), static_cast<const T*>(k), n_heads, head_dim,
-                              tiles_per_cta, npad, part, part_stride, status);
+                              tiles_per_cta, npad, part, part_stride, status, alpha);
 }
 
 }  // namespace
@@ -356,17 +361,17 @@ cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int head_dim, co
 cudaError_t launch_salience(const BatchDesc& bd, int dtype, int n_heads, int head_dim, const void* q,
                             const void* k, const CUtensorMap* tmap_q, const CUtensorMap* tmap_k,
                             bool use_umma, int tiles_per_cta, int cluster, int npad, float* part,
-                            int64_t part_stride, int* status, cudaStream_t stream)
+                            int64_t part_stride, int* status, AlphaOut alpha, cudaStream_t stream)
 {
     if (dtype == MVLA_DTYPE_BF16) {
         if (use_umma)
             return launch_salience_t<__nv_bfloat16, true>(bd, n_heads, head_dim, q, k, tmap_q, tmap_k, tiles_per_cta,
-                                                          cluster, npad, part, part_stride, status, stream);
+                                                          cluster, npad, part, part_stride, status, alpha, stream);
         return launch_salience_t<__nv_bfloat16, false>(bd, n_heads, head_dim, q, k, nullptr, nullptr, tiles_per_cta,
-                                                       cluster, npad, part, part_stride, status, stream);
+                                                       cluster, npad, part, part_stride, status, alpha, stream);
     }
     return launch_salience_t<float, false>(bd, n_heads, head_dim, q, k, nullptr, nullptr, tiles_per_cta, cluster,
-                                           npad, part, part_stride, status, stream);
+                                           npad, part, part_stride, status, alpha, stream);
 }
 
 cudaError_t launch_head_reduce(const float* part, int64_t part_stride, int n_heads, int total_vis, float* attn,

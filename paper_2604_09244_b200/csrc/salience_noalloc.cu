@@ -154,7 +154,7 @@ extern "C" int32_t mvla_salience_noalloc(int32_t device, int32_t dtype, int32_t 
             const int npad = (max_txt + 15) / 16 * 16;
             const cudaError_t e = launch_salience(bd, dtype, n_heads, head_dim, q, k, umma ? &tq : nullptr,
                                                   umma ? &tk : nullptr, umma, tiles_per_cta, cluster, npad, sc->part,
-                                                  total_vis, sc->flag, st);
+                                                  total_vis, sc->flag, AlphaOut{nullptr, 0, 0}, st);
             if (e == cudaErrorInvalidConfiguration) rc = MVLA_ERR_UNSUPPORTED;
             else if (e != cudaSuccess) rc = MVLA_ERR_CUDA;
         }

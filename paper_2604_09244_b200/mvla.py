@@ -23,13 +23,15 @@ _ERR_NAMES = {-1: "MVLA_ERR_INVALID_ARG", -2: "MVLA_ERR_UNSUPPORTED", -3: "MVLA_
               -4: "MVLA_ERR_CUDA", -5: "MVLA_ERR_CAPACITY", -6: "MVLA_ERR_TIMEOUT",
               -7: "MVLA_ERR_STATE"}
 DTYPE_BF16, DTYPE_FP32 = 0, 1
-MODE_FIXED, MODE_ADAPTIVE = 0, 1
+MODE_FIXED, MODE_ADAPTIVE, MODE_PATCH = 0, 1, 2
+LABEL_BG, LABEL_ROB, LABEL_OBJ = 0, 1, 2
 FLAG_RESET_STATE, FLAG_NO_STATE_UPDATE, FLAG_INPUTS_STABLE = 1, 2, 4
 SALIENCE_AUTO, SALIENCE_FMA = 0, 1
 SET_2D, SET_3D = 1, 2
 
 EXPORTS = ("mvla_prune_create", "mvla_salience", "mvla_select", "mvla_compact",
-           "mvla_prune_step", "mvla_prune_destroy")
+           "mvla_prune_step", "mvla_prune_destroy", "mvla_patch_indicators", "mvla_patch_select",
+           "mvla_salience_noalloc")
 
 
 class MvlaError(RuntimeError):
@@ -46,7 +48,8 @@ class Config(C.Structure):
                 ("window_k", C.c_int32), ("cold_start_full_keep", C.c_int32),
                 ("salience_path", C.c_int32),
                 ("tau_2d", C.c_double), ("tau_3d", C.c_double), ("beta", C.c_double),
-                ("eps_3d", C.c_double), ("floor_ratio", C.c_double)]
+                ("eps_3d", C.c_double), ("floor_ratio", C.c_double), ("obj_2d_min", C.c_double),
+                ("patch_path", C.c_int32), ("kmeans_max_iter", C.c_int32)]
 
 
 class CSample(C.Structure):
@@ -64,13 +67,21 @@ class CDiag(C.Structure):
 
 class CTensors(C.Structure):
     _fields_ = [("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("hidden", C.c_void_p),
-                ("rows", C.c_int64)]
+                ("rows", C.c_int64), ("rand_u", C.c_void_p)]
 
 
 class COutputs(C.Structure):
     _fields_ = [("out_hidden", C.c_void_p), ("out_k", C.c_void_p), ("out_v", C.c_void_p),
                 ("kept_idx", C.c_void_p), ("out_offsets", C.c_void_p), ("budgets", C.c_void_p),
-                ("attn", C.c_void_p), ("ahat", C.c_void_p), ("z", C.c_void_p), ("diag", C.c_void_p)]
+                ("attn", C.c_void_p), ("ahat", C.c_void_p), ("z", C.c_void_p), ("diag", C.c_void_p),
+                ("patch_x", C.c_void_p), ("patch_xhat", C.c_void_p), ("patch_info", C.c_void_p),
+                ("patch_diag", C.c_void_p)]
+
+
+class CPatchDiag(C.Structure):
+    _fields_ = [("t", C.c_int32), ("iters", C.c_int32), ("n_label", C.c_int32 * 3), ("k_2d", C.c_int32),
+                ("k_3d", C.c_int32), ("n_out", C.c_int32), ("centre", C.c_float * 3), ("mu_2d", C.c_float),
+                ("mu_3d", C.c_float), ("reserved", C.c_float * 3)]
 
 
 def load_library(path: str = LIB_PATH) -> C.CDLL:
@@ -93,6 +104,10 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.mvla_prune_step.restype = i32
     lib.mvla_prune_destroy.argtypes = [vp]
     lib.mvla_prune_destroy.restype = None
+    lib.mvla_patch_indicators.argtypes = [vp, i32, sp, vp, vp, vp, i64, vp, vp, vp]
+    lib.mvla_patch_indicators.restype = i32
+    lib.mvla_patch_select.argtypes = [vp, i32, i32, sp, u32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.mvla_patch_select.restype = i32
     return lib
 
 
@@ -141,6 +156,11 @@ class StepOutputs:
     z: Optional[torch.Tensor] = None
     diag: Optional[torch.Tensor] = None   # int32 view of mvla_diag records, [batch, 16]
     total_kept: int = 0
+    # patch-by-patch path
+    patch_x: Optional[torch.Tensor] = None      # [sum P, 4]
+    patch_xhat: Optional[torch.Tensor] = None   # [sum P, 4]
+    patch_info: Optional[torch.Tensor] = None   # [sum P] int32
+    patch_diag: Optional[torch.Tensor] = None   # int32 view of mvla_patch_diag records, [batch, 16]
 
 
 class PruneContext:
@@ -151,7 +171,8 @@ class PruneContext:
                  n_state_slots: int = 0, tau_2d: float = 0.08, tau_3d: float = 0.20,
                  beta: float = 0.85, window_k: int = 7, eps_3d: float = 0.02,
                  floor_ratio: float = 0.10, cold_start_full_keep: int = 1,
-                 salience_path: int = SALIENCE_AUTO, device: Optional[int] = None):
+                 salience_path: int = SALIENCE_AUTO, device: Optional[int] = None, patch_path: int = 0,
+                 obj_2d_min: float = 0.5, kmeans_max_iter: int = 32):
         self._h = C.c_void_p()
         self._lib = lib()
         if device is None:
@@ -161,7 +182,8 @@ class PruneContext:
         code = {torch.bfloat16: DTYPE_BF16, torch.float32: DTYPE_FP32}[dtype]
         self.cfg = Config(device, code, n_heads, head_dim, d_model, max_batch, max_text, max_2d,
                           max_3d, n_prune_points, n_state_slots, window_k, cold_start_full_keep,
-                          salience_path, tau_2d, tau_3d, beta, eps_3d, floor_ratio)
+                          salience_path, tau_2d, tau_3d, beta, eps_3d, floor_ratio, obj_2d_min, patch_path,
+                          kmeans_max_iter)
         rc = self._lib.mvla_prune_create(C.byref(self.cfg), C.byref(self._h))
         if rc != OK:
             self._h = C.c_void_p()
@@ -180,9 +202,10 @@ class PruneContext:
             pass
 
     # -- allocation helpers (shapes only) ---------------------------------
-    def alloc_outputs(self, samples: Sequence, *, hidden=True, kv=True, extras=False) -> StepOutputs:
+    def alloc_outputs(self, samples: Sequence, *, hidden=True, kv=True, extras=False, patch=False) -> StepOutputs:
         rows = sum(s.n_txt + s.n_2d + s.n_3d for s in samples)
         nvis = sum(s.n_2d + s.n_3d for s in samples)
+        npat = sum(s.n_2d for s in samples)
         c, dev, dt = self.cfg, self.device, self.torch_dtype
         mk = lambda *shape, dtype=dt: torch.empty(*shape, dtype=dtype, device=dev)
         return StepOutputs(
@@ -195,7 +218,11 @@ class PruneContext:
             attn=mk(nvis, dtype=torch.float32) if extras else None,
             ahat=mk(nvis, dtype=torch.float32) if extras else None,
             z=mk(nvis, dtype=torch.float32) if extras else None,
-            diag=torch.zeros(len(samples), 16, dtype=torch.int32, device=dev) if extras else None)
+            diag=torch.zeros(len(samples), 16, dtype=torch.int32, device=dev) if extras else None,
+            patch_x=mk(npat, 4, dtype=torch.float32) if patch else None,
+            patch_xhat=mk(npat, 4, dtype=torch.float32) if patch else None,
+            patch_info=mk(npat, dtype=torch.int32) if patch else None,
+            patch_diag=torch.zeros(len(samples), 16, dtype=torch.int32, device=dev) if patch else None)
 
     # -- the six entry points ----------------------------------------------
     def salience(self, samples, q, k, hidden=None, *, attn_out=None, l1_out=None, stream=None):
@@ -238,15 +265,45 @@ class PruneContext:
             raise MvlaError(rc, "mvla_compact")
         return out_hidden, out_k, out_v
 
-    def prune_step(self, prune_point, samples, mode, q, k, v, hidden, *, flags=0,
-                   out: StepOutputs = None, stream=None) -> StepOutputs:
+    def patch_indicators(self, samples, q, k, hidden, *, attn_out=None, x_out=None, stream=None):
+        """Per-token scores and the four per-patch indicators (``mvla_patch_indicators``)."""
+        cs = samples if isinstance(samples, C.Array) else c_samples(samples)
+        nvis = sum(s.n_2d + s.n_3d for s in cs)
+        if attn_out is None:
+            attn_out = torch.empty(nvis, dtype=torch.float32, device=self.device)
+        if x_out is None:
+            x_out = torch.empty(nvis // 2, 4, dtype=torch.float32, device=self.device)
+        rc = self._lib.mvla_patch_indicators(self._h, len(cs), cs, _ptr(q), _ptr(k), _ptr(hidden), q.shape[0],
+                                             _ptr(attn_out), _ptr(x_out), _stream(stream))
+        if rc != OK:
+            raise MvlaError(rc, "mvla_patch_indicators")
+        return attn_out, x_out
+
+    def patch_select(self, prune_point, samples, attn, x, rand_u, *, flags=0, out: StepOutputs = None,
+                     stream=None) -> StepOutputs:
+        """Alg. 1 stages 1-4 patch by patch (``mvla_patch_select``); kept counts land in ``out.budgets``."""
         cs = samples if isinstance(samples, C.Array) else c_samples(samples)
         if out is None:
-            out = self.alloc_outputs(cs, hidden=hidden is not None, kv=v is not None, extras=True)
-        tin = CTensors(_ptr(q), _ptr(k), _ptr(v), _ptr(hidden), q.shape[0])
+            out = self.alloc_outputs(cs, hidden=False, kv=False, patch=True)
+        rc = self._lib.mvla_patch_select(self._h, prune_point, len(cs), cs, flags, _ptr(attn), _ptr(x), _ptr(rand_u),
+                                         _ptr(out.kept_idx), _ptr(out.out_offsets), _ptr(out.budgets),
+                                         _ptr(out.patch_xhat), _ptr(out.patch_info), _ptr(out.patch_diag),
+                                         _stream(stream))
+        if rc != OK:
+            raise MvlaError(rc, "mvla_patch_select")
+        return out
+
+    def prune_step(self, prune_point, samples, mode, q, k, v, hidden, *, flags=0,
+                   out: StepOutputs = None, stream=None, rand_u=None) -> StepOutputs:
+        cs = samples if isinstance(samples, C.Array) else c_samples(samples)
+        if out is None:
+            out = self.alloc_outputs(cs, hidden=hidden is not None, kv=v is not None, extras=True,
+                                     patch=mode == MODE_PATCH)
+        tin = CTensors(_ptr(q), _ptr(k), _ptr(v), _ptr(hidden), q.shape[0], _ptr(rand_u))
         tout = COutputs(_ptr(out.out_hidden), _ptr(out.out_k), _ptr(out.out_v), _ptr(out.kept_idx),
                         _ptr(out.out_offsets), _ptr(out.budgets), _ptr(out.attn), _ptr(out.ahat),
-                        _ptr(out.z), _ptr(out.diag))
+                        _ptr(out.z), _ptr(out.diag), _ptr(out.patch_x), _ptr(out.patch_xhat),
+                        _ptr(out.patch_info), _ptr(out.patch_diag))
         total = C.c_int32(0)
         rc = self._lib.mvla_prune_step(self._h, prune_point, len(cs), cs, mode, flags, C.byref(tin),
                                        C.byref(tout), C.byref(total), _stream(stream))
@@ -257,7 +314,7 @@ class PruneContext:
 
 
 def context_for(wl, *, max_batch=None, n_prune_points=1, n_state_slots=0, salience_path=SALIENCE_AUTO,
-                device=None) -> PruneContext:
+                device=None, patch_path=None) -> PruneContext:
     """A context sized for a synthetic workload (see ``workloads``)."""
     dt = {"bf16": torch.bfloat16, "fp32": torch.float32}[wl.dtype]
     return PruneContext(dtype=dt, n_heads=wl.n_heads, head_dim=wl.head_dim, d_model=wl.d_model,
@@ -268,7 +325,10 @@ def context_for(wl, *, max_batch=None, n_prune_points=1, n_state_slots=0, salien
                         n_prune_points=n_prune_points, n_state_slots=n_state_slots, tau_2d=wl.tau_2d, tau_3d=wl.tau_3d,
                         beta=wl.beta, window_k=wl.window_k, eps_3d=wl.eps_3d,
                         floor_ratio=wl.floor_ratio, cold_start_full_keep=wl.cold_start_full_keep,
-                        salience_path=salience_path, device=device)
+                        salience_path=salience_path, device=device,
+                        patch_path=int(wl.mode == MODE_PATCH) if patch_path is None else patch_path,
+                        obj_2d_min=wl.extra.get("obj_2d_min", 0.5),
+                        kmeans_max_iter=wl.extra.get("kmeans_max_iter", 32))
 
 
 def to_device(arr, dtype: str, device) -> torch.Tensor:

@@ -26,11 +26,12 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_struct_sizes_match_the_header_layout():
-    assert C.sizeof(mvla.Config) == 14 * 4 + 5 * 8
+    assert C.sizeof(mvla.Config) == 14 * 4 + 6 * 8 + 2 * 4
     assert C.sizeof(mvla.CSample) == 8 * 4 + 3 * 8
     assert C.sizeof(mvla.CDiag) == 64
-    assert C.sizeof(mvla.CTensors) == 5 * 8
-    assert C.sizeof(mvla.COutputs) == 10 * 8
+    assert C.sizeof(mvla.CTensors) == 6 * 8
+    assert C.sizeof(mvla.COutputs) == 14 * 8
+    assert C.sizeof(mvla.CPatchDiag) == 64
 
 
 def test_bad_arguments_are_error_codes(lib):
@@ -51,6 +52,8 @@ def test_bad_arguments_are_error_codes(lib):
     assert lib.mvla_select(None, 0, 1, None, 0, 0, None, None, None, None, None, None, None, None, None) == mvla.ERR_INVALID_ARG
     assert lib.mvla_compact(None, 1, None, None, None, 0, None, None, None, None, None, None, None) == mvla.ERR_INVALID_ARG
     assert lib.mvla_prune_step(None, 0, 1, None, 0, 0, None, None, None, None) == mvla.ERR_INVALID_ARG
+    assert lib.mvla_patch_indicators(None, 1, None, None, None, None, 1, None, None, None) == mvla.ERR_INVALID_ARG
+    assert lib.mvla_patch_select(None, 0, 1, None, 0, None, None, None, None, None, None, None, None, None, None) == mvla.ERR_INVALID_ARG
     lib.mvla_prune_destroy(None)           # accepted
 
 
