@@ -232,8 +232,8 @@ def run_ours(args, rank, local, world):
     torch.cuda.synchronize()
     # the patch-by-patch path decides its row count on the device (total_kept is then the capacity bound)
     kept_rows = int(o0.out_offsets[-1]) if is_patch else o0.total_kept
-    # patch path: norms, scoring, head sum, indicators, decide, emit, row copy
-    launches_per_step = 7 if is_patch else 3 + (1 if wl.mode == 1 else 0)
+    # patch path: norms, scoring, indicators, select, row copy
+    launches_per_step = 5 if is_patch else 3 + (1 if wl.mode == 1 else 0)
 
     # ---- device-resident timing: CUDA graphs of back-to-back steps over the rotating sets
     per_graph = -(-200 // n_sets) * n_sets   # ~200 steps per graph: the pipeline of overlapping steps fills once per replay

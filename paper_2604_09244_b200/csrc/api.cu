@@ -35,8 +35,7 @@ struct mvla_ctx {
     float* alpha_ws;
     float* xhat_patch;
     float* patch_x_ws;           // [vis_all / 2][4]
-    uint8_t* mask_ws;            // [vis_all]
-    int32_t* nout_ws;            // [max_batch][4]
+    int32_t* nout_ws;            // [max_batch] kept rows, [max_batch] ready flags, [1] finished-CTA counter
     int max_patch;
     unsigned step_parity;        // index of the scratch set of the current step
     // Scoring and selection of a step whose inputs are promised stable run on the side stream of the
@@ -352,11 +351,9 @@ int32_t run_patch_indicators(mvla_ctx* ctx, const Plan& plan, int32_t batch, con
         const int32_t rc = run_salience_chunk(ctx, bd, q, k, rows, hidden, ctx->l1_ws, nullptr, nullptr, false, st, alpha);
         if (rc != MVLA_OK) return rc;
     }
-    cudaError_t e = launch_head_reduce(ctx->part, ctx->part_stride, ctx->cfg.n_heads, plan.total_vis, attn_out, st);
-    if (e != cudaSuccess) return fail_cuda(ctx, e);
     for (int first = 0; first < batch; first += kMaxChunk) {
         const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
-        e = launch_patch_indicators(bd, ctx->cfg.n_heads, alpha, ctx->l1_ws, x_out, st);
+        const cudaError_t e = launch_patch_indicators(bd, ctx->cfg.n_heads, alpha, ctx->l1_ws, x_out, attn_out, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
     return MVLA_OK;
@@ -371,15 +368,15 @@ int32_t run_patch_select(mvla_ctx* ctx, const Plan& plan, int32_t batch, const f
     std::memset(&io, 0, sizeof io);
     io.attn = attn; io.x = x; io.rand_u = rand_u;
     io.xhat_state = ctx->xhat_patch; io.xhat_out = xhat_out; io.info_out = info_out; io.diag = diag;
-    io.counts = counts; io.mask_ws = ctx->mask_ws; io.nout_ws = ctx->nout_ws;
+    io.counts = counts; io.nout_ws = ctx->nout_ws; io.ready_ws = ctx->nout_ws + ctx->cfg.max_batch;
+    io.done_ws = ctx->nout_ws + 2 * ctx->cfg.max_batch; io.status = ctx->status_dev;
     io.kept_idx = kept_idx; io.out_offsets = out_offsets; io.batch_total = batch;
-    for (int pass = 0; pass < 2; ++pass)          // every sample's count is known before any list is placed
-        for (int first = 0; first < batch; first += kMaxChunk) {
-            const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
-            io.chunk_first = first;
-            const cudaError_t e = pass == 0 ? launch_patch_decide(bd, pp, io, st) : launch_patch_emit(bd, io, st);
-            if (e != cudaSuccess) return fail_cuda(ctx, e);
-        }
+    for (int first = 0; first < batch; first += kMaxChunk) {
+        const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
+        io.chunk_first = first;
+        const cudaError_t e = launch_patch_select(bd, pp, io, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
     return MVLA_OK;
 }
 
@@ -477,7 +474,6 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     ctx->part = ctx->attn_ws = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
     ctx->acc64 = nullptr;
     ctx->alpha_ws = ctx->xhat_patch = ctx->patch_x_ws = nullptr;
-    ctx->mask_ws = nullptr;
     ctx->nout_ws = nullptr;
     ctx->max_patch = std::min(c.max_2d, c.max_3d);
     ctx->ev_fork = nullptr;
@@ -518,8 +514,9 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
         alloc(&ctx->alpha_ws, static_cast<size_t>(c.n_heads) * c.max_text * vis_all);
         alloc(&ctx->xhat_patch, n_state * std::max(ctx->max_patch, 1) * 4);
         alloc(&ctx->patch_x_ws, (vis_all / 2 + 1) * 4);
-        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->mask_ws), vis_all);
-        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->nout_ws), static_cast<size_t>(c.max_batch) * 4 * sizeof(int32_t));
+        const size_t nws = (2 * static_cast<size_t>(c.max_batch) + 1) * sizeof(int32_t);
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->nout_ws), nws);
+        if (e == cudaSuccess) e = cudaMemset(ctx->nout_ws, 0, nws);
     }
     for (cudaStream_t* sp = ctx->aux; sp != ctx->aux + kSets; ++sp)
         if (e == cudaSuccess) e = cudaStreamCreateWithFlags(sp, cudaStreamNonBlocking);
@@ -563,7 +560,6 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     cudaFree(ctx->alpha_ws);
     cudaFree(ctx->xhat_patch);
     cudaFree(ctx->patch_x_ws);
-    cudaFree(ctx->mask_ws);
     cudaFree(ctx->nout_ws);
     for (cudaStream_t sp : ctx->aux)
         if (sp) {

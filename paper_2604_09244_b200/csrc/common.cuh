@@ -147,18 +147,18 @@ struct PatchIO {
     int32_t* info_out;       // nullable
     mvla_patch_diag* diag;   // nullable
     int32_t* counts;         // [batch][2] nullable
-    uint8_t* mask_ws;        // [sum 2P] keep flags in visual order (scratch between the two kernels)
     int32_t* nout_ws;        // [batch] kept rows per sample (scratch)
+    int32_t* ready_ws;       // [batch] "count published" flags, zero between launches
+    int32_t* done_ws;        // CTAs of the launch that have finished waiting, zero between launches
+    int* status;             // word that receives MVLA_ERR_TIMEOUT when a bounded wait gives up
     int32_t* kept_idx;
     int32_t* out_offsets;
     int32_t chunk_first, batch_total;
 };
-// x[p] = per-patch indicators from the attention copy and the feature norms.
+// x[p] = per-patch indicators from the attention copy and the feature norms; attn = per-token scores.
 cudaError_t launch_patch_indicators(const BatchDesc& bd, int n_heads, AlphaOut alpha, const float* l1,
-                                    float* x_out, cudaStream_t stream);
-// Stages 1-4 of Alg. 1 for every patch; leaves keep flags and row counts in the scratch of `io`.
-cudaError_t launch_patch_decide(const BatchDesc& bd, const PatchParams& pp, const PatchIO& io, cudaStream_t stream);
-// Offsets over the whole batch and the ordered kept-position lists.
-cudaError_t launch_patch_emit(const BatchDesc& bd, const PatchIO& io, cudaStream_t stream);
+                                    float* x_out, float* attn_out, cudaStream_t stream);
+// Stages 1-4 of Alg. 1 for every patch, output offsets over the batch, ordered kept-position lists.
+cudaError_t launch_patch_select(const BatchDesc& bd, const PatchParams& pp, const PatchIO& io, cudaStream_t stream);
 
 }  // namespace mvla

@@ -3,9 +3,9 @@
 //
 //   patch_indicators_kernel : the four indicators of every patch from the attention copy that the
 //                             salience kernel leaves behind (Eq. 3-1, Eq. 3-4, Eq. P2D, Eq. P3D);
-//   patch_decide_kernel     : temporal predictor (Eqs. 8, 9), dual threshold (Sec. 4.1), 1-D K-Means and
-//                             the semantic rules (Sec. 4.2), fusion (Sec. 4.4) -> keep flags and counts;
-//   patch_emit_kernel       : output offsets over the batch and the ordered kept-position lists (Eq. 10).
+//   patch_select_kernel     : temporal predictor (Eqs. 8, 9), dual threshold (Sec. 4.1), 1-D K-Means and
+//                             the semantic rules (Sec. 4.2), fusion (Sec. 4.4), then the output offsets
+//                             over the batch and the ordered kept-position lists (Eq. 10).
 //
 // The data is a few KB to a few MB that sits in L2; these kernels are latency chains, not bandwidth work.
 // Every comparison that decides a set is taken in double on the fp32 values, and the K-Means runs in
@@ -18,110 +18,139 @@
 namespace mvla {
 namespace {
 
-constexpr int kIndThreads = 256;                     // 32 patches x 8 groups of (head, query) pairs
-constexpr int kIndGroups = kIndThreads / 32;
-constexpr int kPatchThreads = 1024;
+constexpr int kIndThreads = 1024;
+constexpr int kIndPatches = 8;                       // patches per CTA: 8 floats = one 32-byte sector per (head, query)
+constexpr int kIndGroups = kIndThreads / kIndPatches;   // groups of (head, query) pairs
+constexpr int kPatchThreads = 256;
 constexpr int kMaxPatch = kMaxVis / 2;
 constexpr int kPPT = kMaxPatch / kPatchThreads;      // patches per thread, strided by the block size
 
-// grid = (ceil(max P / 32), samples).  Lane = patch (coalesced over the key index), warp = group of pairs.
-__global__ void __launch_bounds__(kIndThreads)
+// grid = (ceil(max P / 8), samples).  Thread = (patch, group): the group walks the (head, query) pairs with
+// stride kIndGroups, so a CTA has all its loads of a pass in flight at once (one or two per thread).
+// Also writes the per-token scores of the patch's two tokens: a_j = ||alpha_j||_1 / (H n_t).
+__global__ void __launch_bounds__(kIndThreads, 1)
 patch_indicators_kernel(const __grid_constant__ BatchDesc bd, int n_heads, const AlphaOut alpha,
-                        const float* __restrict__ l1, float* __restrict__ x_out)
+                        const float* __restrict__ l1, float* __restrict__ x_out, float* __restrict__ attn_out)
 {
-    __shared__ float red[kIndGroups][32][4];
+    __shared__ float red[kIndThreads / 32][kIndPatches][4];
+    __shared__ float tot[kIndPatches][4];
     const SampleDev& s = bd.s[blockIdx.y];
     const int P = s.n_2d;
-    const int p0 = blockIdx.x * 32;
+    const int p0 = blockIdx.x * kIndPatches;
     if (p0 >= P) return;                                  // block-uniform
-    const int lane = threadIdx.x & 31, g = threadIdx.x >> 5;
-    const int p = p0 + lane;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int pl = tid & (kIndPatches - 1), g = tid / kIndPatches;
+    const int p = p0 + pl;
     const bool live = p < P;
     const int npairs = n_heads * s.n_txt;
     const float* base = alpha.ptr + s.vis_off + p;
 
+    // Sum over the lanes of a warp that hold the same patch (lane bits 3 and 4), then over the warps in
+    // a fixed order: tot[patch][c].
+    auto reduce = [&](float (&v)[4], int ncomp) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (c >= ncomp) break;
+            v[c] += __shfl_xor_sync(0xffffffffu, v[c], 8);
+            v[c] += __shfl_xor_sync(0xffffffffu, v[c], 16);
+        }
+        __syncthreads();                                  // earlier readers of red / tot are done
+        if (lane < kIndPatches)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) red[warp][lane][c] = v[c];
+        __syncthreads();
+        if (tid < kIndPatches * 4) {
+            const int q = tid >> 2, c = tid & 3;
+            float acc = 0.f;
+#pragma unroll 8
+            for (int w = 0; w < kIndThreads / 32; ++w) acc += red[w][q][c];
+            tot[q][c] = acc;
+        }
+        __syncthreads();
+    };
+
     // pass 1: <a3, a2>, <a2, a2>, ||a2||_1, ||a3||_1
-    float d32 = 0.f, d22 = 0.f, n2 = 0.f, n3 = 0.f;
+    float v[4] = {0.f, 0.f, 0.f, 0.f};
     if (live) {
 #pragma unroll 4
         for (int idx = g; idx < npairs; idx += kIndGroups) {
             const int h = idx / s.n_txt, i = idx - h * s.n_txt;
             const float* a = base + static_cast<int64_t>(h) * alpha.stride_h + static_cast<int64_t>(i) * alpha.stride_i;
-            const float a2 = __ldg(a), a3 = __ldg(a + P);
-            d32 = fmaf(a3, a2, d32);
-            d22 = fmaf(a2, a2, d22);
-            n2 += fabsf(a2);
-            n3 += fabsf(a3);
+            const float a2 = __ldcg(a), a3 = __ldcg(a + P);
+            v[0] = fmaf(a3, a2, v[0]);
+            v[1] = fmaf(a2, a2, v[1]);
+            v[2] += fabsf(a2);
+            v[3] += fabsf(a3);
         }
     }
-    red[g][lane][0] = d32; red[g][lane][1] = d22; red[g][lane][2] = n2; red[g][lane][3] = n3;
-    __syncthreads();
-    float t[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int w = 0; w < kIndGroups; ++w)                  // fixed order: every warp gets the same totals
-#pragma unroll
-        for (int c = 0; c < 4; ++c) t[c] += red[w][lane][c];
-    const float coef = t[1] > 0.f ? t[0] / t[1] : 0.f;   // projection coefficient of a3 on a2 (Eq. 3-4)
-    __syncthreads();
+    reduce(v, 4);
+    const float t0 = tot[pl][0], t1 = tot[pl][1], t2 = tot[pl][2], t3 = tot[pl][3];
+    const float coef = t1 > 0.f ? t0 / t1 : 0.f;         // projection coefficient of a3 on a2 (Eq. 3-4)
 
     // pass 2: || a3 - coef a2 ||_1, the part of the 3D token's attention that the 2D token's does not explain
-    float no = 0.f;
+    float o[4] = {0.f, 0.f, 0.f, 0.f};
     if (live) {
 #pragma unroll 4
         for (int idx = g; idx < npairs; idx += kIndGroups) {
             const int h = idx / s.n_txt, i = idx - h * s.n_txt;
             const float* a = base + static_cast<int64_t>(h) * alpha.stride_h + static_cast<int64_t>(i) * alpha.stride_i;
-            no += fabsf(fmaf(-coef, __ldg(a), __ldg(a + P)));
+            o[0] += fabsf(fmaf(-coef, __ldcg(a), __ldcg(a + P)));
         }
     }
-    red[g][lane][0] = no;
-    __syncthreads();
+    reduce(o, 1);
     if (g == 0 && live) {
-        float o = 0.f;
-#pragma unroll
-        for (int w = 0; w < kIndGroups; ++w) o += red[w][lane][0];
         const float f2 = l1[s.vis_off + p], f3 = l1[s.vis_off + P + p];
         float4 x;
         x.x = f2 / (f2 + f3);                             // Eq. 3-1, the term of this patch
         x.y = f3 / (f2 + f3);
-        x.z = t[2] / (t[2] + t[3]);                       // Eq. P2D
-        x.w = o / (t[2] + t[3]);                          // Eq. P3D
+        x.z = t2 / (t2 + t3);                             // Eq. P2D
+        x.w = tot[pl][0] / (t2 + t3);                     // Eq. P3D
         reinterpret_cast<float4*>(x_out)[s.vis_off / 2 + p] = x;
+        const float inv = 1.f / static_cast<float>(npairs);
+        attn_out[s.vis_off + p] = t2 * inv;               // mean over heads and text queries
+        attn_out[s.vis_off + P + p] = t3 * inv;
     }
 }
 
 struct PatchSmem {
-    double red[kPatchThreads / 32][6];
-    double tot[6];
+    double mass[kMaxPatch];                 // attention mass of every patch (what K-Means clusters)
+    uint8_t label[kMaxPatch];
+    uint8_t keep[2 * kMaxPatch];            // keep flags in visual order: 2D tokens, then 3D tokens
+    double red[kPatchThreads / 32][5];
+    double tot[5];
     double centre[3];
+    int cnt[5];                             // kept 2D, kept 3D, patches per class
+    int iters;
+    int out_off;
+    int scan[kPatchThreads / 32 + 1];
 };
 
-// Deterministic block reduction of N doubles per thread (fixed shuffle tree, then warp 0 over the warp
+// Deterministic block reduction of 5 doubles per thread (fixed shuffle tree, then warp 0 over the warp
 // partials).  Component c is a maximum when bit c of `max_mask` is set, else a sum.  Result in sm.tot.
-template <int N>
-__device__ __forceinline__ void block_reduce_d(double (&v)[N], unsigned max_mask, PatchSmem& sm)
+__device__ __forceinline__ void block_reduce5(double (&v)[5], unsigned max_mask, PatchSmem& sm)
 {
+    constexpr int NW = kPatchThreads / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
-    for (int c = 0; c < N; ++c)
+    for (int c = 0; c < 5; ++c)
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) {
             const double o = __shfl_xor_sync(0xffffffffu, v[c], off);
             v[c] = (max_mask >> c & 1u) ? fmax(v[c], o) : v[c] + o;
         }
-    __syncthreads();                                      // earlier readers of sm.red / sm.tot are done
     if (lane == 0)
 #pragma unroll
-        for (int c = 0; c < N; ++c) sm.red[warp][c] = v[c];
+        for (int c = 0; c < 5; ++c) sm.red[warp][c] = v[c];
     __syncthreads();
     if (warp == 0) {
 #pragma unroll
-        for (int c = 0; c < N; ++c) {
-            double y = sm.red[lane][c];                   // kPatchThreads / 32 == 32 warps
+        for (int c = 0; c < 5; ++c) {
+            const bool is_max = (max_mask >> c & 1u) != 0;
+            double y = lane < NW ? sm.red[lane][c] : (is_max ? -CUDART_INF : 0.0);
 #pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) {
+            for (int off = NW / 2; off >= 1; off >>= 1) {
                 const double o = __shfl_xor_sync(0xffffffffu, y, off);
-                y = (max_mask >> c & 1u) ? fmax(y, o) : y + o;
+                y = is_max ? fmax(y, o) : y + o;
             }
             if (lane == 0) sm.tot[c] = y;
         }
@@ -129,163 +158,203 @@ __device__ __forceinline__ void block_reduce_d(double (&v)[N], unsigned max_mask
     __syncthreads();
 }
 
-// One CTA per sample.
-__global__ void __launch_bounds__(kPatchThreads, 1)
-patch_decide_kernel(const __grid_constant__ BatchDesc bd, const PatchParams pp, const PatchIO io)
+__device__ __forceinline__ double warp_sum_d(double v)
 {
-    static_assert(kPatchThreads / 32 == 32, "the second reduction level is one warp");
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    return v;
+}
+__device__ __forceinline__ int ld_volatile_i32(const int* p)
+{
+    int v;
+    asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// One CTA per sample: stages 1-4 of Alg. 1 for its patches, then its first output row and the ordered
+// kept positions.  A sample's first output row is the sum of the kept rows of the samples before it:
+// each CTA publishes its count (value, fence, flag) and reads the counts of the samples before it in this
+// launch, which have lower block indices and were therefore dispatched no later than itself; the wait is
+// bounded and reports MVLA_ERR_TIMEOUT.  The CTA that finishes last clears the flags for the next launch.
+__global__ void __launch_bounds__(kPatchThreads, 1)
+patch_select_kernel(const __grid_constant__ BatchDesc bd, const PatchParams pp, const PatchIO io)
+{
     __shared__ PatchSmem sm;
     const SampleDev& s = bd.s[blockIdx.x];
     const int b_glob = io.chunk_first + blockIdx.x;
-    const int tid = threadIdx.x;
-    const int P = s.n_2d;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int P = s.n_2d, nv = 2 * P;
     const int pat_off = s.vis_off / 2;
     const bool carry = s.c_prev != 0.f;
     const bool cold = s.t == 1 && pp.cold_start_full_keep;
     float4* state = reinterpret_cast<float4*>(io.xhat_state) + static_cast<int64_t>(s.mstate_off) * pp.max_patch;
+    if (tid < 5) sm.cnt[tid] = 0;
 
-    // ---- stage 1 (action iteration): X^ = c_prev X^ + c_new X for every patch and indicator (Eqs. 8, 9)
+    // ---- stage 1 (action iteration): X^ = c_prev X^ + c_new X for every patch and indicator (Eqs. 8, 9).
+    //      All loads of a thread are issued before anything depends on them.
+    float4 x[kPPT], pr[kPPT];
+    float a2[kPPT], a3[kPPT], uu[kPPT];
+#pragma unroll
+    for (int e = 0; e < kPPT; ++e) {
+        if (e * kPatchThreads >= P) break;                        // block-uniform
+        const int p = tid + e * kPatchThreads;
+        if (p < P) {
+            x[e] = reinterpret_cast<const float4*>(io.x)[pat_off + p];
+            if (carry) pr[e] = state[p];
+            a2[e] = io.attn[s.vis_off + p];
+            a3[e] = io.attn[s.vis_off + P + p];
+            uu[e] = io.rand_u[pat_off + p];
+        }
+    }
     float4 xh[kPPT];
-    double mass[kPPT], u[kPPT];
-    bool live[kPPT];
     double init[5] = {0.0, -CUDART_INF, -CUDART_INF, 0.0, 0.0};   // sum mass, max mass, max -mass, sum M^S2_2D, sum M^S2_3D
 #pragma unroll
     for (int e = 0; e < kPPT; ++e) {
+        if (e * kPatchThreads >= P) break;
         const int p = tid + e * kPatchThreads;
-        live[e] = p < P;
-        xh[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-        mass[e] = 0.0; u[e] = 0.0;
-        if (live[e]) {
-            const float4 x = reinterpret_cast<const float4*>(io.x)[pat_off + p];
-            float4 v = x;
+        if (p < P) {
+            float4 v = x[e];
             if (carry) {
-                const float4 pr = state[p];
-                v.x = fmaf(s.c_prev, pr.x, s.c_new * x.x);
-                v.y = fmaf(s.c_prev, pr.y, s.c_new * x.y);
-                v.z = fmaf(s.c_prev, pr.z, s.c_new * x.z);
-                v.w = fmaf(s.c_prev, pr.w, s.c_new * x.w);
+                v.x = fmaf(s.c_prev, pr[e].x, s.c_new * x[e].x);
+                v.y = fmaf(s.c_prev, pr[e].y, s.c_new * x[e].y);
+                v.z = fmaf(s.c_prev, pr[e].z, s.c_new * x[e].z);
+                v.w = fmaf(s.c_prev, pr[e].w, s.c_new * x[e].w);
             }
             xh[e] = v;
             if (s.update_state) state[p] = v;
             if (io.xhat_out) reinterpret_cast<float4*>(io.xhat_out)[pat_off + p] = v;
             // the patch's attention response: the mass of its two tokens
-            mass[e] = static_cast<double>(io.attn[s.vis_off + p]) + static_cast<double>(io.attn[s.vis_off + P + p]);
-            u[e] = static_cast<double>(io.rand_u[pat_off + p]);
-            init[0] += mass[e];
-            init[1] = fmax(init[1], mass[e]);
-            init[2] = fmax(init[2], -mass[e]);
+            const double m = static_cast<double>(a2[e]) + static_cast<double>(a3[e]);
+            sm.mass[p] = m;
+            sm.label[p] = 255;
+            init[0] += m;
+            init[1] = fmax(init[1], m);
+            init[2] = fmax(init[2], -m);
             init[3] += static_cast<double>(v.z);
             init[4] += static_cast<double>(v.w);
         }
     }
-    block_reduce_d<5>(init, 0x6u, sm);
+    block_reduce5(init, 0x6u, sm);
     const double mu_2d = sm.tot[3] / P, mu_3d = sm.tot[4] / P;    // baselines: means of the smoothed shares
-    if (tid == 0) {
-        sm.centre[0] = -sm.tot[2];                                // min
-        sm.centre[1] = sm.tot[0] / P;                             // mean
-        sm.centre[2] = sm.tot[1];                                 // max
+
+    // ---- stage 3 preparation: 1-D K-Means, K = 3 (Sec. 4.2), by one warp without block barriers.  A round:
+    //      assign to the nearest centre (ties to the lower one); unless nothing changed, move the centres
+    //      to the class means.
+    if (warp == 0) {
+        double c0 = -sm.tot[2], c1 = sm.tot[0] / P, c2 = sm.tot[1];   // min, mean, max
+        int iters = 0;
+        while (iters < pp.kmeans_max_iter) {                      // warp-uniform
+            ++iters;
+            int changed = 0;
+            double s0 = 0.0, s1 = 0.0, s2 = 0.0, n0 = 0.0, n1 = 0.0, n2 = 0.0;
+            for (int p = lane; p < P; p += 32) {
+                const double m = sm.mass[p];
+                int best = 0;
+                double bdist = fabs(m - c0);
+                const double d1 = fabs(m - c1), d2 = fabs(m - c2);
+                if (d1 < bdist) { bdist = d1; best = 1; }
+                if (d2 < bdist) { bdist = d2; best = 2; }
+                if (sm.label[p] != best) { sm.label[p] = static_cast<uint8_t>(best); changed = 1; }
+                s0 += best == 0 ? m : 0.0; n0 += best == 0 ? 1.0 : 0.0;
+                s1 += best == 1 ? m : 0.0; n1 += best == 1 ? 1.0 : 0.0;
+                s2 += best == 2 ? m : 0.0; n2 += best == 2 ? 1.0 : 0.0;
+            }
+            if (!__any_sync(0xffffffffu, changed)) break;
+            s0 = warp_sum_d(s0); s1 = warp_sum_d(s1); s2 = warp_sum_d(s2);
+            n0 = warp_sum_d(n0); n1 = warp_sum_d(n1); n2 = warp_sum_d(n2);
+            if (n0 > 0.0) c0 = s0 / n0;
+            if (n1 > 0.0) c1 = s1 / n1;
+            if (n2 > 0.0) c2 = s2 / n2;
+        }
+        if (lane == 0) { sm.centre[0] = c0; sm.centre[1] = c1; sm.centre[2] = c2; sm.iters = iters; }
     }
     __syncthreads();
-
-    // ---- stage 3 preparation: 1-D K-Means, K = 3 (Sec. 4.2).  A round: assign to the nearest centre
-    //      (ties to the lower one); unless nothing changed, move the centres to the class means.
-    int label[kPPT];
-#pragma unroll
-    for (int e = 0; e < kPPT; ++e) label[e] = -1;
-    int iters = 0;
-    while (iters < pp.kmeans_max_iter) {                          // block-uniform
-        ++iters;
-        const double c0 = sm.centre[0], c1 = sm.centre[1], c2 = sm.centre[2];
-        int changed = 0;
-        double acc[6] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0};           // class sums, class counts
-#pragma unroll
-        for (int e = 0; e < kPPT; ++e) {
-            if (!live[e]) continue;
-            int best = 0;
-            double bd_ = fabs(mass[e] - c0);
-            const double d1 = fabs(mass[e] - c1), d2 = fabs(mass[e] - c2);
-            if (d1 < bd_) { bd_ = d1; best = 1; }
-            if (d2 < bd_) { bd_ = d2; best = 2; }
-            if (best != label[e]) { label[e] = best; changed = 1; }
-            acc[best] += mass[e];
-            acc[3 + best] += 1.0;
-        }
-        if (!__syncthreads_or(changed)) break;
-        block_reduce_d<6>(acc, 0u, sm);
-        if (tid == 0)
-#pragma unroll
-            for (int c = 0; c < 3; ++c)
-                if (sm.tot[3 + c] > 0.0) sm.centre[c] = sm.tot[c] / sm.tot[3 + c];
-        __syncthreads();
-    }
 
     // ---- stages 2-4 for every patch: C_S1 (dual threshold), C_S2 (semantic rules), fusion, masks
     const int both = MVLA_SET_2D | MVLA_SET_3D;
-    double cnt[5] = {0.0, 0.0, 0.0, 0.0, 0.0};                    // kept 2D, kept 3D, patches per class
 #pragma unroll
     for (int e = 0; e < kPPT; ++e) {
-        if (!live[e]) continue;
+        if (e * kPatchThreads >= P) break;
         const int p = tid + e * kPatchThreads;
-        const double s1_3d = xh[e].y, m2 = xh[e].z, m3 = xh[e].w;
-        const int c1 = s1_3d < pp.tau_2d ? MVLA_SET_2D : (s1_3d > pp.tau_3d ? MVLA_SET_3D : both);
-        int c2;
-        if (label[e] == MVLA_LABEL_BG) c2 = u[e] < pp.bg_prune_prob ? 0 : both;
-        else if (label[e] == MVLA_LABEL_ROB) c2 = m3 > mu_3d ? both : (m2 > mu_2d ? MVLA_SET_2D : 0);
-        else c2 = (m2 > pp.obj_2d_min && m3 < pp.eps_3d) ? MVLA_SET_2D : both;
-        int cf = 0;
-        if (c2 != 0) {
-            cf = c2 & c1;
-            if (cf == 0) cf = c2;                                 // conflict resolution
+        if (p < P) {
+            const int label = sm.label[p];
+            const double s1_3d = xh[e].y, m2 = xh[e].z, m3 = xh[e].w;
+            const int c1 = s1_3d < pp.tau_2d ? MVLA_SET_2D : (s1_3d > pp.tau_3d ? MVLA_SET_3D : both);
+            int c2;
+            if (label == MVLA_LABEL_BG) c2 = static_cast<double>(uu[e]) < pp.bg_prune_prob ? 0 : both;
+            else if (label == MVLA_LABEL_ROB) c2 = m3 > mu_3d ? both : (m2 > mu_2d ? MVLA_SET_2D : 0);
+            else c2 = (m2 > pp.obj_2d_min && m3 < pp.eps_3d) ? MVLA_SET_2D : both;
+            int cf = 0;
+            if (c2 != 0) {
+                cf = c2 & c1;
+                if (cf == 0) cf = c2;                             // conflict resolution
+            }
+            if (cold) cf = both;                                  // cold start: full unpruned tokens
+            if (io.info_out) io.info_out[pat_off + p] = label | (c1 << 2) | (c2 << 4) | (cf << 6);
+            const int k2 = (cf & MVLA_SET_2D) ? 1 : 0, k3 = (cf & MVLA_SET_3D) ? 1 : 0;
+            sm.keep[p] = static_cast<uint8_t>(k2);
+            sm.keep[P + p] = static_cast<uint8_t>(k3);
+            if (k2) atomicAdd(&sm.cnt[0], 1);                     // integer counts: the order of the adds is immaterial
+            if (k3) atomicAdd(&sm.cnt[1], 1);
+            atomicAdd(&sm.cnt[2 + label], 1);
         }
-        if (cold) cf = both;                                      // cold start: full unpruned tokens
-        if (io.info_out) io.info_out[pat_off + p] = label[e] | (c1 << 2) | (c2 << 4) | (cf << 6);
-        io.mask_ws[s.vis_off + p] = (cf & MVLA_SET_2D) ? 1 : 0;
-        io.mask_ws[s.vis_off + P + p] = (cf & MVLA_SET_3D) ? 1 : 0;
-        cnt[0] += (cf & MVLA_SET_2D) ? 1.0 : 0.0;
-        cnt[1] += (cf & MVLA_SET_3D) ? 1.0 : 0.0;
-        cnt[2 + label[e]] += 1.0;
-    }
-    block_reduce_d<5>(cnt, 0u, sm);
-    if (tid == 0) {
-        const int k2 = static_cast<int>(sm.tot[0]), k3 = static_cast<int>(sm.tot[1]);
-        io.nout_ws[b_glob * 4 + 0] = s.n_txt + k2 + k3;
-        io.nout_ws[b_glob * 4 + 1] = k2;
-        io.nout_ws[b_glob * 4 + 2] = k3;
-        if (io.counts) { io.counts[b_glob * 2] = k2; io.counts[b_glob * 2 + 1] = k3; }
-        if (io.diag) {
-            mvla_patch_diag dg;
-            dg.t = s.t; dg.iters = iters;
-            for (int c = 0; c < 3; ++c) { dg.n_label[c] = static_cast<int>(sm.tot[2 + c]); dg.centre[c] = static_cast<float>(sm.centre[c]); }
-            dg.k_2d = k2; dg.k_3d = k3; dg.n_out = s.n_txt + k2 + k3;
-            dg.mu_2d = static_cast<float>(mu_2d); dg.mu_3d = static_cast<float>(mu_3d);
-            dg.reserved[0] = dg.reserved[1] = dg.reserved[2] = 0.f;
-            io.diag[b_glob] = dg;
-        }
-    }
-}
-
-// One CTA per sample: its first output row (the kept rows of the samples before it), then the kept
-// positions in sequence order.  The three segments are contiguous, so a kept token's output row is the
-// rows of the segments lying before its own plus its rank inside its modality.
-__global__ void __launch_bounds__(kPatchThreads, 1)
-patch_emit_kernel(const __grid_constant__ BatchDesc bd, const PatchIO io)
-{
-    __shared__ int scan[kPatchThreads / 32 + 1];
-    __shared__ int s_off;
-    const SampleDev& s = bd.s[blockIdx.x];
-    const int b_glob = io.chunk_first + blockIdx.x;
-    const int tid = threadIdx.x;
-    const int P = s.n_2d, nv = 2 * P;
-    if (tid == 0) {
-        int off = 0;
-        for (int b = 0; b < b_glob; ++b) off += io.nout_ws[b * 4];
-        s_off = off;
-        io.out_offsets[b_glob] = off;
-        if (b_glob == io.batch_total - 1) io.out_offsets[io.batch_total] = off + io.nout_ws[b_glob * 4];
     }
     __syncthreads();
-    const int out_off = s_off;
-    const int k2 = io.nout_ws[b_glob * 4 + 1], k3 = io.nout_ws[b_glob * 4 + 2];
+    const int k2 = sm.cnt[0], k3 = sm.cnt[1];
+    const int n_out = s.n_txt + k2 + k3;
+
+    // ---- first output row: publish this sample's count, add up the counts of the samples before it
+    if (warp == 0) {
+        if (lane == 0) {
+            io.nout_ws[b_glob] = n_out;
+            __threadfence();
+            asm volatile("st.volatile.global.s32 [%0], %1;" ::"l"(io.ready_ws + b_glob), "r"(1) : "memory");
+        }
+        int off = 0;
+        bool ok = true;
+        for (int b = lane; b < b_glob; b += 32) {
+            if (b >= io.chunk_first) {                            // same launch: wait for its flag (bounded)
+                bool got = false;
+                for (uint32_t it = 0; it < kSpinLimit && !got; ++it) {
+                    got = ld_volatile_i32(io.ready_ws + b) != 0;
+                    if (!got) __nanosleep(64);
+                }
+                ok &= got;
+                __threadfence();
+            }
+            off += ld_volatile_i32(io.nout_ws + b);               // earlier launches of this call are complete
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
+        if (!__all_sync(0xffffffffu, ok) && lane == 0) *reinterpret_cast<volatile int*>(io.status) = MVLA_ERR_TIMEOUT;
+        if (lane == 0) {
+            sm.out_off = off;
+            io.out_offsets[b_glob] = off;
+            if (b_glob == io.batch_total - 1) io.out_offsets[io.batch_total] = off + n_out;
+            if (io.counts) { io.counts[b_glob * 2] = k2; io.counts[b_glob * 2 + 1] = k3; }
+            if (io.diag) {
+                mvla_patch_diag dg;
+                dg.t = s.t; dg.iters = sm.iters;
+                for (int c = 0; c < 3; ++c) { dg.n_label[c] = sm.cnt[2 + c]; dg.centre[c] = static_cast<float>(sm.centre[c]); }
+                dg.k_2d = k2; dg.k_3d = k3; dg.n_out = n_out;
+                dg.mu_2d = static_cast<float>(mu_2d); dg.mu_3d = static_cast<float>(mu_3d);
+                dg.reserved[0] = dg.reserved[1] = dg.reserved[2] = 0.f;
+                io.diag[b_glob] = dg;
+            }
+            // every wait of this CTA is over: the CTA that gets here last clears the flags of the launch
+            __threadfence();
+            if (atomicAdd(io.done_ws, 1) == static_cast<int>(gridDim.x) - 1) {
+                for (int b = 0; b < static_cast<int>(gridDim.x); ++b) io.ready_ws[io.chunk_first + b] = 0;
+                *io.done_ws = 0;
+                __threadfence();
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- Eq. 10 as an ordered list.  The three segments are contiguous, so a kept token's output row is
+    //      the rows of the segments lying before its own plus its rank inside its modality.
+    const int out_off = sm.out_off;
     const int base2 = (s.off_txt < s.off_2d ? s.n_txt : 0) + (s.off_3d < s.off_2d ? k3 : 0);
     const int base3 = (s.off_txt < s.off_3d ? s.n_txt : 0) + (s.off_2d < s.off_3d ? k2 : 0);
     const int baset = (s.off_2d < s.off_txt ? k2 : 0) + (s.off_3d < s.off_txt ? k3 : 0);
@@ -293,9 +362,9 @@ patch_emit_kernel(const __grid_constant__ BatchDesc bd, const PatchIO io)
     int run = 0;
     for (int j0 = 0; j0 < nv; j0 += kPatchThreads) {              // block-uniform
         const int j = j0 + tid;
-        const int c = j < nv ? io.mask_ws[s.vis_off + j] : 0;
+        const int c = j < nv ? sm.keep[j] : 0;
         int tot = 0;
-        const int r = run + block_exscan<kPatchThreads>(c, scan, &tot);
+        const int r = run + block_exscan<kPatchThreads>(c, sm.scan, &tot);
         run += tot;
         if (c) {
             if (j < P) io.kept_idx[out_off + base2 + r] = s.off_2d + j;
@@ -307,24 +376,19 @@ patch_emit_kernel(const __grid_constant__ BatchDesc bd, const PatchIO io)
 }  // namespace
 
 cudaError_t launch_patch_indicators(const BatchDesc& bd, int n_heads, AlphaOut alpha, const float* l1,
-                                    float* x_out, cudaStream_t stream)
+                                    float* x_out, float* attn_out, cudaStream_t stream)
 {
     int max_p = 0;
     for (int b = 0; b < bd.n; ++b) max_p = max(max_p, bd.s[b].n_2d);
     if (max_p == 0) return cudaSuccess;
-    patch_indicators_kernel<<<dim3((max_p + 31) / 32, bd.n), kIndThreads, 0, stream>>>(bd, n_heads, alpha, l1, x_out);
+    patch_indicators_kernel<<<dim3((max_p + kIndPatches - 1) / kIndPatches, bd.n), kIndThreads, 0, stream>>>(
+        bd, n_heads, alpha, l1, x_out, attn_out);
     return cudaGetLastError();
 }
 
-cudaError_t launch_patch_decide(const BatchDesc& bd, const PatchParams& pp, const PatchIO& io, cudaStream_t stream)
+cudaError_t launch_patch_select(const BatchDesc& bd, const PatchParams& pp, const PatchIO& io, cudaStream_t stream)
 {
-    patch_decide_kernel<<<bd.n, kPatchThreads, 0, stream>>>(bd, pp, io);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_patch_emit(const BatchDesc& bd, const PatchIO& io, cudaStream_t stream)
-{
-    patch_emit_kernel<<<bd.n, kPatchThreads, 0, stream>>>(bd, io);
+    patch_select_kernel<<<bd.n, kPatchThreads, 0, stream>>>(bd, pp, io);
     return cudaGetLastError();
 }
 
