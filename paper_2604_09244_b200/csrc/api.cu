@@ -348,12 +348,13 @@ int32_t run_patch_indicators(mvla_ctx* ctx, const Plan& plan, int32_t batch, con
     const AlphaOut alpha = alpha_of(ctx);
     for (int first = 0; first < batch; first += kMaxChunk) {
         const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
-        const int32_t rc = run_salience_chunk(ctx, bd, q, k, rows, hidden, ctx->l1_ws, nullptr, nullptr, false, st, alpha);
+        const int32_t rc = run_salience_chunk(ctx, bd, q, k, rows, nullptr, nullptr, nullptr, nullptr, false, st, alpha);
         if (rc != MVLA_OK) return rc;
     }
     for (int first = 0; first < batch; first += kMaxChunk) {
         const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
-        const cudaError_t e = launch_patch_indicators(bd, ctx->cfg.n_heads, alpha, ctx->l1_ws, x_out, attn_out, st);
+        const cudaError_t e = launch_patch_indicators(bd, ctx->cfg.n_heads, alpha, ctx->cfg.dtype, ctx->cfg.d_model, hidden,
+                                                      x_out, attn_out, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
     return MVLA_OK;

@@ -155,9 +155,9 @@ struct PatchIO {
     int32_t* out_offsets;
     int32_t chunk_first, batch_total;
 };
-// x[p] = per-patch indicators from the attention copy and the feature norms; attn = per-token scores.
-cudaError_t launch_patch_indicators(const BatchDesc& bd, int n_heads, AlphaOut alpha, const float* l1,
-                                    float* x_out, float* attn_out, cudaStream_t stream);
+// x[p] = per-patch indicators from the attention copy and the L1 norms of the hidden rows; attn = per-token scores.
+cudaError_t launch_patch_indicators(const BatchDesc& bd, int n_heads, AlphaOut alpha, int dtype, int d_model,
+                                    const void* hidden, float* x_out, float* attn_out, cudaStream_t stream);
 // Stages 1-4 of Alg. 1 for every patch, output offsets over the batch, ordered kept-position lists.
 cudaError_t launch_patch_select(const BatchDesc& bd, const PatchParams& pp, const PatchIO& io, cudaStream_t stream);
 

@@ -19,24 +19,33 @@ namespace mvla {
 namespace {
 
 constexpr int kIndThreads = 1024;
-constexpr int kIndPatches = 8;                       // patches per CTA: 8 floats = one 32-byte sector per (head, query)
-constexpr int kIndGroups = kIndThreads / kIndPatches;   // groups of (head, query) pairs
 constexpr int kPatchThreads = 256;
 constexpr int kMaxPatch = kMaxVis / 2;
 constexpr int kPPT = kMaxPatch / kPatchThreads;      // patches per thread, strided by the block size
 
-// grid = (ceil(max P / 8), samples).  Thread = (patch, group): the group walks the (head, query) pairs with
-// stride kIndGroups, so a CTA has all its loads of a pass in flight at once (one or two per thread).
+// grid = (ceil(max P / PP), samples), PP = 2, 4 or 8 patches per CTA (8 floats = one 32-byte sector per
+// (head, query); fewer patches per CTA when the batch is too small to fill the SMs otherwise).
+// Thread = (patch, group): the group walks the (head, query) pairs with stride 1024 / PP, so a CTA has
+// all its loads of a pass in flight at once (a few per thread).
 // Also writes the per-token scores of the patch's two tokens: a_j = ||alpha_j||_1 / (H n_t).
+// The L1 feature norms of the CTA's 2 PP rows (Sec. 3.1.2) are taken here too, 512 / PP threads per row,
+// their loads issued before the kernel waits for the attention copy of the kernel before it.
+template <typename T, int PP>
 __global__ void __launch_bounds__(kIndThreads, 1)
 patch_indicators_kernel(const __grid_constant__ BatchDesc bd, int n_heads, const AlphaOut alpha,
-                        const float* __restrict__ l1, float* __restrict__ x_out, float* __restrict__ attn_out)
+                        const T* __restrict__ hidden, int d_model, float* __restrict__ x_out,
+                        float* __restrict__ attn_out)
 {
+    constexpr int kIndPatches = PP;
+    constexpr int kIndGroups = kIndThreads / PP;          // groups of (head, query) pairs
+    constexpr int kRowThreads = kIndThreads / (2 * PP);   // threads that share one hidden row
     __shared__ float red[kIndThreads / 32][kIndPatches][4];
     __shared__ float tot[kIndPatches][4];
+    __shared__ float rown[kIndThreads / 32];
     const SampleDev& s = bd.s[blockIdx.y];
     const int P = s.n_2d;
     const int p0 = blockIdx.x * kIndPatches;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p0 >= P) return;                                  // block-uniform
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int pl = tid & (kIndPatches - 1), g = tid / kIndPatches;
@@ -45,14 +54,46 @@ patch_indicators_kernel(const __grid_constant__ BatchDesc bd, int n_heads, const
     const int npairs = n_heads * s.n_txt;
     const float* base = alpha.ptr + s.vis_off + p;
 
-    // Sum over the lanes of a warp that hold the same patch (lane bits 3 and 4), then over the warps in
-    // a fixed order: tot[patch][c].
+    // ---- feature norms: row r of the CTA = 2D token p0 + r (r < PP) or 3D token p0 + r - PP
+    {
+        const int r = tid / kRowThreads, within = tid % kRowThreads;
+        const int pr = p0 + (r & (kIndPatches - 1));
+        float acc = 0.f;
+        if (pr < P) {
+            const int row = s.seq_off + (r < kIndPatches ? s.off_2d : s.off_3d) + pr;
+            constexpr int kVec = 16 / sizeof(T);
+            const uint4* src = reinterpret_cast<const uint4*>(hidden + static_cast<int64_t>(row) * d_model);
+            const int nvec = d_model / kVec;
+#pragma unroll 8
+            for (int i = within; i < nvec; i += kRowThreads) {
+                const uint4 u = __ldg(src + i);
+                if constexpr (sizeof(T) == 2) {
+                    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        acc += fabsf(__uint_as_float(w[e] << 16));           // low bf16
+                        acc += fabsf(__uint_as_float(w[e] & 0xFFFF0000u));   // high bf16
+                    }
+                } else {
+                    acc += fabsf(__uint_as_float(u.x)) + fabsf(__uint_as_float(u.y)) +
+                           fabsf(__uint_as_float(u.z)) + fabsf(__uint_as_float(u.w));
+                }
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (lane == 0) rown[warp] = acc;                  // read after the barriers of the first reduction
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");    // the attention copy comes from the kernel before this one
+
+    // Sum over the lanes of a warp that hold the same patch (the lane bits above log2 PP), then over the
+    // warps in a fixed order: tot[patch][c].
     auto reduce = [&](float (&v)[4], int ncomp) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             if (c >= ncomp) break;
-            v[c] += __shfl_xor_sync(0xffffffffu, v[c], 8);
-            v[c] += __shfl_xor_sync(0xffffffffu, v[c], 16);
+#pragma unroll
+            for (int off = PP; off < 32; off <<= 1) v[c] += __shfl_xor_sync(0xffffffffu, v[c], off);
         }
         __syncthreads();                                  // earlier readers of red / tot are done
         if (lane < kIndPatches)
@@ -99,7 +140,13 @@ patch_indicators_kernel(const __grid_constant__ BatchDesc bd, int n_heads, const
     }
     reduce(o, 1);
     if (g == 0 && live) {
-        const float f2 = l1[s.vis_off + p], f3 = l1[s.vis_off + P + p];
+        constexpr int kRowWarps = kRowThreads / 32;
+        float f2 = 0.f, f3 = 0.f;                         // the patch's 2D token, its 3D token
+#pragma unroll
+        for (int w = 0; w < kRowWarps; ++w) {
+            f2 += rown[pl * kRowWarps + w];
+            f3 += rown[(kIndPatches + pl) * kRowWarps + w];
+        }
         float4 x;
         x.x = f2 / (f2 + f3);                             // Eq. 3-1, the term of this patch
         x.y = f3 / (f2 + f3);
@@ -189,6 +236,8 @@ patch_select_kernel(const __grid_constant__ BatchDesc bd, const PatchParams pp, 
     const bool cold = s.t == 1 && pp.cold_start_full_keep;
     float4* state = reinterpret_cast<float4*>(io.xhat_state) + static_cast<int64_t>(s.mstate_off) * pp.max_patch;
     if (tid < 5) sm.cnt[tid] = 0;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");    // scores and indicators come from the kernel before this one
 
     // ---- stage 1 (action iteration): X^ = c_prev X^ + c_new X for every patch and indicator (Eqs. 8, 9).
     //      All loads of a thread are issued before anything depends on them.
@@ -304,11 +353,14 @@ patch_select_kernel(const __grid_constant__ BatchDesc bd, const PatchParams pp, 
     const int n_out = s.n_txt + k2 + k3;
 
     // ---- first output row: publish this sample's count, add up the counts of the samples before it
+    const bool alone = gridDim.x == 1;                            // nobody in this launch to wait for or to tell
     if (warp == 0) {
         if (lane == 0) {
-            io.nout_ws[b_glob] = n_out;
-            __threadfence();
-            asm volatile("st.volatile.global.s32 [%0], %1;" ::"l"(io.ready_ws + b_glob), "r"(1) : "memory");
+            io.nout_ws[b_glob] = n_out;                           // later launches of this call read it in stream order
+            if (!alone) {
+                __threadfence();
+                asm volatile("st.volatile.global.s32 [%0], %1;" ::"l"(io.ready_ws + b_glob), "r"(1) : "memory");
+            }
         }
         int off = 0;
         bool ok = true;
@@ -342,8 +394,8 @@ patch_select_kernel(const __grid_constant__ BatchDesc bd, const PatchParams pp, 
                 io.diag[b_glob] = dg;
             }
             // every wait of this CTA is over: the CTA that gets here last clears the flags of the launch
-            __threadfence();
-            if (atomicAdd(io.done_ws, 1) == static_cast<int>(gridDim.x) - 1) {
+            if (!alone) __threadfence();
+            if (!alone && atomicAdd(io.done_ws, 1) == static_cast<int>(gridDim.x) - 1) {
                 for (int b = 0; b < static_cast<int>(gridDim.x); ++b) io.ready_ws[io.chunk_first + b] = 0;
                 *io.done_ws = 0;
                 __threadfence();
@@ -375,21 +427,42 @@ patch_select_kernel(const __grid_constant__ BatchDesc bd, const PatchParams pp, 
 
 }  // namespace
 
-cudaError_t launch_patch_indicators(const BatchDesc& bd, int n_heads, AlphaOut alpha, const float* l1,
-                                    float* x_out, float* attn_out, cudaStream_t stream)
+cudaError_t launch_patch_indicators(const BatchDesc& bd, int n_heads, AlphaOut alpha, int dtype, int d_model,
+                                    const void* hidden, float* x_out, float* attn_out, cudaStream_t stream)
 {
     int max_p = 0;
     for (int b = 0; b < bd.n; ++b) max_p = max(max_p, bd.s[b].n_2d);
     if (max_p == 0) return cudaSuccess;
-    patch_indicators_kernel<<<dim3((max_p + kIndPatches - 1) / kIndPatches, bd.n), kIndThreads, 0, stream>>>(
-        bd, n_heads, alpha, l1, x_out, attn_out);
-    return cudaGetLastError();
+    // as many patches per CTA as still give every SM a CTA (148 SMs)
+    int pp = 8;
+    while (pp > 2 && static_cast<int64_t>(bd.n) * ((max_p + pp - 1) / pp) < 148) pp >>= 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((max_p + pp - 1) / pp, bd.n);
+    cfg.blockDim = dim3(kIndThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1] = {pdl_attribute()};
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+#define MVLA_IND(T, PPV)                                                                                  \
+    if (pp == PPV)                                                                                        \
+        return cudaLaunchKernelEx(&cfg, patch_indicators_kernel<T, PPV>, bd, n_heads, alpha,              \
+                                  static_cast<const T*>(hidden), d_model, x_out, attn_out);
+    if (dtype == MVLA_DTYPE_BF16) { MVLA_IND(__nv_bfloat16, 8) MVLA_IND(__nv_bfloat16, 4) MVLA_IND(__nv_bfloat16, 2) }
+    else { MVLA_IND(float, 8) MVLA_IND(float, 4) MVLA_IND(float, 2) }
+#undef MVLA_IND
+    return cudaErrorInvalidConfiguration;
 }
 
 cudaError_t launch_patch_select(const BatchDesc& bd, const PatchParams& pp, const PatchIO& io, cudaStream_t stream)
 {
-    patch_select_kernel<<<bd.n, kPatchThreads, 0, stream>>>(bd, pp, io);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(bd.n);
+    cfg.blockDim = dim3(kPatchThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1] = {pdl_attribute()};
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, patch_select_kernel, bd, pp, io);
 }
 
 }  // namespace mvla
