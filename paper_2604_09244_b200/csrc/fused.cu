@@ -62,14 +62,14 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
 template <int TCOL, int NTILE>
 __global__ void __launch_bounds__(kFastThreads, 1)
 salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
-                     const __grid_constant__ CUtensorMap tmap_k, int n_heads, int head_dim, int npad,
+                     const __grid_constant__ CUtensorMap tmap_k, int n_heads, int head_dim, int npad_max,
                      float* __restrict__ part, int64_t part_stride, unsigned long long* __restrict__ acc64,
                      int* status, int free_running, const AlphaOut alpha)
 {
     constexpr int CC = TCOL * NTILE;
     extern __shared__ uint8_t dyn_smem_raw[];
     uint8_t* dyn_smem = dyn_smem_raw + ((1024u - (smem_u32(dyn_smem_raw) & 1023u)) & 1023u);   // swizzle atoms are 1 KB
-    __shared__ float s_m[kMaxText];                       // local max per query (log2 domain), -inf replaced by 0
+    __shared__ float s_m[kMaxText];                       // local max per query (scaled, log2 domain), -inf replaced by 0
     __shared__ float s_w[kMaxText];                       // final weight per query
     __shared__ float2 s_peer[kMaxCluster][kMaxText];      // (raw local max, local sum) of every CTA of the cluster
     __shared__ float2 s_loc[kMaxText];                    // this CTA's pairs, staged for the push
@@ -80,6 +80,8 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     const SampleDev& s = bd.s[blockIdx.z];
     const int h = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // queries padded to the MMA's N granularity for THIS sample (the launch is sized for the longest text)
+    const int npad = min(npad_max, (s.n_txt + 15) & ~15);
     const uint32_t crank = cluster_ctarank();
     const uint32_t csize = gridDim.x;
     const int d = head_dim;
@@ -175,11 +177,15 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
 #pragma unroll
         for (int i = 0; i < CC; ++i) L[i] = 0.f;
     }
+    // The registers keep the raw dot products; the scale enters with the exponent below (one FFMA).  Keys
+    // past the end of a ragged tile are masked; a full tile needs no pass over the registers at all, and
+    // columns past the padded query count are never looked at.
 #pragma unroll
     for (int t = 0; t < NTILE; ++t) {
+        if (ok && valid[t] == kKeyTile) continue;         // block-uniform
         const bool live = ok && tid < valid[t];
 #pragma unroll
-        for (int i = 0; i < TCOL; ++i) L[t * TCOL + i] = (live && i < npad) ? L[t * TCOL + i] * cscale : -CUDART_INF_F;
+        for (int i = 0; i < TCOL; ++i) L[t * TCOL + i] = live ? L[t * TCOL + i] : -CUDART_INF_F;
     }
 
     // ---- local maximum per query
@@ -199,7 +205,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     __syncthreads();
     float m_raw = -CUDART_INF_F;
     if (tid < npad) {
-        m_raw = fmaxf(fmaxf(s_wred[0][tid], s_wred[1][tid]), fmaxf(s_wred[2][tid], s_wred[3][tid]));
+        m_raw = fmaxf(fmaxf(s_wred[0][tid], s_wred[1][tid]), fmaxf(s_wred[2][tid], s_wred[3][tid])) * cscale;
         s_m[tid] = (m_raw == -CUDART_INF_F) ? 0.f : m_raw;
     }
     __syncthreads();
@@ -215,7 +221,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
             sum[i] = 0.f;
 #pragma unroll
             for (int t = 0; t < NTILE; ++t) {
-                const float e = ex2_approx(L[t * TCOL + qc * 16 + i] - mm);
+                const float e = ex2_approx(fmaf(L[t * TCOL + qc * 16 + i], cscale, -mm));
                 L[t * TCOL + qc * 16 + i] = e;
                 sum[i] += e;
             }
