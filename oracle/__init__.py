@@ -84,6 +84,8 @@ def load(path: str):
         sp, pp = C.POINTER(CSample), C.POINTER(CParams)
         L.oracle_salience.argtypes = [fp, fp, C.c_int32, C.c_int32, sp, dp]
         L.oracle_salience.restype = None
+        L.oracle_salience_gqa.argtypes = [fp, fp, C.c_int32, C.c_int32, C.c_int32, sp, dp]
+        L.oracle_salience_gqa.restype = None
         L.oracle_l1norm.argtypes = [fp, C.c_int32, sp, dp]
         L.oracle_l1norm.restype = None
         L.oracle_indicators.argtypes = [dp, dp, C.c_int32, C.c_int32, dp]
@@ -186,6 +188,17 @@ def salience(q, k, n_heads, head_dim, s) -> np.ndarray:
     cs = c_sample(s)
     out = np.zeros(cs.n_2d + cs.n_3d, dtype=np.float64)
     lib().oracle_salience(qp, kp, n_heads, head_dim, C.byref(cs), out.ctypes.data_as(C.POINTER(C.c_double)))
+    return out
+
+
+def salience_gqa(q, k, n_heads, n_kv_heads, head_dim, s) -> np.ndarray:
+    """q: [rows, H, d]; k: [rows, H_kv, d]."""
+    q, qp = _f32(q)
+    k, kp = _f32(k)
+    cs = c_sample(s)
+    out = np.zeros(cs.n_2d + cs.n_3d, dtype=np.float64)
+    lib().oracle_salience_gqa(qp, kp, n_heads, n_kv_heads, head_dim, C.byref(cs),
+                              out.ctypes.data_as(C.POINTER(C.c_double)))
     return out
 
 

@@ -27,8 +27,18 @@ static int32_t vis_row(const oracle_sample *s, int32_t j)
 void oracle_salience(const float *q, const float *k, int32_t n_heads, int32_t head_dim,
                      const oracle_sample *s, double *a_out)
 {
+    oracle_salience_gqa(q, k, n_heads, n_heads, head_dim, s, a_out);
+}
+
+/* The same with grouped key heads: K is [rows, n_kv_heads, d] and query head h reads key head
+ * h / (n_heads / n_kv_heads) (the usual grouped-query layout of the host models). */
+void oracle_salience_gqa(const float *q, const float *k, int32_t n_heads, int32_t n_kv_heads,
+                         int32_t head_dim, const oracle_sample *s, double *a_out)
+{
     const int32_t H = n_heads, d = head_dim, nt = s->n_txt, nv = s->n_2d + s->n_3d;
-    const int64_t row = (int64_t)H * d;
+    const int64_t row = (int64_t)H * d;                  /* elements of a Q row */
+    const int64_t krow = (int64_t)n_kv_heads * d;        /* elements of a K row */
+    const int32_t group = H / n_kv_heads;                /* query heads per key head */
     double *per_head = (double *)calloc((size_t)H * nv, sizeof(double));
 
 #pragma omp parallel for schedule(static)
@@ -39,7 +49,7 @@ void oracle_salience(const float *q, const float *k, int32_t n_heads, int32_t he
             /* logits l[h,i,j] = <q_hi, k_hj> / sqrt(d) */
             double mx = -INFINITY;
             for (int32_t j = 0; j < nv; ++j) {
-                const float *kj = k + ((int64_t)s->seq_off + vis_row(s, j)) * row + (int64_t)h * d;
+                const float *kj = k + ((int64_t)s->seq_off + vis_row(s, j)) * krow + (int64_t)(h / group) * d;
                 double acc = 0.0;
                 for (int32_t c = 0; c < d; ++c) acc += (double)qi[c] * (double)kj[c];
                 logit[j] = acc / sqrt((double)d);

@@ -83,6 +83,11 @@ typedef struct oracle_diag {
 void oracle_salience(const float *q, const float *k, int32_t n_heads, int32_t head_dim,
                      const oracle_sample *s, double *a_out);
 
+/* The same for grouped-query attention: k is [rows, n_kv_heads, d], n_heads a multiple of
+ * n_kv_heads, query head h attends through key head h / (n_heads / n_kv_heads). */
+void oracle_salience_gqa(const float *q, const float *k, int32_t n_heads, int32_t n_kv_heads,
+                         int32_t head_dim, const oracle_sample *s, double *a_out);
+
 /* Sec. 3.1.2: L1 norm of each visual token's feature row.  hidden: [rows, D]. */
 void oracle_l1norm(const float *hidden, int32_t d_model, const oracle_sample *s, double *n_out);
 

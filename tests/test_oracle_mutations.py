@@ -21,8 +21,10 @@ MUTATIONS = {
     "logit scale dropped": ("logit[j] = acc / sqrt((double)d);", "logit[j] = acc;"),
     "logit sign flipped": ("acc += (double)qi[c] * (double)kj[c];", "acc -= (double)qi[c] * (double)kj[c];"),
     "query head offset wrong": ("+ s->off_txt + i) * row + (int64_t)h * d;", "+ s->off_txt + i) * row + (int64_t)h;"),
-    "key row ignores the sample offset": ("const float *kj = k + ((int64_t)s->seq_off + vis_row(s, j)) * row",
-                                          "const float *kj = k + ((int64_t)vis_row(s, j)) * row"),
+    "key row ignores the sample offset": ("const float *kj = k + ((int64_t)s->seq_off + vis_row(s, j)) * krow",
+                                          "const float *kj = k + ((int64_t)vis_row(s, j)) * krow"),
+    "grouped key head taken modulo": ("(int64_t)(h / group) * d;", "(int64_t)(h % n_kv_heads) * d;"),
+    "key row stride of the query tensor": ("const int64_t krow = (int64_t)n_kv_heads * d;", "const int64_t krow = (int64_t)H * d;"),
     "mean over heads only": ("a_out[j] = acc / ((double)H * (double)nt);", "a_out[j] = acc / ((double)H);"),
     "softmax denominator over 2D keys only": ("for (int32_t j = 0; j < nv; ++j) den += exp(logit[j] - mx);",
                                               "for (int32_t j = 0; j < s->n_2d; ++j) den += exp(logit[j] - mx);"),

@@ -191,6 +191,22 @@ def test_segments_in_any_order_3d_text_2d():
 
 
 # ---------------------------------------------------------------- L1 norms, indicators
+def test_salience_grouped_key_heads_equal_repeated_keys():
+    # grouped-query attention is plain attention on keys repeated per group (numpy's repeat is the definition)
+    rng = np.random.default_rng(41)
+    H, Hkv, d = 6, 2, 8
+    for text_first in (False, True):
+        s = S(3, 5, 7, seq_off=2, text_first=text_first)
+        rows = s.seq_off + s.seq_len
+        q = rng.standard_normal((rows, H, d)).astype(np.float32)
+        k = rng.standard_normal((rows, Hkv, d)).astype(np.float32)
+        a = oracle.salience_gqa(q, k, H, Hkv, d, s)
+        np.testing.assert_allclose(a, oracle.salience(q, np.repeat(k, H // Hkv, axis=1), H, d, s), rtol=1e-14)
+        assert a.sum() == pytest.approx(1.0, rel=1e-13)
+    np.testing.assert_array_equal(oracle.salience_gqa(q, np.repeat(k, 3, axis=1), H, H, d, s),
+                                  oracle.salience(q, np.repeat(k, 3, axis=1), H, d, s))
+
+
 def test_l1norm_closed_forms():
     s = S(2, 3, 4, seq_off=1)
     D = 6
