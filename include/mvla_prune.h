@@ -19,7 +19,8 @@
  *   - No function synchronises the stream; work is enqueued on `stream` (a cudaStream_t passed
  *     as void*, NULL = the legacy default stream).  Host arrays (`samples`) are consumed before
  *     the call returns.  The library keeps no caller pointer beyond the enqueued work.
- *   - Input tensors are token-major and packed ragged: Q, K, V are [rows, n_heads, head_dim],
+ *   - Input tensors are token-major and packed ragged: Q is [rows, n_heads, head_dim], K and V are
+ *     [rows, n_kv_heads, head_dim] (n_kv_heads == n_heads unless the configuration groups them),
  *     hidden is [rows, d_model], rows contiguous, dtype as given at create.  A sample owns the
  *     rows [seq_off, seq_off + n_txt + n_2d + n_3d) split in three contiguous segments.
  *     Base pointers must be 16-byte aligned.
@@ -84,7 +85,7 @@ typedef struct mvla_ctx mvla_ctx;   /* opaque */
 typedef struct mvla_config {
     int32_t device;            /* CUDA device ordinal */
     int32_t dtype;             /* MVLA_DTYPE_*: element type of q, k, v, hidden */
-    int32_t n_heads;           /* H; k/v heads == q heads */
+    int32_t n_heads;           /* H: query heads (key / value heads: n_kv_heads below) */
     int32_t head_dim;          /* d: 64 or 128 */
     int32_t d_model;           /* D: hidden width, multiple of 8 (bf16) / 4 (fp32) */
     int32_t max_batch;         /* capacity: samples per call */
@@ -107,6 +108,9 @@ typedef struct mvla_config {
     int32_t patch_path;        /* 1: allocate the per-patch state and the attention scratch
                                   (n_heads x max_text x max_batch x (max_2d + max_3d) floats) */
     int32_t kmeans_max_iter;   /* rounds of the 1-D K-Means (Sec. 4.2); 0 -> 32 */
+    int32_t n_kv_heads;        /* grouped-query attention: k and v are [rows, n_kv_heads, head_dim] and query head h
+                                  reads key head h / (n_heads / n_kv_heads); 0 -> n_heads.  Must divide n_heads.
+                                  Not available together with patch_path */
 } mvla_config;
 
 /* One batch element (host array).  Offsets are rows relative to seq_off; the three segments

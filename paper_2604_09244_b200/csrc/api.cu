@@ -20,6 +20,7 @@ struct mvla_ctx {
     int max_vis;
     size_t elem;                 // bytes per input element
     bool use_umma;               // bf16 tensor-core salience path
+    int kv_heads;                // key / value heads (== n_heads unless grouped)
     float* part;                 // [H][max_batch * max_vis] per-head partial scores
     int64_t part_stride;
     float* attn_ws;              // [max_batch * max_vis]
@@ -223,9 +224,9 @@ int32_t tensor_map(mvla_ctx* ctx, int which, const void* ptr, int64_t rows, int 
         return MVLA_OK;
     }
     const mvla_config& c = ctx->cfg;
-    cuuint64_t dims[3] = {static_cast<cuuint64_t>(c.head_dim), static_cast<cuuint64_t>(c.n_heads),
-                          static_cast<cuuint64_t>(rows)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(c.head_dim) * 2, static_cast<cuuint64_t>(c.head_dim) * c.n_heads * 2};
+    const cuuint64_t heads = static_cast<cuuint64_t>(which == 1 ? ctx->kv_heads : c.n_heads);   // map 1 is the key tensor
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(c.head_dim), heads, static_cast<cuuint64_t>(rows)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(c.head_dim) * 2, static_cast<cuuint64_t>(c.head_dim) * heads * 2};
     cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(box_rows)};
     cuuint32_t estr[3] = {1, 1, 1};
     const CUresult r = ctx->encode(&ctx->tm[which], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims,
@@ -277,11 +278,11 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
     if (fast) {
-        e = launch_salience_fast(bd, c.n_heads, c.head_dim, tq, tk, tiles_per_cta, cluster, npad, ctx->part,
+        e = launch_salience_fast(bd, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, tq, tk, tiles_per_cta, cluster, npad, ctx->part,
                                  ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, st);
         if (used_acc64) *used_acc64 = acc64 != nullptr;
     } else {
-        e = launch_salience(bd, c.dtype, c.n_heads, c.head_dim, q, k, tq, tk, ctx->use_umma, tiles_per_cta,
+        e = launch_salience(bd, c.dtype, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, q, k, tq, tk, ctx->use_umma, tiles_per_cta,
                             cluster, npad, ctx->part, ctx->part_stride, ctx->status_dev, alpha, st);
     }
     if (e == cudaErrorInvalidConfiguration) return MVLA_ERR_UNSUPPORTED;
@@ -416,7 +417,7 @@ int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, cons
     int64_t cap = 0;                               // the row count is known only on the device: cover the capacity
     for (int b = 0; b < batch; ++b) cap += samples[b].n_txt + samples[b].n_2d + samples[b].n_3d;
     CompactJob job;
-    const int32_t kv_bytes = static_cast<int32_t>(ctx->cfg.n_heads * ctx->cfg.head_dim * ctx->elem);
+    const int32_t kv_bytes = static_cast<int32_t>(ctx->kv_heads * ctx->cfg.head_dim * ctx->elem);
     for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
     job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
     for (int first = 0; first < batch; first += kMaxChunk) {
@@ -449,6 +450,8 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if ((c.patch_path != 0 && c.patch_path != 1) || c.kmeans_max_iter < 0 || !(c.obj_2d_min >= 0.0 && c.obj_2d_min <= 1.0))
         return MVLA_ERR_INVALID_ARG;
     if (c.head_dim != 64 && c.head_dim != 128) return MVLA_ERR_UNSUPPORTED;
+    if (c.n_kv_heads < 0 || (c.n_kv_heads > 0 && (c.n_kv_heads > c.n_heads || c.n_heads % c.n_kv_heads != 0))) return MVLA_ERR_INVALID_ARG;
+    if (c.patch_path && c.n_kv_heads > 0 && c.n_kv_heads != c.n_heads) return MVLA_ERR_UNSUPPORTED;   // the patch path is built for ungrouped keys
     if (c.max_text > kMaxText || c.max_2d + c.max_3d > kMaxVis || c.max_batch > 64) return MVLA_ERR_UNSUPPORTED;
     const size_t elem = c.dtype == MVLA_DTYPE_BF16 ? 2 : 4;
     if ((static_cast<size_t>(c.d_model) * elem) % 16 != 0) return MVLA_ERR_UNSUPPORTED;
@@ -471,6 +474,7 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     ctx->max_vis = c.max_2d + c.max_3d;
     ctx->elem = elem;
     ctx->use_umma = c.dtype == MVLA_DTYPE_BF16;
+    ctx->kv_heads = c.n_kv_heads > 0 ? c.n_kv_heads : c.n_heads;
     if (c.salience_path == MVLA_SALIENCE_FMA) ctx->use_umma = false;
     ctx->part = ctx->attn_ws = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
     ctx->acc64 = nullptr;
@@ -662,7 +666,7 @@ int32_t mvla_compact(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, c
     rc = make_plan(ctx, 0, batch, samples, MVLA_MODE_FIXED, 0, false, &plan);
     if (rc != MVLA_OK) return rc;
     CompactJob job;
-    const int32_t kv_bytes = static_cast<int32_t>(ctx->cfg.n_heads * ctx->cfg.head_dim * ctx->elem);
+    const int32_t kv_bytes = static_cast<int32_t>(ctx->kv_heads * ctx->cfg.head_dim * ctx->elem);
     for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
     job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -751,7 +755,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     const bool adaptive = mode == MVLA_MODE_ADAPTIVE;
     const GateParams gp = gate_params(ctx, mode, adaptive);
     CompactJob job;
-    const int32_t kv_bytes = static_cast<int32_t>(ctx->cfg.n_heads * ctx->cfg.head_dim * ctx->elem);
+    const int32_t kv_bytes = static_cast<int32_t>(ctx->kv_heads * ctx->cfg.head_dim * ctx->elem);
     for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
     job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
 
@@ -777,6 +781,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     const unsigned par = ctx->step_parity;
     const size_t nvis_b = static_cast<size_t>(plan.total_vis), nout_b = static_cast<size_t>(plan.total_out);
     const size_t hb = static_cast<size_t>(ctx->cfg.d_model) * ctx->elem, kb = static_cast<size_t>(kv_bytes);
+    const size_t qb = static_cast<size_t>(ctx->cfg.n_heads) * ctx->cfg.head_dim * ctx->elem;
     if ((flags & MVLA_FLAG_INPUTS_STABLE) && batch <= kMaxChunk && chunk_is_fast(ctx, chunk_of(plan, 0, batch))) {
         cudaStreamCaptureStatus cst = cudaStreamCaptureStatusNone;
         if (cudaStreamGetCaptureInfo(st, &cst, &cap_id) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
@@ -788,7 +793,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
             range_of(out->kept_idx, nout_b * 4), range_of(out->out_offsets, (batch + 1) * 4u),
             range_of(out->budgets, batch * 8u), range_of(out->attn, nvis_b * 4), range_of(out->ahat, nvis_b * 4),
             range_of(out->z, nvis_b * 4), range_of(out->diag, batch * sizeof(mvla_diag)),
-            range_of(in->q, in_rows * kb), range_of(in->k, in_rows * kb),
+            range_of(in->q, in_rows * qb), range_of(in->k, in_rows * kb),
             range_of(adaptive ? in->hidden : nullptr, in_rows * hb)};
         bool clash = ctx->hist_unknown;
         for (unsigned s = 0; !clash && s < kSets; ++s) {

@@ -93,7 +93,9 @@ struct AlphaOut {
 };
 
 bool fast_salience_supported(int tiles_per_cta);
-cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int head_dim, const CUtensorMap* tmap_q,
+// `kv_group`: query heads per key head (1 unless the keys are grouped); the key tensor map then has
+// n_heads / kv_group heads.
+cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
                                  bool free_running, AlphaOut alpha, cudaStream_t stream);
@@ -101,7 +103,7 @@ cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int head_dim,
 
 // Salience: per-head partial scores part[h][vis] (already scaled by 1/(H n_t)).
 // `use_umma`: tensor-core path (bf16 only).  tmaps: device-usable tensor maps (passed by value).
-cudaError_t launch_salience(const BatchDesc& bd, int dtype, int n_heads, int head_dim,
+cudaError_t launch_salience(const BatchDesc& bd, int dtype, int n_heads, int kv_group, int head_dim,
                             const void* q, const void* k, const CUtensorMap* tmap_q,
                             const CUtensorMap* tmap_k, bool use_umma, int tiles_per_cta,
                             int cluster, int npad, float* part, int64_t part_stride,

@@ -62,7 +62,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
 template <int TCOL, int NTILE>
 __global__ void __launch_bounds__(kFastThreads, 1)
 salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
-                     const __grid_constant__ CUtensorMap tmap_k, int n_heads, int head_dim, int npad_max,
+                     const __grid_constant__ CUtensorMap tmap_k, int n_heads, int kv_group, int head_dim, int npad_max,
                      float* __restrict__ part, int64_t part_stride, unsigned long long* __restrict__ acc64,
                      int* status, int free_running, const AlphaOut alpha)
 {
@@ -127,7 +127,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
             if (valid[t] <= 0) continue;
             const int row0 = tile_info(s, tt0 + t).row0;
             for (int kh = 0; kh < khalves; ++kh)
-                tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * 64, h, row0, bar_full);
+                tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * 64, h / kv_group, row0, bar_full);
         }
     }
     if (tid < kMaxText) s_w[tid] = 0.f;
@@ -291,7 +291,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
 }
 
 template <int TCOL, int NTILE>
-cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int head_dim, const CUtensorMap* tq,
+cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, const CUtensorMap* tq,
                           const CUtensorMap* tk, int cluster, int npad, float* part, int64_t part_stride,
                           unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, cudaStream_t stream)
 {
@@ -312,14 +312,14 @@ cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int head_dim, const 
     attr[1] = pdl_attribute();
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, head_dim, npad, part, part_stride, acc64, status, free_running, alpha);
+    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, kv_group, head_dim, npad, part, part_stride, acc64, status, free_running, alpha);
 }
 
 }  // namespace
 
 bool fast_salience_supported(int tiles_per_cta) { return tiles_per_cta >= 1 && tiles_per_cta <= 2; }
 
-cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int head_dim, const CUtensorMap* tmap_q,
+cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
                                  bool free_running, AlphaOut alpha, cudaStream_t stream)
@@ -327,7 +327,7 @@ cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int head_dim,
     const int tcol = npad <= 16 ? 16 : (npad <= 32 ? 32 : 64);
 #define MVLA_FAST(TC, NTL)                                                                                      \
     if (tcol == TC && tiles_per_cta == NTL)                                                                     \
-        return launch_fast_t<TC, NTL>(bd, n_heads, head_dim, tmap_q, tmap_k, cluster, npad, part, part_stride, \
+        return launch_fast_t<TC, NTL>(bd, n_heads, kv_group, head_dim, tmap_q, tmap_k, cluster, npad, part, part_stride, \
                                       acc64, status, free_running ? 1 : 0, alpha, stream);
     MVLA_FAST(16, 1) MVLA_FAST(32, 1) MVLA_FAST(64, 1) MVLA_FAST(16, 2) MVLA_FAST(32, 2) MVLA_FAST(64, 2)
 #undef MVLA_FAST

@@ -25,7 +25,7 @@ template <typename T, bool UMMA>
 __global__ void __launch_bounds__(kThreads, 1)
 salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
                 const __grid_constant__ CUtensorMap tmap_k, const T* __restrict__ q,
-                const T* __restrict__ k, int n_heads, int head_dim, int tiles_per_cta, int npad,
+                const T* __restrict__ k, int n_heads, int kv_group, int head_dim, int tiles_per_cta, int npad,
                 float* __restrict__ part, int64_t part_stride, int* status, const AlphaOut alpha)
 {
     extern __shared__ uint8_t dyn_smem_raw[];
@@ -45,6 +45,8 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
     const uint32_t csize = gridDim.x;
     const int d = head_dim;
     const int64_t row_elems = static_cast<int64_t>(n_heads) * d;
+    const int64_t kv_row_elems = static_cast<int64_t>(n_heads / kv_group) * d;   // grouped key heads: K rows are narrower
+    const int hk = h / kv_group;                                                 // the key head this query head reads
     // logits are kept in the log2 domain: y = <q, k> * log2(e) / sqrt(d)
     const float cscale = 1.4426950408889634f * rsqrtf(static_cast<float>(d));
     const int tt0 = static_cast<int>(crank) * tiles_per_cta;
@@ -79,7 +81,7 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
                 const TileInfo ti = tile_info(s, tt0 + t);
                 if (ti.valid <= 0) continue;
                 for (int kh = 0; kh < khalves; ++kh)
-                    tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * 64, h, ti.row0, bar_full);
+                    tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * 64, hk, ti.row0, bar_full);
             }
         }
         if (warp == 1) tmem_alloc(smem_u32(&s_tmem), tmem_cols);
@@ -135,7 +137,7 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
             for (int idx = tid; idx < kKeyTile * d; idx += kThreads) {
                 const int r = idx / d, c = idx - r * d;
                 Ks[r * kp + c] = r < ti.valid
-                    ? to_f32(k[static_cast<int64_t>(ti.row0 + r) * row_elems + static_cast<int64_t>(h) * d + c])
+                    ? to_f32(k[static_cast<int64_t>(ti.row0 + r) * kv_row_elems + static_cast<int64_t>(hk) * d + c])
                     : 0.f;
             }
             __syncthreads();
@@ -323,7 +325,7 @@ l1norm_kernel(const __grid_constant__ BatchDesc bd, int d_model, const T* __rest
 }
 
 template <typename T, bool UMMA>
-cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int head_dim, const void* q, const void* k,
+cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, const void* q, const void* k,
                               const CUtensorMap* tq, const CUtensorMap* tk, int tiles_per_cta, int cluster,
                               int npad, float* part, int64_t part_stride, int* status, AlphaOut alpha,
                               cudaStream_t stream)
@@ -352,25 +354,25 @@ cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int head_dim, co
     cfg.numAttrs = 1;
     static const CUtensorMap zero_map = {};
     return cudaLaunchKernelEx(&cfg, kern, bd, tq ? *tq : zero_map, tk ? *tk : zero_map,
-                              static_cast<const T*>(q), static_cast<const T*>(k), n_heads, head_dim,
+                              static_cast<const T*>(q), static_cast<const T*>(k), n_heads, kv_group, head_dim,
                               tiles_per_cta, npad, part, part_stride, status, alpha);
 }
 
 }  // namespace
 
-cudaError_t launch_salience(const BatchDesc& bd, int dtype, int n_heads, int head_dim, const void* q,
+cudaError_t launch_salience(const BatchDesc& bd, int dtype, int n_heads, int kv_group, int head_dim, const void* q,
                             const void* k, const CUtensorMap* tmap_q, const CUtensorMap* tmap_k,
                             bool use_umma, int tiles_per_cta, int cluster, int npad, float* part,
                             int64_t part_stride, int* status, AlphaOut alpha, cudaStream_t stream)
 {
     if (dtype == MVLA_DTYPE_BF16) {
         if (use_umma)
-            return launch_salience_t<__nv_bfloat16, true>(bd, n_heads, head_dim, q, k, tmap_q, tmap_k, tiles_per_cta,
+            return launch_salience_t<__nv_bfloat16, true>(bd, n_heads, kv_group, head_dim, q, k, tmap_q, tmap_k, tiles_per_cta,
                                                           cluster, npad, part, part_stride, status, alpha, stream);
-        return launch_salience_t<__nv_bfloat16, false>(bd, n_heads, head_dim, q, k, nullptr, nullptr, tiles_per_cta,
+        return launch_salience_t<__nv_bfloat16, false>(bd, n_heads, kv_group, head_dim, q, k, nullptr, nullptr, tiles_per_cta,
                                                        cluster, npad, part, part_stride, status, alpha, stream);
     }
-    return launch_salience_t<float, false>(bd, n_heads, head_dim, q, k, nullptr, nullptr, tiles_per_cta, cluster,
+    return launch_salience_t<float, false>(bd, n_heads, kv_group, head_dim, q, k, nullptr, nullptr, tiles_per_cta, cluster,
                                            npad, part, part_stride, status, alpha, stream);
 }
 

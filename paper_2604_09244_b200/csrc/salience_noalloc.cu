@@ -152,7 +152,7 @@ extern "C" int32_t mvla_salience_noalloc(int32_t device, int32_t dtype, int32_t 
             const int tiles_per_cta = (max_tiles + kMaxCluster - 1) / kMaxCluster;
             const int cluster = (max_tiles + tiles_per_cta - 1) / tiles_per_cta;
             const int npad = (max_txt + 15) / 16 * 16;
-            const cudaError_t e = launch_salience(bd, dtype, n_heads, head_dim, q, k, umma ? &tq : nullptr,
+            const cudaError_t e = launch_salience(bd, dtype, n_heads, 1, head_dim, q, k, umma ? &tq : nullptr,
                                                   umma ? &tk : nullptr, umma, tiles_per_cta, cluster, npad, sc->part,
                                                   total_vis, sc->flag, AlphaOut{nullptr, 0, 0}, st);
             if (e == cudaErrorInvalidConfiguration) rc = MVLA_ERR_UNSUPPORTED;

@@ -49,7 +49,7 @@ class Config(C.Structure):
                 ("salience_path", C.c_int32),
                 ("tau_2d", C.c_double), ("tau_3d", C.c_double), ("beta", C.c_double),
                 ("eps_3d", C.c_double), ("floor_ratio", C.c_double), ("obj_2d_min", C.c_double),
-                ("patch_path", C.c_int32), ("kmeans_max_iter", C.c_int32)]
+                ("patch_path", C.c_int32), ("kmeans_max_iter", C.c_int32), ("n_kv_heads", C.c_int32)]
 
 
 class CSample(C.Structure):
@@ -172,7 +172,7 @@ class PruneContext:
                  beta: float = 0.85, window_k: int = 7, eps_3d: float = 0.02,
                  floor_ratio: float = 0.10, cold_start_full_keep: int = 1,
                  salience_path: int = SALIENCE_AUTO, device: Optional[int] = None, patch_path: int = 0,
-                 obj_2d_min: float = 0.5, kmeans_max_iter: int = 32):
+                 obj_2d_min: float = 0.5, kmeans_max_iter: int = 32, n_kv_heads: int = 0):
         self._h = C.c_void_p()
         self._lib = lib()
         if device is None:
@@ -183,7 +183,7 @@ class PruneContext:
         self.cfg = Config(device, code, n_heads, head_dim, d_model, max_batch, max_text, max_2d,
                           max_3d, n_prune_points, n_state_slots, window_k, cold_start_full_keep,
                           salience_path, tau_2d, tau_3d, beta, eps_3d, floor_ratio, obj_2d_min, patch_path,
-                          kmeans_max_iter)
+                          kmeans_max_iter, n_kv_heads)
         rc = self._lib.mvla_prune_create(C.byref(self.cfg), C.byref(self._h))
         if rc != OK:
             self._h = C.c_void_p()
@@ -210,8 +210,8 @@ class PruneContext:
         mk = lambda *shape, dtype=dt: torch.empty(*shape, dtype=dtype, device=dev)
         return StepOutputs(
             out_hidden=mk(rows, c.d_model) if hidden else None,
-            out_k=mk(rows, c.n_heads, c.head_dim) if kv else None,
-            out_v=mk(rows, c.n_heads, c.head_dim) if kv else None,
+            out_k=mk(rows, c.n_kv_heads or c.n_heads, c.head_dim) if kv else None,
+            out_v=mk(rows, c.n_kv_heads or c.n_heads, c.head_dim) if kv else None,
             kept_idx=mk(rows, dtype=torch.int32),
             out_offsets=mk(len(samples) + 1, dtype=torch.int32),
             budgets=mk(len(samples), 2, dtype=torch.int32),
@@ -328,7 +328,8 @@ def context_for(wl, *, max_batch=None, n_prune_points=1, n_state_slots=0, salien
                         salience_path=salience_path, device=device,
                         patch_path=int(wl.mode == MODE_PATCH) if patch_path is None else patch_path,
                         obj_2d_min=wl.extra.get("obj_2d_min", 0.5),
-                        kmeans_max_iter=wl.extra.get("kmeans_max_iter", 32))
+                        kmeans_max_iter=wl.extra.get("kmeans_max_iter", 32),
+                        n_kv_heads=wl.extra.get("n_kv_heads", 0))
 
 
 def to_device(arr, dtype: str, device) -> torch.Tensor:

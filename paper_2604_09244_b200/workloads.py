@@ -134,23 +134,24 @@ def layout_2d_3d_txt(seq_off: int, n_txt: int, n_2d: int, n_3d: int, **kw) -> Sa
 # --------------------------------------------------------------------------
 # drawing
 # --------------------------------------------------------------------------
-def _draw_weights(rng: np.random.Generator, D: int, out: int = 0):
+def _draw_weights(rng: np.random.Generator, D: int, out: int = 0, out_kv: int = 0):
     out = out or D          # projection width H*d (equal to D in the paper-shaped workloads)
+    out_kv = out_kv or out  # narrower when the key / value heads are grouped
     std = 1.0 / np.sqrt(D)
     wq = rng.standard_normal((D, out), dtype=np.float32) * np.float32(std)
-    wk = rng.standard_normal((D, out), dtype=np.float32) * np.float32(std)
-    wv = rng.standard_normal((D, out), dtype=np.float32) * np.float32(std)
+    wk = rng.standard_normal((D, out_kv), dtype=np.float32) * np.float32(std)
+    wv = rng.standard_normal((D, out_kv), dtype=np.float32) * np.float32(std)
     return wq, wk, wv
 
 
-def _project(hidden: np.ndarray, w, H: int, d: int, dtype: str) -> Tensors:
+def _project(hidden: np.ndarray, w, H: int, d: int, dtype: str, H_kv: int = 0) -> Tensors:
     """hidden is fp32 (not yet rounded).  Projections are taken from the
     unrounded fp32 hidden, then all four tensors are rounded once."""
     wq, wk, wv = w
     S = hidden.shape[0]
     q = (hidden @ wq).reshape(S, H, d)
-    k = (hidden @ wk).reshape(S, H, d)
-    v = (hidden @ wv).reshape(S, H, d)
+    k = (hidden @ wk).reshape(S, H_kv or H, d)
+    v = (hidden @ wv).reshape(S, H_kv or H, d)
     return Tensors(hidden=round_to_dtype(hidden, dtype), q=round_to_dtype(q, dtype),
                    k=round_to_dtype(k, dtype), v=round_to_dtype(v, dtype))
 
@@ -314,7 +315,7 @@ def config5_action_iteration(seed: int = 4, T: int = 16, D=4096, H=32, d=128, dt
 def small_workload(seed: int, *, batch=2, D=256, H=4, d=64, dtype="bf16", mode=MODE_ADAPTIVE,
                    n_txt=(5, 19), n_2d=(70, 130), n_3d=(150, 37), keep=(0.4, 0.3),
                    keep_fixed=(0.4, 0.3), steps=1, cold_start=0, text_first=False, scale_3d: float = 1.0,
-                   spike_frac=0.05) -> Workload:
+                   spike_frac=0.05, n_kv_heads: int = 0) -> Workload:
     """Small ragged cases for parity tests: arbitrary segment lengths (several
     128-key tiles plus a ragged tail), optional [text | 2D | 3D] order, an
     optional scale on the 3D hidden rows (to move the feature-norm share), and
@@ -335,7 +336,7 @@ def small_workload(seed: int, *, batch=2, D=256, H=4, d=64, dtype="bf16", mode=M
         samples.append(s)
         off += s.seq_len
     hidden = rng.standard_normal((off, D), dtype=np.float32)
-    w = _draw_weights(rng, D, H * d)
+    w = _draw_weights(rng, D, H * d, n_kv_heads * d)
     for s in samples:
         if spike_frac > 0:
             hidden[s.seq_off + _spike_rows(rng, s, spike_frac)] *= np.float32(4.0)
@@ -346,9 +347,10 @@ def small_workload(seed: int, *, batch=2, D=256, H=4, d=64, dtype="bf16", mode=M
         if t > 0:
             rows = np.sort(rng.choice(off, size=max(1, _rhu(0.10 * off)), replace=False))
             hidden[rows] += rng.standard_normal((len(rows), D), dtype=np.float32) * np.float32(0.1)
-        out.append(_project(hidden.copy(), w, H, d, dtype))
+        out.append(_project(hidden.copy(), w, H, d, dtype, n_kv_heads))
     return Workload(f"small_{seed}", dtype, H, d, D, mode, samples, out,
-                    cold_start_full_keep=cold_start, seed=seed)
+                    cold_start_full_keep=cold_start, seed=seed,
+                    extra={"n_kv_heads": n_kv_heads} if n_kv_heads else {})
 
 def patch_workload(seed: int = 5, *, batch: int = 1, D=4096, H=32, d=128, dtype="bf16", n_txt=(32,),
                    n_patch=(256,), steps: int = 1, cold_start: int = 0, text_first: bool = False) -> Workload:

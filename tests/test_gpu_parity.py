@@ -8,8 +8,8 @@ import torch
 import oracle
 from paper_2604_09244_b200 import mvla
 from paper_2604_09244_b200 import workloads as W
-from parity_util import (assert_salience_close, check_compaction, device_tensors, diag_records,
-                         run_and_check_step)
+from parity_util import (assert_salience_close, check_compaction, check_kept_against_oracle,
+                         check_stagewise_exact, device_tensors, diag_records, run_and_check_step)
 
 pytestmark = pytest.mark.gpu
 
@@ -432,4 +432,33 @@ def test_step_segments_in_order_3d_text_2d():
                     samples, [ten])
     ctx = mvla.context_for(wl)
     out, refs = run_and_check_step(ctx, wl, 0, _fresh_states(wl))
+    ctx.close()
+
+
+@pytest.mark.parametrize("dtype,path", [("bf16", mvla.SALIENCE_AUTO), ("bf16", mvla.SALIENCE_FMA), ("fp32", mvla.SALIENCE_AUTO)])
+def test_grouped_key_heads(dtype, path):
+    # 8 query heads read 2 key heads: K and V rows are a quarter as wide as Q rows
+    wl = W.small_workload(17, batch=2, D=256, H=8, d=64, dtype=dtype, mode=W.MODE_FIXED, n_txt=(9, 33),
+                          n_2d=(130, 70), n_3d=(150, 300), n_kv_heads=2)
+    t = wl.steps[0]
+    assert t.k.shape[1] == 2 and t.q.shape[1] == 8
+    ctx = mvla.context_for(wl, salience_path=path)
+    dev = device_tensors(wl)
+    attn, _ = ctx.salience(wl.samples, dev["q"], dev["k"])
+    out = ctx.prune_step(0, wl.samples, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"])
+    torch.cuda.synchronize()
+    attn, attn_step = attn.cpu().numpy(), out.attn.cpu().numpy()
+    offs, kept_all, budgets = out.out_offsets.cpu().numpy(), out.kept_idx.cpu().numpy(), out.budgets.cpu().numpy()
+    vis = 0
+    for b, s in enumerate(wl.samples):
+        ref = oracle.salience_gqa(t.q, t.k, 8, 2, 64, s)
+        assert_salience_close(attn[vis:vis + s.n_vis], ref, "stand-alone scores")
+        assert_salience_close(attn_step[vis:vis + s.n_vis], ref, "scores of the fused step")
+        k2, k3 = oracle.budget_fixed(s)
+        assert (int(budgets[b, 0]), int(budgets[b, 1])) == (k2, k3)
+        kept = kept_all[offs[b]:offs[b + 1]]
+        check_kept_against_oracle(s, kept, k2, k3, oracle.normalise(ref, s.n_2d, s.n_3d))
+        check_stagewise_exact(s, kept, k2, k3, out.ahat.cpu().numpy()[vis:vis + s.n_vis])
+        check_compaction(t, out, s, kept, int(offs[b]), wl.dtype)        # K / V rows of 2 x 64 elements
+        vis += s.n_vis
     ctx.close()
