@@ -283,6 +283,7 @@ __global__ void head_reduce_kernel(const float* __restrict__ part, int64_t part_
                                    int total_vis, float* __restrict__ attn)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_wait();                               // launched while the scoring kernel still runs: wait for its partials
     if (j >= total_vis) return;
     float acc = 0.f;
     for (int h = 0; h < n_heads; ++h) acc += part[static_cast<int64_t>(h) * part_stride + j];
@@ -380,8 +381,14 @@ cudaError_t launch_head_reduce(const float* part, int64_t part_stride, int n_hea
                                cudaStream_t stream)
 {
     if (total_vis <= 0) return cudaSuccess;
-    head_reduce_kernel<<<(total_vis + 255) / 256, 256, 0, stream>>>(part, part_stride, n_heads, total_vis, attn);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((total_vis + 255) / 256);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1] = {pdl_attribute()};
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, head_reduce_kernel, part, part_stride, n_heads, total_vis, attn);
 }
 
 cudaError_t launch_l1norm(const BatchDesc& bd, int dtype, int d_model, const void* hidden, float* l1,

@@ -5,7 +5,7 @@
 namespace mvla {
 namespace {
 
-constexpr int kSelThreads = 1024;
+constexpr int kSelThreads = 512;
 
 __global__ void __launch_bounds__(kSelThreads, 1)
 select_kernel(const __grid_constant__ BatchDesc bd, const GateParams gp, const SelectIO io)

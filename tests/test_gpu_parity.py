@@ -462,3 +462,11 @@ def test_grouped_key_heads(dtype, path):
         check_compaction(t, out, s, kept, int(offs[b]), wl.dtype)        # K / V rows of 2 x 64 elements
         vis += s.n_vis
     ctx.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_head_dim_256(dtype):
+    wl = W.small_workload(19, batch=2, D=512, H=2, d=256, dtype=dtype, n_txt=(7, 30), n_2d=(140, 60), n_3d=(100, 270))
+    ctx = mvla.context_for(wl)
+    run_and_check_step(ctx, wl, 0, [oracle.State(s.n_vis) for s in wl.samples])
+    ctx.close()
