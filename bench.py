@@ -44,8 +44,14 @@ def measured_peaks():
 
 # DRAM bytes (read + write) per launch of the stage's main kernel from one ncu capture of this benchmark
 # (profiles/), valid only for the kernel sources they were taken on: the digest below is over csrc/.
-NCU_CSRC_SHA256 = ""
-NCU_TRAFFIC = {}            # (workload, stage) -> bytes per launch
+NCU_CSRC_SHA256 = "72429f42da935634b2151818e7eaa0c02df1ba71fe8a59f436d41dd27a449f70"
+NCU_TRAFFIC = {             # (workload, stage) -> dram__bytes_read.sum + dram__bytes_write.sum per launch
+    ("config2", "salience"): 6621440,      # salience_fast_kernel<32,1>
+    ("config2", "select"): 76544,          # select_kernel
+    ("config2", "compact"): 7085440,       # compact_kernel: the written half is still in L2 when the kernel ends
+    ("patch_mla", "salience"): 4516736 + 6316800,   # salience_fast_kernel + patch_indicators_kernel
+    ("patch_mla", "select"): 61696,        # patch_select_kernel
+}
 
 
 def csrc_digest() -> str:

@@ -86,7 +86,7 @@ typedef struct mvla_config {
     int32_t device;            /* CUDA device ordinal */
     int32_t dtype;             /* MVLA_DTYPE_*: element type of q, k, v, hidden */
     int32_t n_heads;           /* H: query heads (key / value heads: n_kv_heads below) */
-    int32_t head_dim;          /* d: 64, 128 or 256 */
+    int32_t head_dim;          /* d: a multiple of 32 from 64 to 256 (64, 96, 128, ... 256) */
     int32_t d_model;           /* D: hidden width, multiple of 8 (bf16) / 4 (fp32) */
     int32_t max_batch;         /* capacity: samples per call */
     int32_t max_text;          /* capacity: text tokens per sample, <= 64 */
@@ -185,7 +185,7 @@ typedef struct mvla_outputs {
 /*
  * Create a context on cfg->device: workspace, smoothed state for n_prune_points x
  * n_state_slots episodes, a device status word.  Supported: dtype bf16 or fp32,
- * head_dim 64, 128 or 256 (fp32 with head_dim 256: up to 32 text tokens), max_text <= 64, max_2d + max_3d <= 4096, max_batch <= 64.
+ * head_dim a multiple of 32 in [64, 256] (fp32 with head_dim 256: up to 32 text tokens), max_text <= 64, max_2d + max_3d <= 4096, max_batch <= 64.
  * The library owns *out until mvla_prune_destroy.  (Alg. 1 "Input" / "Init".)
  * Errors: INVALID_ARG, UNSUPPORTED, OOM, CUDA (no usable device).
  */

@@ -449,7 +449,7 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (c.salience_path != MVLA_SALIENCE_AUTO && c.salience_path != MVLA_SALIENCE_FMA) return MVLA_ERR_INVALID_ARG;
     if ((c.patch_path != 0 && c.patch_path != 1) || c.kmeans_max_iter < 0 || !(c.obj_2d_min >= 0.0 && c.obj_2d_min <= 1.0))
         return MVLA_ERR_INVALID_ARG;
-    if (c.head_dim != 64 && c.head_dim != 128 && c.head_dim != 256) return MVLA_ERR_UNSUPPORTED;
+    if (c.head_dim < 64 || c.head_dim > 256 || c.head_dim % 32 != 0) return MVLA_ERR_UNSUPPORTED;
     if (c.n_kv_heads < 0 || (c.n_kv_heads > 0 && (c.n_kv_heads > c.n_heads || c.n_heads % c.n_kv_heads != 0))) return MVLA_ERR_INVALID_ARG;
     if (c.patch_path && c.n_kv_heads > 0 && c.n_kv_heads != c.n_heads) return MVLA_ERR_UNSUPPORTED;   // the patch path is built for ungrouped keys
     if (c.max_text > kMaxText || c.max_2d + c.max_3d > kMaxVis || c.max_batch > 64) return MVLA_ERR_UNSUPPORTED;

@@ -85,7 +85,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     const uint32_t crank = cluster_ctarank();
     const uint32_t csize = gridDim.x;
     const int d = head_dim;
-    const int khalves = d / 64;                           // 64 bf16 = one 128-byte swizzle row
+    const int khalves = (d + 63) / 64;                    // 64 bf16 = one 128-byte swizzle row; a last partial box is zero-filled by TMA
     const float cscale = 1.4426950408889634f * rsqrtf(static_cast<float>(d));   // log2 domain
     const int tt0 = static_cast<int>(crank) * NTILE;
     uint8_t* Ks = dyn_smem;                               // [tile][khalf][128 rows x 128 B]
@@ -153,7 +153,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
 #pragma unroll
             for (int t = 0; t < NTILE; ++t) {
                 if (valid[t] <= 0) continue;
-                for (int kb = 0; kb < d / 16; ++kb) {
+                for (int kb = 0; kb < khalves * 4; ++kb) {     // columns past d are zeros: they add nothing
                     const int kh = kb >> 2, kin = kb & 3;          // 4 K-steps of 16 inside a 64-wide half
                     const uint64_t a = smem_desc_sw128(smem_u32(Ks + (t * khalves + kh) * 16384) + kin * 32);
                     const uint64_t b = smem_desc_sw128(smem_u32(Qs + kh * npad * 128) + kin * 32);
@@ -295,7 +295,7 @@ cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int he
                           const CUtensorMap* tk, int cluster, int npad, float* part, int64_t part_stride,
                           unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, cudaStream_t stream)
 {
-    const size_t smem = 1024 + static_cast<size_t>(head_dim / 64) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
+    const size_t smem = 1024 + static_cast<size_t>((head_dim + 63) / 64) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
     auto kern = salience_fast_kernel<TCOL, NTILE>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;

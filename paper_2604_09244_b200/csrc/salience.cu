@@ -57,7 +57,7 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
     bool ok = true;
 
     if constexpr (UMMA) {
-        const int khalves = d / 64;                           // 64 bf16 = one 128-byte swizzle row
+        const int khalves = (d + 63) / 64;                    // 64 bf16 = one 128-byte swizzle row; a last partial box is zero-filled by TMA
         uint8_t* Ks = dyn_smem;                               // [tile][khalf][128 rows x 128 B]
         uint8_t* Qs = dyn_smem + static_cast<size_t>(tiles_per_cta) * khalves * 16384;   // [khalf][npad rows x 128 B]
         const uint32_t bar_full = smem_u32(&s_bar[0]), bar_mma = smem_u32(&s_bar[1]);
@@ -101,7 +101,7 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
                 const uint32_t idesc = idesc_bf16_m128(npad);
                 for (int t = 0; t < tiles_per_cta; ++t) {
                     if (tile_info(s, tt0 + t).valid <= 0) continue;
-                    for (int kb = 0; kb < d / 16; ++kb) {
+                    for (int kb = 0; kb < khalves * 4; ++kb) {     // columns past d are zeros
                         const int kh = kb >> 2, kin = kb & 3;      // 4 K-steps of 16 inside a 64-wide half
                         const uint64_t a = smem_desc_sw128(smem_u32(Ks + (t * khalves + kh) * 16384) + kin * 32);
                         const uint64_t b = smem_desc_sw128(smem_u32(Qs + kh * npad * 128) + kin * 32);
@@ -333,7 +333,7 @@ cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int kv_group, in
 {
     size_t smem;
     if (UMMA)
-        smem = 1024 + static_cast<size_t>(head_dim / 64) * (static_cast<size_t>(tiles_per_cta) * 16384 + npad * 128);
+        smem = 1024 + static_cast<size_t>((head_dim + 63) / 64) * (static_cast<size_t>(tiles_per_cta) * 16384 + npad * 128);
     else
         smem = 1024 + sizeof(float) * (static_cast<size_t>(npad) * head_dim + kKeyTile * (head_dim + 1) +
                                 static_cast<size_t>(tiles_per_cta) * npad * kKeyTile);

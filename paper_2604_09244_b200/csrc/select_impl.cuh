@@ -256,12 +256,12 @@ __device__ void select_sample(const SampleDev& s, int b_local, const GateParams&
         }
       if (lane == 0) {
         float x[4];
-        x[3] = __fdividef(t1, t0 + t1);                                   // attention share of 3D (Eq. P2D / P3D)
+        x[3] = t1 / (t0 + t1);                                            // attention share of 3D (Eq. P2D / P3D); IEEE division: a share of an only modality is exactly 1
         x[2] = 1.f - x[3];
         if (gp.has_l1) {                                          // feature-norm share (Eq. 3-1), mean norms
-            const float m2 = n2 > 0 ? __fdividef(t2, static_cast<float>(n2)) : 0.f;
-            const float m3 = n3 > 0 ? __fdividef(t3, static_cast<float>(n3)) : 0.f;
-            x[1] = __fdividef(m3, m2 + m3);
+            const float m2 = n2 > 0 ? t2 / static_cast<float>(n2) : 0.f;
+            const float m3 = n3 > 0 ? t3 / static_cast<float>(n3) : 0.f;
+            x[1] = m3 / (m2 + m3);
             x[0] = 1.f - x[1];
         } else {
             x[0] = x[1] = 0.5f;

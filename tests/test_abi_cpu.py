@@ -39,7 +39,7 @@ def test_bad_arguments_are_error_codes(lib):
     assert lib.mvla_prune_create(None, C.byref(h)) == mvla.ERR_INVALID_ARG
     cfg = mvla.Config(0, mvla.DTYPE_BF16, 32, 128, 4096, 1, 32, 256, 512, 1, 0, 7, 1, 0, 0.08, 0.2, 0.85, 0.02, 0.1)
     assert lib.mvla_prune_create(C.byref(cfg), None) == mvla.ERR_INVALID_ARG
-    bad = mvla.Config.from_buffer_copy(cfg); bad.head_dim = 96
+    bad = mvla.Config.from_buffer_copy(cfg); bad.head_dim = 48
     assert lib.mvla_prune_create(C.byref(bad), C.byref(h)) == mvla.ERR_UNSUPPORTED
     bad = mvla.Config.from_buffer_copy(cfg); bad.max_text = 65
     assert lib.mvla_prune_create(C.byref(bad), C.byref(h)) == mvla.ERR_UNSUPPORTED

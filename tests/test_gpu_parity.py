@@ -279,7 +279,7 @@ def test_error_codes_never_fault():
     torch.cuda.synchronize()
     ctx.close()
     with pytest.raises(mvla.MvlaError) as e:
-        mvla.PruneContext(dtype=torch.bfloat16, n_heads=4, head_dim=96, d_model=256, max_batch=1, max_text=8,
+        mvla.PruneContext(dtype=torch.bfloat16, n_heads=4, head_dim=48, d_model=256, max_batch=1, max_text=8,
                           max_2d=8, max_3d=8)
     assert e.value.code == mvla.ERR_UNSUPPORTED
 
@@ -464,9 +464,42 @@ def test_grouped_key_heads(dtype, path):
     ctx.close()
 
 
+@pytest.mark.parametrize("d", [96, 160, 256])
 @pytest.mark.parametrize("dtype", ["bf16", "fp32"])
-def test_head_dim_256(dtype):
-    wl = W.small_workload(19, batch=2, D=512, H=2, d=256, dtype=dtype, n_txt=(7, 30), n_2d=(140, 60), n_3d=(100, 270))
+def test_other_head_dims(dtype, d):
+    # 96 and 160 are not multiples of the 64-element TMA box: the last box is partly out of range and zero-filled
+    wl = W.small_workload(19, batch=2, D=512, H=2, d=d, dtype=dtype, n_txt=(7, 30), n_2d=(140, 60), n_3d=(100, 270))
+    ctx = mvla.context_for(wl)
+    run_and_check_step(ctx, wl, 0, [oracle.State(s.n_vis) for s in wl.samples])
+    ctx.close()
+
+
+@pytest.mark.parametrize("mode", [W.MODE_FIXED, W.MODE_ADAPTIVE])
+def test_step_with_an_empty_modality(mode):
+    # one sample without 2D tokens, one without 3D tokens, one ordinary
+    wl = W.small_workload(23, batch=3, D=256, H=4, d=64, dtype="bf16", mode=mode, n_txt=(6, 17, 9),
+                          n_2d=(0, 150, 40), n_3d=(200, 0, 70))
+    ctx = mvla.context_for(wl)
+    out, refs = run_and_check_step(ctx, wl, 0, [oracle.State(s.n_vis) for s in wl.samples])
+    b = out.budgets.cpu().numpy()
+    assert b[0, 0] == 0 and b[1, 1] == 0
+    ctx.close()
+
+
+def test_step_more_samples_than_one_launch_carries():
+    # 40 samples: the per-sample descriptors travel 32 to a launch, so every stage runs in two launches
+    wl = W.small_workload(29, batch=40, D=128, H=2, d=64, dtype="bf16", n_txt=(3, 11, 6), n_2d=(33, 140, 64),
+                          n_3d=(129, 20, 75), keep=(0.3, 0.5, 0.25))
+    ctx = mvla.context_for(wl)
+    states = [oracle.State(s.n_vis) for s in wl.samples]
+    run_and_check_step(ctx, wl, 0, states)
+    ctx.close()
+
+
+def test_step_at_the_capacity_limits():
+    # 64 text tokens, 2048 + 2048 visual tokens: 32 key tiles, four per CTA in a cluster of eight
+    wl = W.small_workload(37, batch=1, D=64, H=1, d=64, dtype="bf16", n_txt=(64,), n_2d=(2048,), n_3d=(2048,),
+                          keep=(0.1,))
     ctx = mvla.context_for(wl)
     run_and_check_step(ctx, wl, 0, [oracle.State(s.n_vis) for s in wl.samples])
     ctx.close()
