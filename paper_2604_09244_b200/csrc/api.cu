@@ -33,9 +33,11 @@ struct mvla_ctx {
     size_t vis_all;              // max_batch * max_vis
     // patch-by-patch path (cfg.patch_path): attention copy [H][max_text][vis_all], per-patch smoothed
     // indicators [n_prune_points][n_slots][max_patch][4], and the scratch between its kernels
-    float* alpha_ws;
+    float* alpha_ws;             // [patch_sets] copies: steps in flight beside one another each have their own
     float* xhat_patch;
-    float* patch_x_ws;           // [vis_all / 2][4]
+    float* patch_x_ws;           // [patch_sets][vis_all / 2 + 1][4]
+    float* patch_attn_ws;        // [patch_sets][vis_all]
+    int patch_sets;              // kSets when the attention copies fit a modest budget, else 1 (then no overlap)
     int32_t* nout_ws;            // [max_batch] kept rows, [max_batch] ready flags, [1] finished-CTA counter
     int max_patch;
     unsigned step_parity;        // index of the scratch set of the current step
@@ -50,7 +52,7 @@ struct mvla_ctx {
     // one entry per scratch set.  A step whose side-stream work reads or writes any of them (its inputs,
     // its selection outputs) is ordered after everything enqueued on the caller's stream instead.
     struct Range { const char* lo; const char* hi; };
-    Range hist[kSets][10];
+    Range hist[kSets][16];
     int n_hist[kSets];
     bool hist_unknown;                         // the stream ran other work of this context since: order after it
     // Smoothed states (prune point x slot) that the step last run on each scratch set reads and writes:
@@ -278,7 +280,8 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
     if (fast) {
-        e = launch_salience_fast(bd, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, tq, tk, tiles_per_cta, cluster, npad, ctx->part,
+        e = launch_salience_fast(bd, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, tq, tk, tiles_per_cta, cluster, npad,
+                                 alpha.ptr && !acc64 ? nullptr : ctx->part,     // the patch path reads the attention copy only
                                  ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, st);
         if (used_acc64) *used_acc64 = acc64 != nullptr;
     } else {
@@ -314,6 +317,105 @@ GateParams gate_params(const mvla_ctx* ctx, int32_t mode, bool has_l1)
     return gp;
 }
 
+// ---- overlap of neighbouring prune steps (MVLA_FLAG_INPUTS_STABLE) ----
+// With stable inputs, scoring and selection of a step go to the side stream of the step's scratch set
+// (`par`); only the row copy stays on the caller's stream.  What the side-stream work of step k must follow:
+//   * selection and row copy of step k - kSets (same scratch set; the copy also frees that step's
+//     output buffers, so at most kSets - 1 earlier copies can still be running);
+//   * every selection of the kSets - 1 steps before that touches a smoothed state (prune point,
+//     slot) this step touches: a state is updated in call order.  Steps on other slots -- independent
+//     requests -- are not waited for;
+//   * if it reads or writes a buffer that one of those kSets - 1 steps writes, or if the stream has
+//     run other work of this context since: everything enqueued on the caller's stream so far.
+// Events recorded under another stream capture cannot be waited on; then, too, the step starts
+// after everything enqueued so far.
+struct ForkPlan {
+    bool ordered_after_all = false;
+    unsigned dep_mask = 0;               // scratch sets whose selection event this step's selection waits for
+    unsigned long long cap_id = 0;       // stream capture the events of this step belong to (0: none)
+};
+
+// `side`: buffers the side-stream work reads or writes, the first `n_side_written` of them written by it;
+// `copied`: buffers the row copy writes.  Enqueues the wait that opens the side stream and records what the
+// step writes and which states it touches.
+int32_t plan_fork(mvla_ctx* ctx, cudaStream_t st, unsigned par, int32_t prune_point, int32_t batch,
+                  const mvla_sample* samples, const mvla_ctx::Range* side, int n_side, int n_side_written,
+                  const mvla_ctx::Range* copied, int n_copied, ForkPlan* fp)
+{
+    cudaStreamCaptureStatus cst = cudaStreamCaptureStatusNone;
+    if (cudaStreamGetCaptureInfo(st, &cst, &fp->cap_id) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
+    if (cst != cudaStreamCaptureStatusActive) fp->cap_id = 0;
+    bool clash = ctx->hist_unknown;
+    for (unsigned s = 0; !clash && s < kSets; ++s) {
+        if (s == par) continue;
+        for (int i = 0; !clash && i < n_side; ++i)
+            for (int j = 0; !clash && j < ctx->n_hist[s]; ++j)
+                clash = side[i].lo && side[i].lo < ctx->hist[s][j].hi && ctx->hist[s][j].lo < side[i].hi;
+    }
+    // earlier selections still possibly in flight that touch a smoothed state this step touches: the
+    // state is updated in call order, so this step's selection waits for the most recent one per
+    // state (dep_mask; that one has in turn waited for those before it).  Steps older than
+    // kSets - 1 calls are ordered through the row-copy event or the stream itself.
+    const bool own_ok = ctx->sel_valid[par] && ctx->sel_capture[par] == fp->cap_id;
+    bool stale = false;
+    bool covered[kMaxChunk] = {};            // per sample of this step: most recent toucher of its state found
+    for (unsigned back = 1; back < kSets; ++back) {          // most recent step first
+        const unsigned s = (par + kSets - back) % kSets;
+        bool hit = false;
+        for (int b = 0; b < batch; ++b) {
+            if (covered[b]) continue;        // an even later step touches it and has waited for this one
+            const int32_t mine = prune_point * ctx->n_slots + samples[b].state_slot;
+            for (int i = 0; i < ctx->n_state_of[s]; ++i)
+                if (ctx->state_of[s][i] == mine) { covered[b] = hit = true; break; }
+        }
+        if (!hit) continue;
+        if (ctx->sel_valid[s] && ctx->sel_capture[s] == fp->cap_id) fp->dep_mask |= 1u << s;
+        else stale = true;                   // its event cannot be waited on from here
+    }
+    fp->ordered_after_all = clash || !own_ok || stale;
+    cudaError_t e;
+    if (fp->ordered_after_all) {
+        e = cudaEventRecord(ctx->ev_fork, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->aux[par], ctx->ev_fork, 0);
+        if (ctx->hist_unknown) {
+            for (int& n : ctx->n_hist) n = 0;
+            for (int& n : ctx->n_state_of) n = 0;
+        }
+    } else {
+        e = cudaStreamWaitEvent(ctx->aux[par], ctx->ev_copy[par], 0);
+    }
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    // remember what this step writes
+    int m = 0;
+    for (int i = 0; i < n_side_written; ++i) if (side[i].lo) ctx->hist[par][m++] = side[i];
+    for (int i = 0; i < n_copied; ++i) if (copied[i].lo) ctx->hist[par][m++] = copied[i];
+    ctx->n_hist[par] = m;
+    ctx->hist_unknown = false;
+    for (int b = 0; b < batch; ++b) ctx->state_of[par][b] = prune_point * ctx->n_slots + samples[b].state_slot;
+    ctx->n_state_of[par] = batch;
+    return MVLA_OK;
+}
+
+// Selection of a forked step: wait for the earlier selections on the same states.
+int32_t wait_state_deps(mvla_ctx* ctx, const ForkPlan& fp, cudaStream_t sel_stream)
+{
+    for (unsigned s = 0; !fp.ordered_after_all && s < kSets; ++s)
+        if ((fp.dep_mask >> s & 1u) && cudaStreamWaitEvent(sel_stream, ctx->ev_sel[s], 0) != cudaSuccess)
+            return fail_cuda(ctx, cudaGetLastError());
+    return MVLA_OK;
+}
+
+// Join of a forked step: the row copy on the caller's stream (and whatever the caller enqueues next) follows the selection.
+int32_t join_selection(mvla_ctx* ctx, const ForkPlan& fp, unsigned par, cudaStream_t sel_stream, cudaStream_t st)
+{
+    if (cudaEventRecord(ctx->ev_sel[par], sel_stream) != cudaSuccess ||
+        cudaStreamWaitEvent(st, ctx->ev_sel[par], 0) != cudaSuccess)
+        return fail_cuda(ctx, cudaGetLastError());
+    ctx->sel_valid[par] = true;
+    ctx->sel_capture[par] = fp.cap_id;
+    return MVLA_OK;
+}
+
 // ---- patch-by-patch path ----
 int32_t validate_patch(const mvla_ctx* ctx, int32_t batch, const mvla_sample* samples)
 {
@@ -323,9 +425,15 @@ int32_t validate_patch(const mvla_ctx* ctx, int32_t batch, const mvla_sample* sa
     return MVLA_OK;
 }
 
-AlphaOut alpha_of(const mvla_ctx* ctx)
+size_t alpha_floats(const mvla_ctx* ctx)
 {
-    return AlphaOut{ctx->alpha_ws, static_cast<int64_t>(ctx->cfg.max_text) * static_cast<int64_t>(ctx->vis_all),
+    return static_cast<size_t>(ctx->cfg.n_heads) * ctx->cfg.max_text * ctx->vis_all;
+}
+
+AlphaOut alpha_of(const mvla_ctx* ctx, unsigned set)
+{
+    return AlphaOut{ctx->alpha_ws + set * alpha_floats(ctx),
+                    static_cast<int64_t>(ctx->cfg.max_text) * static_cast<int64_t>(ctx->vis_all),
                     static_cast<int64_t>(ctx->vis_all)};
 }
 
@@ -343,10 +451,10 @@ PatchParams patch_params(const mvla_ctx* ctx)
 }
 
 // Salience with the attention copy, feature norms, head sum, per-patch indicators.
-int32_t run_patch_indicators(mvla_ctx* ctx, const Plan& plan, int32_t batch, const void* q, const void* k,
+int32_t run_patch_indicators(mvla_ctx* ctx, unsigned set, const Plan& plan, int32_t batch, const void* q, const void* k,
                              const void* hidden, int64_t rows, float* attn_out, float* x_out, cudaStream_t st)
 {
-    const AlphaOut alpha = alpha_of(ctx);
+    const AlphaOut alpha = alpha_of(ctx, set);
     for (int first = 0; first < batch; first += kMaxChunk) {
         const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
         const int32_t rc = run_salience_chunk(ctx, bd, q, k, rows, nullptr, nullptr, nullptr, nullptr, false, st, alpha);
@@ -361,7 +469,7 @@ int32_t run_patch_indicators(mvla_ctx* ctx, const Plan& plan, int32_t batch, con
     return MVLA_OK;
 }
 
-int32_t run_patch_select(mvla_ctx* ctx, const Plan& plan, int32_t batch, const float* attn, const float* x,
+int32_t run_patch_select(mvla_ctx* ctx, unsigned set, const Plan& plan, int32_t batch, const float* attn, const float* x,
                          const float* rand_u, int32_t* kept_idx, int32_t* out_offsets, int32_t* counts,
                          float* xhat_out, int32_t* info_out, mvla_patch_diag* diag, cudaStream_t st)
 {
@@ -370,8 +478,9 @@ int32_t run_patch_select(mvla_ctx* ctx, const Plan& plan, int32_t batch, const f
     std::memset(&io, 0, sizeof io);
     io.attn = attn; io.x = x; io.rand_u = rand_u;
     io.xhat_state = ctx->xhat_patch; io.xhat_out = xhat_out; io.info_out = info_out; io.diag = diag;
-    io.counts = counts; io.nout_ws = ctx->nout_ws; io.ready_ws = ctx->nout_ws + ctx->cfg.max_batch;
-    io.done_ws = ctx->nout_ws + 2 * ctx->cfg.max_batch; io.status = ctx->status_dev;
+    int32_t* ws = ctx->nout_ws + set * (2 * static_cast<size_t>(ctx->cfg.max_batch) + 1);
+    io.counts = counts; io.nout_ws = ws; io.ready_ws = ws + ctx->cfg.max_batch;
+    io.done_ws = ws + 2 * ctx->cfg.max_batch; io.status = ctx->status_dev;
     io.kept_idx = kept_idx; io.out_offsets = out_offsets; io.batch_total = batch;
     for (int first = 0; first < batch; first += kMaxChunk) {
         const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
@@ -402,29 +511,68 @@ int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, cons
     if (rc != MVLA_OK) return rc;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return MVLA_ERR_CUDA;
-    ctx->hist_unknown = true;
     Plan plan;
     rc = make_plan(ctx, prune_point, batch, samples, MVLA_MODE_ADAPTIVE, flags, true, &plan);
     if (rc != MVLA_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    float* attn = out->attn ? out->attn : ctx->attn_ws;
-    float* x = out->patch_x ? out->patch_x : ctx->patch_x_ws;
-    rc = run_patch_indicators(ctx, plan, batch, in->q, in->k, in->hidden, in->rows, attn, x, st);
-    if (rc != MVLA_OK) return rc;
-    rc = run_patch_select(ctx, plan, batch, attn, x, in->rand_u, out->kept_idx, out->out_offsets, out->budgets,
-                          out->patch_xhat, out->patch_info, out->patch_diag, st);
-    if (rc != MVLA_OK) return rc;
     int64_t cap = 0;                               // the row count is known only on the device: cover the capacity
     for (int b = 0; b < batch; ++b) cap += samples[b].n_txt + samples[b].n_2d + samples[b].n_3d;
     CompactJob job;
     const int32_t kv_bytes = static_cast<int32_t>(ctx->kv_heads * ctx->cfg.head_dim * ctx->elem);
     for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
     job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
+
+    // Scratch set of this step; with stable inputs its scoring, indicators and selection run on that set's
+    // side stream beside the steps before (plan_fork), the row copy stays on the caller's stream.
+    ctx->step_parity = (ctx->step_parity + 1u) % kSets;
+    const unsigned par = ctx->step_parity;
+    bool forked = false;
+    ForkPlan fp;
+    if ((flags & MVLA_FLAG_INPUTS_STABLE) && ctx->patch_sets == kSets && batch <= kMaxChunk &&
+        chunk_is_fast(ctx, chunk_of(plan, 0, batch))) {
+        forked = true;
+        const size_t nvis_b = static_cast<size_t>(plan.total_vis), npat_b = nvis_b / 2, in_rows = static_cast<size_t>(in->rows);
+        const size_t hb = static_cast<size_t>(ctx->cfg.d_model) * ctx->elem, kb = static_cast<size_t>(kv_bytes);
+        const size_t qb = static_cast<size_t>(ctx->cfg.n_heads) * ctx->cfg.head_dim * ctx->elem;
+        const mvla_ctx::Range side[12] = {
+            range_of(out->kept_idx, static_cast<size_t>(cap) * 4), range_of(out->out_offsets, (batch + 1) * 4u),
+            range_of(out->budgets, batch * 8u), range_of(out->attn, nvis_b * 4), range_of(out->patch_x, npat_b * 16),
+            range_of(out->patch_xhat, npat_b * 16), range_of(out->patch_info, npat_b * 4),
+            range_of(out->patch_diag, batch * sizeof(mvla_patch_diag)),
+            range_of(in->q, in_rows * qb), range_of(in->k, in_rows * kb), range_of(in->hidden, in_rows * hb),
+            range_of(in->rand_u, npat_b * 4)};
+        const mvla_ctx::Range copied[3] = {range_of(out->out_hidden, static_cast<size_t>(cap) * hb),
+                                           range_of(out->out_k, static_cast<size_t>(cap) * kb),
+                                           range_of(out->out_v, static_cast<size_t>(cap) * kb)};
+        rc = plan_fork(ctx, st, par, prune_point, batch, samples, side, 12, 8, copied, 3, &fp);
+        if (rc != MVLA_OK) return rc;
+    } else {
+        ctx->hist_unknown = true;
+        ctx->sel_valid[par] = false;               // this set is used outside the event chain
+    }
+    const unsigned set = forked ? par : 0;
+    cudaStream_t side_stream = forked ? ctx->aux[par] : st;
+    float* attn = out->attn ? out->attn : ctx->patch_attn_ws + set * ctx->vis_all;
+    float* x = out->patch_x ? out->patch_x : ctx->patch_x_ws + set * (ctx->vis_all / 2 + 1) * 4;
+    rc = run_patch_indicators(ctx, set, plan, batch, in->q, in->k, in->hidden, in->rows, attn, x, side_stream);
+    if (rc != MVLA_OK) return rc;
+    if (forked) {
+        rc = wait_state_deps(ctx, fp, side_stream);
+        if (rc != MVLA_OK) return rc;
+    }
+    rc = run_patch_select(ctx, set, plan, batch, attn, x, in->rand_u, out->kept_idx, out->out_offsets, out->budgets,
+                          out->patch_xhat, out->patch_info, out->patch_diag, side_stream);
+    if (rc != MVLA_OK) return rc;
+    if (forked) {
+        rc = join_selection(ctx, fp, par, side_stream, st);
+        if (rc != MVLA_OK) return rc;
+    }
     for (int first = 0; first < batch; first += kMaxChunk) {
         const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
         const cudaError_t e = launch_compact(bd, job, out->kept_idx, static_cast<int32_t>(cap), 0, out->out_offsets, first, batch, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
+    if (forked && cudaEventRecord(ctx->ev_copy[par], st) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
     commit_steps(ctx, prune_point, plan, samples);
     if (total_kept_out) *total_kept_out = static_cast<int32_t>(cap);
     return MVLA_OK;
@@ -478,7 +626,8 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (c.salience_path == MVLA_SALIENCE_FMA) ctx->use_umma = false;
     ctx->part = ctx->attn_ws = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
     ctx->acc64 = nullptr;
-    ctx->alpha_ws = ctx->xhat_patch = ctx->patch_x_ws = nullptr;
+    ctx->alpha_ws = ctx->xhat_patch = ctx->patch_x_ws = ctx->patch_attn_ws = nullptr;
+    ctx->patch_sets = 1;
     ctx->nout_ws = nullptr;
     ctx->max_patch = std::min(c.max_2d, c.max_3d);
     ctx->ev_fork = nullptr;
@@ -516,10 +665,13 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->acc64), kSets * vis_all * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(ctx->acc64, 0, kSets * vis_all * sizeof(unsigned long long));
     if (c.patch_path) {
-        alloc(&ctx->alpha_ws, static_cast<size_t>(c.n_heads) * c.max_text * vis_all);
+        const size_t alpha_n = static_cast<size_t>(c.n_heads) * c.max_text * vis_all;
+        ctx->patch_sets = alpha_n * sizeof(float) * kSets <= (size_t(1) << 30) ? kSets : 1;   // at most 1 GiB of attention copies
+        alloc(&ctx->alpha_ws, alpha_n * ctx->patch_sets);
         alloc(&ctx->xhat_patch, n_state * std::max(ctx->max_patch, 1) * 4);
-        alloc(&ctx->patch_x_ws, (vis_all / 2 + 1) * 4);
-        const size_t nws = (2 * static_cast<size_t>(c.max_batch) + 1) * sizeof(int32_t);
+        alloc(&ctx->patch_x_ws, (vis_all / 2 + 1) * 4 * ctx->patch_sets);
+        alloc(&ctx->patch_attn_ws, vis_all * ctx->patch_sets);
+        const size_t nws = (2 * static_cast<size_t>(c.max_batch) + 1) * sizeof(int32_t) * ctx->patch_sets;
         if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->nout_ws), nws);
         if (e == cudaSuccess) e = cudaMemset(ctx->nout_ws, 0, nws);
     }
@@ -565,6 +717,7 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     cudaFree(ctx->alpha_ws);
     cudaFree(ctx->xhat_patch);
     cudaFree(ctx->patch_x_ws);
+    cudaFree(ctx->patch_attn_ws);
     cudaFree(ctx->nout_ws);
     for (cudaStream_t sp : ctx->aux)
         if (sp) {
@@ -695,7 +848,7 @@ int32_t mvla_patch_indicators(mvla_ctx* ctx, int32_t batch, const mvla_sample* s
     Plan plan;
     rc = make_plan(ctx, 0, batch, samples, MVLA_MODE_FIXED, 0, false, &plan);
     if (rc != MVLA_OK) return rc;
-    return run_patch_indicators(ctx, plan, batch, q, k, hidden, rows, attn_out, x_out, static_cast<cudaStream_t>(stream));
+    return run_patch_indicators(ctx, 0, plan, batch, q, k, hidden, rows, attn_out, x_out, static_cast<cudaStream_t>(stream));
 }
 
 int32_t mvla_patch_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, uint32_t flags,
@@ -718,7 +871,7 @@ int32_t mvla_patch_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, con
     Plan plan;
     rc = make_plan(ctx, prune_point, batch, samples, MVLA_MODE_ADAPTIVE, flags, true, &plan);
     if (rc != MVLA_OK) return rc;
-    rc = run_patch_select(ctx, plan, batch, attn, x, rand_u, kept_idx, out_offsets, counts, xhat_out, info_out, diag,
+    rc = run_patch_select(ctx, 0, plan, batch, attn, x, rand_u, kept_idx, out_offsets, counts, xhat_out, info_out, diag,
                           static_cast<cudaStream_t>(stream));
     if (rc != MVLA_OK) return rc;
     commit_steps(ctx, prune_point, plan, samples);
@@ -763,29 +916,15 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     ctx->step_parity = (ctx->step_parity + 1u) % kSets;
     unsigned long long* acc64 = ctx->acc64 + ctx->step_parity * ctx->vis_all;
     float* l1_ws = ctx->l1_ws + ctx->step_parity * ctx->vis_all;
-    // With stable inputs (and the fast scoring kernel, whose scratch rotates over kSets sets) scoring
-    // and selection go to the side stream of this step's scratch set; only the row copy stays on the
-    // caller's stream.  What the side-stream work of step k must follow:
-    //   * selection and row copy of step k - kSets (same scratch set; the copy also frees that step's
-    //     output buffers, so at most kSets - 1 earlier copies can still be running);
-    //   * every selection of the kSets - 1 steps before that touches a smoothed state (prune point,
-    //     slot) this step touches: a state is updated in call order.  Steps on other slots -- independent
-    //     requests -- are not waited for;
-    //   * if it reads or writes a buffer that one of those kSets - 1 steps writes, or if the stream has
-    //     run other work of this context since: everything enqueued on the caller's stream so far.
-    // Events recorded under another stream capture cannot be waited on; then, too, the step starts
-    // after everything enqueued so far.
-    bool forked = false, ordered_after_all = false;
-    unsigned dep_mask = 0;
-    unsigned long long cap_id = 0;
+    // With stable inputs (and the fast scoring kernel, whose scratch rotates over kSets sets) scoring and
+    // selection go to the side stream of this step's scratch set (see plan_fork).
+    bool forked = false;
+    ForkPlan fp;
     const unsigned par = ctx->step_parity;
     const size_t nvis_b = static_cast<size_t>(plan.total_vis), nout_b = static_cast<size_t>(plan.total_out);
     const size_t hb = static_cast<size_t>(ctx->cfg.d_model) * ctx->elem, kb = static_cast<size_t>(kv_bytes);
     const size_t qb = static_cast<size_t>(ctx->cfg.n_heads) * ctx->cfg.head_dim * ctx->elem;
     if ((flags & MVLA_FLAG_INPUTS_STABLE) && batch <= kMaxChunk && chunk_is_fast(ctx, chunk_of(plan, 0, batch))) {
-        cudaStreamCaptureStatus cst = cudaStreamCaptureStatusNone;
-        if (cudaStreamGetCaptureInfo(st, &cst, &cap_id) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
-        if (cst != cudaStreamCaptureStatusActive) cap_id = 0;
         forked = true;
         // buffers the side-stream work touches: selection outputs, and the inputs of scoring
         const size_t in_rows = static_cast<size_t>(in->rows);
@@ -795,56 +934,10 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
             range_of(out->z, nvis_b * 4), range_of(out->diag, batch * sizeof(mvla_diag)),
             range_of(in->q, in_rows * qb), range_of(in->k, in_rows * kb),
             range_of(adaptive ? in->hidden : nullptr, in_rows * hb)};
-        bool clash = ctx->hist_unknown;
-        for (unsigned s = 0; !clash && s < kSets; ++s) {
-            if (s == par) continue;
-            for (int i = 0; !clash && i < 10; ++i)
-                for (int j = 0; !clash && j < ctx->n_hist[s]; ++j)
-                    clash = side[i].lo && side[i].lo < ctx->hist[s][j].hi && ctx->hist[s][j].lo < side[i].hi;
-        }
-        // earlier selections still possibly in flight that touch a smoothed state this step touches: the
-        // state is updated in call order, so this step's selection waits for the most recent one per
-        // state (dep_mask; that one has in turn waited for those before it).  Steps older than
-        // kSets - 1 calls are ordered through the row-copy event or the stream itself.
-        const bool own_ok = ctx->sel_valid[par] && ctx->sel_capture[par] == cap_id;
-        bool stale = false;
-        bool covered[kMaxChunk] = {};            // per sample of this step: most recent toucher of its state found
-        for (unsigned back = 1; back < kSets; ++back) {          // most recent step first
-            const unsigned s = (par + kSets - back) % kSets;
-            bool hit = false;
-            for (int b = 0; b < batch; ++b) {
-                if (covered[b]) continue;        // an even later step touches it and has waited for this one
-                const int32_t mine = prune_point * ctx->n_slots + samples[b].state_slot;
-                for (int i = 0; i < ctx->n_state_of[s]; ++i)
-                    if (ctx->state_of[s][i] == mine) { covered[b] = hit = true; break; }
-            }
-            if (!hit) continue;
-            if (ctx->sel_valid[s] && ctx->sel_capture[s] == cap_id) dep_mask |= 1u << s;
-            else stale = true;                   // its event cannot be waited on from here
-        }
-        ordered_after_all = clash || !own_ok || stale;
-        cudaError_t e;
-        if (ordered_after_all) {
-            e = cudaEventRecord(ctx->ev_fork, st);
-            if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->aux[par], ctx->ev_fork, 0);
-            if (ctx->hist_unknown) {
-                for (int& n : ctx->n_hist) n = 0;
-                for (int& n : ctx->n_state_of) n = 0;
-            }
-        } else {
-            e = cudaStreamWaitEvent(ctx->aux[par], ctx->ev_copy[par], 0);
-        }
-        if (e != cudaSuccess) return fail_cuda(ctx, e);
-        // remember what this step writes
-        int m = 0;
-        for (int i = 0; i < 7; ++i) if (side[i].lo) ctx->hist[par][m++] = side[i];
-        if (out->out_hidden) ctx->hist[par][m++] = range_of(out->out_hidden, nout_b * hb);
-        if (out->out_k) ctx->hist[par][m++] = range_of(out->out_k, nout_b * kb);
-        if (out->out_v) ctx->hist[par][m++] = range_of(out->out_v, nout_b * kb);
-        ctx->n_hist[par] = m;
-        ctx->hist_unknown = false;
-        for (int b = 0; b < batch; ++b) ctx->state_of[par][b] = prune_point * ctx->n_slots + samples[b].state_slot;
-        ctx->n_state_of[par] = batch;
+        const mvla_ctx::Range copied[3] = {range_of(out->out_hidden, nout_b * hb), range_of(out->out_k, nout_b * kb),
+                                           range_of(out->out_v, nout_b * kb)};
+        rc = plan_fork(ctx, st, par, prune_point, batch, samples, side, 10, 7, copied, 3, &fp);
+        if (rc != MVLA_OK) return rc;
     } else {
         ctx->hist_unknown = true;
     }
@@ -858,9 +951,8 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         cudaStream_t sel_stream = st;
         if (forked) {
             sel_stream = ctx->aux[par];
-            for (unsigned s = 0; !ordered_after_all && s < kSets; ++s)
-                if ((dep_mask >> s & 1u) && cudaStreamWaitEvent(sel_stream, ctx->ev_sel[s], 0) != cudaSuccess)
-                    return fail_cuda(ctx, cudaGetLastError());
+            rc = wait_state_deps(ctx, fp, sel_stream);
+            if (rc != MVLA_OK) return rc;
         }
         SelectIO io;
         std::memset(&io, 0, sizeof io);
@@ -876,11 +968,8 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         cudaError_t e = launch_select(bd, gp, io, sel_stream);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
         if (forked) {                                // join: the row copy, and whatever the caller enqueues next
-            if (cudaEventRecord(ctx->ev_sel[par], sel_stream) != cudaSuccess ||
-                cudaStreamWaitEvent(st, ctx->ev_sel[par], 0) != cudaSuccess)
-                return fail_cuda(ctx, cudaGetLastError());
-            ctx->sel_valid[par] = true;
-            ctx->sel_capture[par] = cap_id;
+            rc = join_selection(ctx, fp, par, sel_stream, st);
+            if (rc != MVLA_OK) return rc;
         } else {
             ctx->sel_valid[par] = false;             // this set was used outside the event chain
         }

@@ -82,7 +82,8 @@ inline cudaLaunchAttribute pdl_attribute()
 
 // bf16 tensor-core salience with logits held in registers (one or two key tiles per CTA).  With
 // `acc64` the per-head contributions are added into 64-bit fixed-point accumulators (scale 2^60, one
-// per visual token, zero on entry); without it they go to part[h][vis] as in launch_salience.
+// per visual token, zero on entry); without it they go to part[h][vis] as in launch_salience (nowhere when
+// `part` is null too: only the attention copy is wanted).
 // `free_running`: the kernel does not wait for the kernel before it in its stream (the caller orders
 // everything it depends on with events).
 // Optional copy of the attention itself for the patch-by-patch path:

@@ -273,7 +273,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         if (tid < valid[t]) {
             if (acc64)
                 atomicAdd(acc64 + s.vis_off + vis0[t] + tid, __float2ull_rn(acc * kFixScale));
-            else
+            else if (part)                    // neither: the caller wants the attention copy only
                 part[static_cast<int64_t>(h) * part_stride + s.vis_off + vis0[t] + tid] = acc;
             if (alpha.ptr) {              // the attention itself, for the per-patch indicators (coalesced over keys)
                 float* ap = alpha.ptr + static_cast<int64_t>(h) * alpha.stride_h + s.vis_off + vis0[t] + tid;

@@ -247,3 +247,42 @@ def test_patch_path_error_codes():
     torch.cuda.synchronize()
     assert int(out.out_offsets[-1]) <= wl.total_rows
     ctx.close()
+
+
+def test_pipelined_patch_steps_match_serial_steps():
+    # MVLA_FLAG_INPUTS_STABLE lets neighbouring steps overlap inside the library; results must not change.
+    # Two episodes (state slots 0-1 and 2-3) interleaved over four action steps, seven rotating output sets.
+    import dataclasses
+    wl = W.patch_workload(27, batch=2, D=256, H=4, d=128, n_txt=(10, 32), n_patch=(130, 256), steps=4, cold_start=1)
+    devs = [device_tensors(wl, t) for t in range(4)]
+    us = [torch.from_numpy(wl.extra["rand_u"][t]).cuda() for t in range(4)]
+    episodes = [wl.samples, [dataclasses.replace(s, state_slot=s.state_slot + 2) for s in wl.samples]]
+
+    def run(flag):
+        ctx = mvla.context_for(wl, n_state_slots=4)
+        outs = [ctx.alloc_outputs(wl.samples, patch=True) for _ in range(7)]
+        seen = []
+        i = 0
+        for t in range(4):
+            for ep in episodes:
+                o = outs[i % 7]
+                ctx.prune_step(0, ep, mvla.MODE_PATCH, devs[t]["q"], devs[t]["k"], devs[t]["v"], devs[t]["hidden"],
+                               flags=flag, out=o, rand_u=us[t])
+                if i % 7 == 6 or (t == 3 and ep is episodes[-1]):
+                    torch.cuda.synchronize()
+                # results are complete in stream order: reading them on the same stream needs no sync
+                n = int(o.out_offsets[-1])
+                seen.append((o.out_offsets.cpu().numpy().copy(), o.kept_idx[:n].cpu().numpy().copy(),
+                             o.budgets.cpu().numpy().copy(), o.patch_info.cpu().numpy().copy(),
+                             o.out_hidden[:n].float().cpu().numpy().copy()))
+                i += 1
+        torch.cuda.synchronize()
+        ctx.close()
+        return seen
+
+    serial, piped = run(0), run(mvla.FLAG_INPUTS_STABLE)
+    assert len(serial) == len(piped) == 8
+    for a, b in zip(serial, piped):
+        for x, y in zip(a, b):
+            assert np.array_equal(x, y)
+    assert serial[0][2].sum() > serial[-1][2].sum()      # the cold-start step kept everything, later steps prune
