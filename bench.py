@@ -42,31 +42,34 @@ def measured_peaks():
     return {"hbm_gbs": HBM_FALLBACK_GBS}, "fallback"
 
 
-# DRAM bytes (read + write) per launch of the stage's main kernel from one ncu capture of this benchmark
-# (profiles/), valid only for the kernel sources they were taken on: the digest below is over csrc/.
-NCU_CSRC_SHA256 = "72429f42da935634b2151818e7eaa0c02df1ba71fe8a59f436d41dd27a449f70"
-NCU_TRAFFIC = {             # (workload, stage) -> dram__bytes_read.sum + dram__bytes_write.sum per launch
-    ("config2", "salience"): 6621440,      # salience_fast_kernel<32,1>
-    ("config2", "select"): 76544,          # select_kernel
-    ("config2", "compact"): 7085440,       # compact_kernel: the written half is still in L2 when the kernel ends
-    ("patch_mla", "salience"): 4516736 + 6316800,   # salience_fast_kernel + patch_indicators_kernel
-    ("patch_mla", "select"): 61696,        # patch_select_kernel
+# DRAM bytes (read + write) per launch of the stage's kernel(s) from one ncu capture of this benchmark
+# (summaries under profiles/), valid only for the kernel sources they were taken on: per stage a digest over
+# the source files its kernels are compiled from.
+NCU_SOURCES = {
+    "salience": ("fused.cu", "device_utils.cuh", "tmem_ld.cuh", "select_impl.cuh", "common.cuh"),
+    "select": ("select.cu", "select_impl.cuh", "common.cuh"),
+    "compact": ("compact.cu", "common.cuh"),
+    "patch_salience": ("fused.cu", "patch.cu", "device_utils.cuh", "tmem_ld.cuh", "select_impl.cuh", "common.cuh"),
+    "patch_select": ("patch.cu", "select_impl.cuh", "common.cuh"),
 }
+NCU_DIGEST = {}             # stage -> sha256 of its sources when the counters were taken
+NCU_TRAFFIC = {}            # (workload, stage) -> dram__bytes_read.sum + dram__bytes_write.sum per launch
 
 
-def csrc_digest() -> str:
+def source_digest(files) -> str:
     import hashlib
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2604_09244_b200", "csrc")
-    for name in sorted(os.listdir(d)):
+    for name in files:
         with open(os.path.join(d, name), "rb") as f:
             h.update(name.encode() + b"\0" + f.read())
     return h.hexdigest()
 
 
 def ncu_traffic(workload: str, stage: str):
-    """Null once a kernel source has changed since the counters were taken."""
-    if not NCU_CSRC_SHA256 or csrc_digest() != NCU_CSRC_SHA256:
+    """Null once a source of the stage's kernels has changed since the counters were taken."""
+    key = ("patch_" + stage) if workload.startswith("patch") and stage != "compact" else stage
+    if key not in NCU_DIGEST or source_digest(NCU_SOURCES[key]) != NCU_DIGEST[key]:
         return None
     return NCU_TRAFFIC.get((workload, stage))
 

@@ -18,17 +18,17 @@
 namespace mvla {
 namespace {
 
-constexpr int kIndThreads = 1024;
+constexpr int kIndThreads = 512;
 constexpr int kPatchThreads = 256;
 constexpr int kMaxPatch = kMaxVis / 2;
 constexpr int kPPT = kMaxPatch / kPatchThreads;      // patches per thread, strided by the block size
 
 // grid = (ceil(max P / PP), samples), PP = 2, 4 or 8 patches per CTA (8 floats = one 32-byte sector per
 // (head, query); fewer patches per CTA when the batch is too small to fill the SMs otherwise).
-// Thread = (patch, group): the group walks the (head, query) pairs with stride 1024 / PP, so a CTA has
+// Thread = (patch, group): the group walks the (head, query) pairs with stride 512 / PP, so a CTA has
 // all its loads of a pass in flight at once (a few per thread).
 // Also writes the per-token scores of the patch's two tokens: a_j = ||alpha_j||_1 / (H n_t).
-// The L1 feature norms of the CTA's 2 PP rows (Sec. 3.1.2) are taken here too, 512 / PP threads per row,
+// The L1 feature norms of the CTA's 2 PP rows (Sec. 3.1.2) are taken here too, 256 / PP threads per row,
 // their loads issued before the kernel waits for the attention copy of the kernel before it.
 template <typename T, int PP>
 __global__ void __launch_bounds__(kIndThreads, 1)
