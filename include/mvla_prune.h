@@ -240,7 +240,8 @@ int32_t mvla_compact(mvla_ctx *ctx, int32_t batch, const mvla_sample *samples,
  * the number of output rows.  In MVLA_MODE_PATCH the chain is mvla_patch_indicators, mvla_patch_select,
  * mvla_compact; the row count is then known only on the device (out_offsets[batch]) and
  * `total_kept_out` receives the capacity bound sum(n_txt + n_2d + n_3d); `budgets` receives the kept
- * counts per modality; MVLA_FLAG_INPUTS_STABLE is accepted and ignored.
+ * counts per modality; MVLA_FLAG_INPUTS_STABLE overlaps neighbouring steps as on the budgeted path (when the
+ * context could afford one attention copy per step in flight: six copies within 1 GiB).
  */
 int32_t mvla_prune_step(mvla_ctx *ctx, int32_t prune_point, int32_t batch,
                         const mvla_sample *samples, int32_t mode, uint32_t flags,

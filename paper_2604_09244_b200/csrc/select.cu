@@ -1,31 +1,40 @@
 // Stand-alone select kernel: one CTA per sample running select_sample (see select_impl.cuh).
+//
+// Two CTA sizes.  512 threads for samples of up to 1024 visual tokens: steps of independent requests run
+// beside one another, and a 1024-thread CTA (64 registers per thread: a whole SM's register file) would
+// have to wait for an SM that the other steps' CTAs have left.  1024 threads above that: the kernel
+// itself is then shorter, which is what counts when the steps of one episode follow one another through
+// the smoothed state.
 #include "common.cuh"
 #include "select_impl.cuh"
 
 namespace mvla {
 namespace {
 
-constexpr int kSelThreads = 512;
-
-__global__ void __launch_bounds__(kSelThreads, 1)
+template <int NT>
+__global__ void __launch_bounds__(NT, 1)
 select_kernel(const __grid_constant__ BatchDesc bd, const GateParams gp, const SelectIO io)
 {
-    __shared__ SelectSmem<kSelThreads> sm;
-    select_sample<kSelThreads>(bd.s[blockIdx.x], blockIdx.x, gp, io, sm);
+    __shared__ SelectSmem<NT> sm;
+    select_sample<NT>(bd.s[blockIdx.x], blockIdx.x, gp, io, sm);
 }
 
 }  // namespace
 
 cudaError_t launch_select(const BatchDesc& bd, const GateParams& gp, const SelectIO& io, cudaStream_t stream)
 {
+    int max_vis = 0;
+    for (int b = 0; b < bd.n; ++b) max_vis = max(max_vis, bd.s[b].n_2d + bd.s[b].n_3d);
+    const bool wide = max_vis > 1024;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(bd.n);
-    cfg.blockDim = dim3(kSelThreads);
+    cfg.blockDim = dim3(wide ? 1024 : 512);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1] = {pdl_attribute()};
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, select_kernel, bd, gp, io);
+    return wide ? cudaLaunchKernelEx(&cfg, select_kernel<1024>, bd, gp, io)
+                : cudaLaunchKernelEx(&cfg, select_kernel<512>, bd, gp, io);
 }
 
 }  // namespace mvla
