@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """The CUDA library (nvcc cross-compiles without a GPU) and the C oracle are built in-tree before any
+    test runs; a failed build fails the session instead of letting tests look for a missing library."""
+    from paper_2604_09244_b200 import build
+    import oracle
+    build.build_library()
+    oracle.build()

@@ -503,3 +503,59 @@ def test_step_at_the_capacity_limits():
     ctx = mvla.context_for(wl)
     run_and_check_step(ctx, wl, 0, [oracle.State(s.n_vis) for s in wl.samples])
     ctx.close()
+
+
+def test_head_sharded_step_two_ranks_emulated_on_one_gpu():
+    # Tensor-parallel serving: each rank scores its own heads, the scores are averaged over the ranks, every
+    # rank selects on the same scores and copies its own K / V heads.  The two ranks run one after the other
+    # here (their kernels do not wait on one another); the average is taken in place of the all-reduce.
+    from paper_2604_09244_b200 import tensor_parallel as TP
+    wl = W.small_workload(73, batch=2, D=256, H=8, d=64, dtype="bf16", mode=W.MODE_FIXED, n_txt=(9, 20),
+                          n_2d=(130, 64), n_3d=(200, 300), n_kv_heads=4)
+    t = wl.steps[0]
+    dev = device_tensors(wl)
+    world = 2
+    ctxs, shards, partial = [], [], []
+    for r in range(world):
+        ctx = mvla.PruneContext(dtype=torch.bfloat16, n_heads=8 // world, n_kv_heads=4 // world, head_dim=64, d_model=256,
+                                max_batch=2, max_text=32, max_2d=256, max_3d=512, tau_2d=wl.tau_2d, tau_3d=wl.tau_3d,
+                                cold_start_full_keep=0)
+        sh = {n: TP.head_shard(dev[n], r, world) for n in ("q", "k", "v")}
+        a, _ = ctx.salience(wl.samples, sh["q"], sh["k"])
+        ctxs.append(ctx); shards.append(sh); partial.append(a)
+    torch.cuda.synchronize()
+    attn = (partial[0] + partial[1]) / world                    # what the all-reduce leaves on every rank
+    vis = 0
+    for s in wl.samples:
+        assert_salience_close(attn[vis:vis + s.n_vis].cpu().numpy(), oracle.salience_gqa(t.q, t.k, 8, 4, 64, s))
+        vis += s.n_vis
+    kept_by_rank = []
+    for r in range(world):
+        out = ctxs[r].alloc_outputs(wl.samples, extras=True)
+        ctxs[r].select(0, wl.samples, wl.mode, attn, None, out=out)
+        total = sum(s.seq_len for s in wl.samples)
+        ctxs[r].compact(wl.samples, out.kept_idx, out.out_offsets, total, dev["hidden"], shards[r]["k"], shards[r]["v"],
+                        out_hidden=out.out_hidden, out_k=out.out_k, out_v=out.out_v)
+        torch.cuda.synchronize()
+        offs, kept_all = out.out_offsets.cpu().numpy(), out.kept_idx.cpu().numpy()
+        kept_by_rank.append(kept_all[:offs[-1]].copy())
+        vis = 0
+        for b, s in enumerate(wl.samples):
+            kept = kept_all[offs[b]:offs[b + 1]]
+            k2, k3 = oracle.budget_fixed(s)
+            check_kept_against_oracle(s, kept, k2, k3, oracle.normalise(oracle.salience_gqa(t.q, t.k, 8, 4, 64, s), s.n_2d, s.n_3d))
+            n = len(kept)
+            rows = s.seq_off + kept
+            assert torch.equal(out.out_hidden[offs[b]:offs[b] + n], dev["hidden"][rows])
+            assert torch.equal(out.out_k[offs[b]:offs[b] + n], shards[r]["k"][rows])       # this rank's key heads
+            assert torch.equal(out.out_v[offs[b]:offs[b] + n], shards[r]["v"][rows])
+            vis += s.n_vis
+    assert np.array_equal(kept_by_rank[0], kept_by_rank[1])      # identical scores, identical decisions
+    # the packaged call on a group of one rank: same kept positions as the ranks above
+    full = mvla.context_for(wl)
+    o = TP.prune_step_head_sharded(full, 0, wl.samples, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"])
+    torch.cuda.synchronize()
+    n = int(o.out_offsets[-1])
+    assert np.array_equal(o.kept_idx[:n].cpu().numpy(), kept_by_rank[0])
+    for c in ctxs + [full]:
+        c.close()
