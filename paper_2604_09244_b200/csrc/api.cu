@@ -23,7 +23,6 @@ struct mvla_ctx {
     int kv_heads;                // key / value heads (== n_heads unless grouped)
     float* part;                 // [H][max_batch * max_vis] per-head partial scores
     int64_t part_stride;
-    float* attn_ws;              // [max_batch * max_vis]
     float* l1_ws;                // [kSets][max_batch * max_vis] feature norms, one set per step in flight
     float* ahat_state;           // [n_prune_points][n_slots][max_vis]
     float* mhat_state;           // [n_prune_points][n_slots][4]
@@ -624,7 +623,7 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     ctx->use_umma = c.dtype == MVLA_DTYPE_BF16;
     ctx->kv_heads = c.n_kv_heads > 0 ? c.n_kv_heads : c.n_heads;
     if (c.salience_path == MVLA_SALIENCE_FMA) ctx->use_umma = false;
-    ctx->part = ctx->attn_ws = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
+    ctx->part = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
     ctx->acc64 = nullptr;
     ctx->alpha_ws = ctx->xhat_patch = ctx->patch_x_ws = ctx->patch_attn_ws = nullptr;
     ctx->patch_sets = 1;
@@ -656,7 +655,6 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
         if (e == cudaSuccess) e = cudaMemset(*p, 0, n * sizeof(float));
     };
     alloc(&ctx->part, vis_all * c.n_heads);
-    alloc(&ctx->attn_ws, vis_all);
     alloc(&ctx->l1_ws, kSets * vis_all);
     ctx->vis_all = vis_all;
     ctx->step_parity = 0;
@@ -709,7 +707,6 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     if (!ctx) return;
     DeviceGuard guard(ctx->cfg.device);
     cudaFree(ctx->part);
-    cudaFree(ctx->attn_ws);
     cudaFree(ctx->l1_ws);
     cudaFree(ctx->ahat_state);
     cudaFree(ctx->mhat_state);
