@@ -91,6 +91,9 @@ def make_workload(name: str):
     if name == "config2":
         return W.config2_single_frame(), "configs[1]: 7B-shaped single frame, batch 1, D=4096, 32 heads x 128, " \
                                          "32 text + 256 2D + 512 3D tokens, bf16, FIXED keep 2D 40 % / 3D 30 %"
+    if name == "config2_fp8":
+        return W.config2_single_frame(dtype="fp8"), "configs[1] with q, k, v in 8-bit e4m3 (hidden bf16): 7B-shaped single frame, " \
+                                                    "32 text + 256 2D + 512 3D tokens, FIXED keep 2D 40 % / 3D 30 %"
     if name == "config1":
         return W.config1_tiny(), "configs[0]: tiny reference, fp32"
     if name == "config3":
@@ -110,13 +113,15 @@ def make_workload(name: str):
 def algorithmic_bytes(wl, kept_rows: int):
     """Bytes the method must move per step (read K and Q of the visual/text rows, read hidden for the
     norms in ADAPTIVE mode, read+write the kept rows of hidden/K/V, ~12 bytes of scores per token)."""
-    e = 2 if wl.dtype == "bf16" else 4
+    e = {"bf16": 2, "fp8": 2, "fp32": 4}[wl.dtype]          # hidden
+    eq = 1 if wl.dtype == "fp8" else e                       # q, k, v
     hd = wl.n_heads * wl.head_dim
+    hkv = (wl.extra.get("n_kv_heads", 0) or wl.n_heads) * wl.head_dim
     nv = wl.total_vis
     nt = sum(s.n_txt for s in wl.samples)
-    sal = (nv + nt) * hd * e
+    sal = (nv * hkv + nt * hd) * eq
     l1 = nv * wl.d_model * e if wl.mode in (1, 2) else 0
-    comp = 2 * kept_rows * (wl.d_model + 2 * hd) * e
+    comp = 2 * kept_rows * (wl.d_model * e + 2 * hkv * eq)
     return {"salience": sal, "l1": l1, "compact": comp, "scores": 12 * nv,
             "total": sal + l1 + comp + 12 * nv}
 
@@ -237,8 +242,9 @@ def run_ours(args, rank, local, world):
     wl, desc = make_workload(args.workload)
     step_t = wl.steps[-1]
     names = ("q", "k", "v", "hidden")
-    host = {n: (torch.from_numpy(getattr(step_t, n)).to(torch.bfloat16) if wl.dtype == "bf16"
-                else torch.from_numpy(getattr(step_t, n))).contiguous() for n in names}
+    tdt = {"bf16": torch.bfloat16, "fp32": torch.float32, "fp8": torch.float8_e4m3fn}[wl.dtype]
+    host = {n: torch.from_numpy(getattr(step_t, n)).to(torch.bfloat16 if (wl.dtype == "fp8" and n == "hidden") else tdt).contiguous()
+            for n in names}
     in_bytes = sum(t.numel() * t.element_size() for t in host.values())
 
     # A single-frame workload is a stream of independent requests: each step starts a fresh smoothed
@@ -448,7 +454,7 @@ def run_ours(args, rank, local, world):
     line = {"metric": "visual_tokens_per_s_pruned", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": K, "warmup": warm_replays * per_graph, "ms_per_step": ms_per_step,
             "latency_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": wl.dtype if wl.dtype != "fp32" else "f32", "data": "synthetic",
+            "dtype": {"bf16": "bf16", "fp32": "f32", "fp8": "e4m3"}[wl.dtype], "data": "synthetic",
             "config": {"workload": desc, "l2": f"inputs and outputs rotate over {n_sets} distinct sets "
                                                f"(about {touched * n_sets / 2**20:.0f} MiB touched per cycle, L2 is 126 MiB; "
                                                f"{(in_bytes + out_bytes_alloc) * n_sets / 2**20:.0f} MiB allocated)",

@@ -50,6 +50,8 @@ extern "C" {
 
 #define MVLA_DTYPE_BF16 0
 #define MVLA_DTYPE_FP32 1
+#define MVLA_DTYPE_FP8_E4M3 2   /* q, k, v in 8-bit floating point (e4m3, finite: no infinities); hidden stays bf16.
+                                   Tensor-core scoring only; not available together with patch_path */
 
 #define MVLA_SALIENCE_AUTO 0
 #define MVLA_SALIENCE_FMA  1
@@ -84,7 +86,7 @@ typedef struct mvla_ctx mvla_ctx;   /* opaque */
  * survives, the deterministic form of the 90 % background pruning (Sec. 4.2). */
 typedef struct mvla_config {
     int32_t device;            /* CUDA device ordinal */
-    int32_t dtype;             /* MVLA_DTYPE_*: element type of q, k, v, hidden */
+    int32_t dtype;             /* MVLA_DTYPE_*: element type of q, k, v, hidden (FP8_E4M3: of q, k, v; hidden bf16) */
     int32_t n_heads;           /* H: query heads (key / value heads: n_kv_heads below) */
     int32_t head_dim;          /* d: a multiple of 32 from 64 to 256 (64, 96, 128, ... 256) */
     int32_t d_model;           /* D: hidden width, multiple of 8 (bf16) / 4 (fp32) */

@@ -18,7 +18,9 @@ struct mvla_ctx {
     mvla_config cfg;
     int n_slots;
     int max_vis;
-    size_t elem;                 // bytes per input element
+    size_t elem;                 // bytes per element of hidden
+    size_t qk_elem;              // bytes per element of q, k, v (1 for e4m3, else = elem)
+    int hidden_dtype;            // MVLA_DTYPE_BF16 or MVLA_DTYPE_FP32
     bool use_umma;               // bf16 tensor-core salience path
     int kv_heads;                // key / value heads (== n_heads unless grouped)
     float* part;                 // [H][max_batch * max_vis] per-head partial scores
@@ -216,7 +218,7 @@ int tiles_of(const SampleDev& s)
     return (s.n_2d + kKeyTile - 1) / kKeyTile + (s.n_3d + kKeyTile - 1) / kKeyTile;
 }
 
-// 3-D view (head_dim, heads, rows) of a token-major [rows, H, d] bf16 tensor; boxes of 64 x 1 x
+// 3-D view (head_dim, heads, rows) of a token-major [rows, H, d] bf16 or e4m3 tensor; boxes of 128 bytes x 1 x
 // `box_rows` land in shared memory as `box_rows` rows of 128 bytes with the 128-byte swizzle.
 int32_t tensor_map(mvla_ctx* ctx, int which, const void* ptr, int64_t rows, int box_rows, const CUtensorMap** out)
 {
@@ -227,10 +229,12 @@ int32_t tensor_map(mvla_ctx* ctx, int which, const void* ptr, int64_t rows, int 
     const mvla_config& c = ctx->cfg;
     const cuuint64_t heads = static_cast<cuuint64_t>(which == 1 ? ctx->kv_heads : c.n_heads);   // map 1 is the key tensor
     cuuint64_t dims[3] = {static_cast<cuuint64_t>(c.head_dim), heads, static_cast<cuuint64_t>(rows)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(c.head_dim) * 2, static_cast<cuuint64_t>(c.head_dim) * heads * 2};
-    cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(box_rows)};
+    const cuuint64_t es = static_cast<cuuint64_t>(ctx->qk_elem);
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(c.head_dim) * es, static_cast<cuuint64_t>(c.head_dim) * heads * es};
+    cuuint32_t box[3] = {static_cast<cuuint32_t>(128 / es), 1, static_cast<cuuint32_t>(box_rows)};
     cuuint32_t estr[3] = {1, 1, 1};
-    const CUresult r = ctx->encode(&ctx->tm[which], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims,
+    const CUtensorMapDataType dt = es == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const CUresult r = ctx->encode(&ctx->tm[which], dt, 3, const_cast<void*>(ptr), dims,
                                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -275,11 +279,12 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
     cudaError_t e;
     const bool fast = ctx->use_umma && fast_salience_supported(tiles_per_cta);
     if (hidden && l1) {
-        e = launch_l1norm(bd, c.dtype, c.d_model, hidden, l1, st);
+        e = launch_l1norm(bd, ctx->hidden_dtype, c.d_model, hidden, l1, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
     if (fast) {
-        e = launch_salience_fast(bd, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, tq, tk, tiles_per_cta, cluster, npad,
+        e = launch_salience_fast(bd, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, static_cast<int>(ctx->qk_elem), tq, tk,
+                                 tiles_per_cta, cluster, npad,
                                  alpha.ptr && !acc64 ? nullptr : ctx->part,     // the patch path reads the attention copy only
                                  ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, st);
         if (used_acc64) *used_acc64 = acc64 != nullptr;
@@ -461,7 +466,7 @@ int32_t run_patch_indicators(mvla_ctx* ctx, unsigned set, const Plan& plan, int3
     }
     for (int first = 0; first < batch; first += kMaxChunk) {
         const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
-        const cudaError_t e = launch_patch_indicators(bd, ctx->cfg.n_heads, alpha, ctx->cfg.dtype, ctx->cfg.d_model, hidden,
+        const cudaError_t e = launch_patch_indicators(bd, ctx->cfg.n_heads, alpha, ctx->hidden_dtype, ctx->cfg.d_model, hidden,
                                                       x_out, attn_out, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
@@ -517,7 +522,7 @@ int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, cons
     int64_t cap = 0;                               // the row count is known only on the device: cover the capacity
     for (int b = 0; b < batch; ++b) cap += samples[b].n_txt + samples[b].n_2d + samples[b].n_3d;
     CompactJob job;
-    const int32_t kv_bytes = static_cast<int32_t>(ctx->kv_heads * ctx->cfg.head_dim * ctx->elem);
+    const int32_t kv_bytes = static_cast<int32_t>(ctx->kv_heads * ctx->cfg.head_dim * ctx->qk_elem);
     for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
     job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
 
@@ -532,7 +537,7 @@ int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, cons
         forked = true;
         const size_t nvis_b = static_cast<size_t>(plan.total_vis), npat_b = nvis_b / 2, in_rows = static_cast<size_t>(in->rows);
         const size_t hb = static_cast<size_t>(ctx->cfg.d_model) * ctx->elem, kb = static_cast<size_t>(kv_bytes);
-        const size_t qb = static_cast<size_t>(ctx->cfg.n_heads) * ctx->cfg.head_dim * ctx->elem;
+        const size_t qb = static_cast<size_t>(ctx->cfg.n_heads) * ctx->cfg.head_dim * ctx->qk_elem;
         const mvla_ctx::Range side[12] = {
             range_of(out->kept_idx, static_cast<size_t>(cap) * 4), range_of(out->out_offsets, (batch + 1) * 4u),
             range_of(out->budgets, batch * 8u), range_of(out->attn, nvis_b * 4), range_of(out->patch_x, npat_b * 16),
@@ -592,7 +597,8 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (!(c.beta >= 0.0 && c.beta <= 1.0) || !(c.floor_ratio >= 0.0 && c.floor_ratio <= 1.0) ||
         !std::isfinite(c.tau_2d) || !std::isfinite(c.tau_3d) || !std::isfinite(c.eps_3d))
         return MVLA_ERR_INVALID_ARG;
-    if (c.dtype != MVLA_DTYPE_BF16 && c.dtype != MVLA_DTYPE_FP32) return MVLA_ERR_UNSUPPORTED;
+    if (c.dtype != MVLA_DTYPE_BF16 && c.dtype != MVLA_DTYPE_FP32 && c.dtype != MVLA_DTYPE_FP8_E4M3) return MVLA_ERR_UNSUPPORTED;
+    if (c.dtype == MVLA_DTYPE_FP8_E4M3 && (c.salience_path == MVLA_SALIENCE_FMA || c.patch_path)) return MVLA_ERR_UNSUPPORTED;
     if (c.salience_path != MVLA_SALIENCE_AUTO && c.salience_path != MVLA_SALIENCE_FMA) return MVLA_ERR_INVALID_ARG;
     if ((c.patch_path != 0 && c.patch_path != 1) || c.kmeans_max_iter < 0 || !(c.obj_2d_min >= 0.0 && c.obj_2d_min <= 1.0))
         return MVLA_ERR_INVALID_ARG;
@@ -600,7 +606,7 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (c.n_kv_heads < 0 || (c.n_kv_heads > 0 && (c.n_kv_heads > c.n_heads || c.n_heads % c.n_kv_heads != 0))) return MVLA_ERR_INVALID_ARG;
     if (c.patch_path && c.n_kv_heads > 0 && c.n_kv_heads != c.n_heads) return MVLA_ERR_UNSUPPORTED;   // the patch path is built for ungrouped keys
     if (c.max_text > kMaxText || c.max_2d + c.max_3d > kMaxVis || c.max_batch > 64) return MVLA_ERR_UNSUPPORTED;
-    const size_t elem = c.dtype == MVLA_DTYPE_BF16 ? 2 : 4;
+    const size_t elem = c.dtype == MVLA_DTYPE_FP32 ? 4 : 2;       // hidden: fp32, or bf16 (also beside e4m3 q / k / v)
     if ((static_cast<size_t>(c.d_model) * elem) % 16 != 0) return MVLA_ERR_UNSUPPORTED;
 
     int ndev = 0;
@@ -620,7 +626,9 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     ctx->n_slots = c.n_state_slots > 0 ? c.n_state_slots : c.max_batch;
     ctx->max_vis = c.max_2d + c.max_3d;
     ctx->elem = elem;
-    ctx->use_umma = c.dtype == MVLA_DTYPE_BF16;
+    ctx->qk_elem = c.dtype == MVLA_DTYPE_FP8_E4M3 ? 1 : elem;
+    ctx->hidden_dtype = c.dtype == MVLA_DTYPE_FP32 ? MVLA_DTYPE_FP32 : MVLA_DTYPE_BF16;
+    ctx->use_umma = c.dtype != MVLA_DTYPE_FP32;
     ctx->kv_heads = c.n_kv_heads > 0 ? c.n_kv_heads : c.n_heads;
     if (c.salience_path == MVLA_SALIENCE_FMA) ctx->use_umma = false;
     ctx->part = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
@@ -816,7 +824,7 @@ int32_t mvla_compact(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, c
     rc = make_plan(ctx, 0, batch, samples, MVLA_MODE_FIXED, 0, false, &plan);
     if (rc != MVLA_OK) return rc;
     CompactJob job;
-    const int32_t kv_bytes = static_cast<int32_t>(ctx->kv_heads * ctx->cfg.head_dim * ctx->elem);
+    const int32_t kv_bytes = static_cast<int32_t>(ctx->kv_heads * ctx->cfg.head_dim * ctx->qk_elem);
     for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
     job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -905,7 +913,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     const bool adaptive = mode == MVLA_MODE_ADAPTIVE;
     const GateParams gp = gate_params(ctx, mode, adaptive);
     CompactJob job;
-    const int32_t kv_bytes = static_cast<int32_t>(ctx->kv_heads * ctx->cfg.head_dim * ctx->elem);
+    const int32_t kv_bytes = static_cast<int32_t>(ctx->kv_heads * ctx->cfg.head_dim * ctx->qk_elem);
     for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
     job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
 
@@ -920,7 +928,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     const unsigned par = ctx->step_parity;
     const size_t nvis_b = static_cast<size_t>(plan.total_vis), nout_b = static_cast<size_t>(plan.total_out);
     const size_t hb = static_cast<size_t>(ctx->cfg.d_model) * ctx->elem, kb = static_cast<size_t>(kv_bytes);
-    const size_t qb = static_cast<size_t>(ctx->cfg.n_heads) * ctx->cfg.head_dim * ctx->elem;
+    const size_t qb = static_cast<size_t>(ctx->cfg.n_heads) * ctx->cfg.head_dim * ctx->qk_elem;
     if ((flags & MVLA_FLAG_INPUTS_STABLE) && batch <= kMaxChunk && chunk_is_fast(ctx, chunk_of(plan, 0, batch))) {
         forked = true;
         // buffers the side-stream work touches: selection outputs, and the inputs of scoring

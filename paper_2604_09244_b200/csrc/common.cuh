@@ -96,7 +96,8 @@ struct AlphaOut {
 bool fast_salience_supported(int tiles_per_cta);
 // `kv_group`: query heads per key head (1 unless the keys are grouped); the key tensor map then has
 // n_heads / kv_group heads.
-cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, const CUtensorMap* tmap_q,
+// `esize`: bytes per element of q and k (2: bf16, 1: e4m3).
+cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
                                  bool free_running, AlphaOut alpha, cudaStream_t stream);

@@ -107,6 +107,23 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// The same for 8-bit floating-point operands (both e4m3), fp32 accumulate; one instruction covers 32
+// elements of the contraction.
+__device__ __forceinline__ void umma_e4m3(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "setp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Element size 2: bf16 operands; 1: e4m3 operands.  Either way one instruction consumes 32 bytes of every row.
+__device__ __forceinline__ void umma_by_size(int esize, uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                             uint32_t idesc, uint32_t accumulate)
+{
+    if (esize == 2) umma_bf16(d_tmem, a_desc, b_desc, idesc, accumulate);
+    else umma_e4m3(d_tmem, a_desc, b_desc, idesc, accumulate);
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -141,6 +158,15 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
 __device__ __forceinline__ uint32_t idesc_bf16_m128(int n)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+// Instruction descriptor: e4m3 x e4m3 -> fp32 (operand format code 0 for both), K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t idesc_e4m3_m128(int n)
+{
+    return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ uint32_t idesc_by_size(int esize, int n)
+{
+    return esize == 2 ? idesc_bf16_m128(n) : idesc_e4m3_m128(n);
 }
 
 // Reduce 16 per-thread values across the 32 lanes of a warp in 16 shuffles.  On return lane L

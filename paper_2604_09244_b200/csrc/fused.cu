@@ -62,7 +62,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
 template <int TCOL, int NTILE>
 __global__ void __launch_bounds__(kFastThreads, 1)
 salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
-                     const __grid_constant__ CUtensorMap tmap_k, int n_heads, int kv_group, int head_dim, int npad_max,
+                     const __grid_constant__ CUtensorMap tmap_k, int n_heads, int kv_group, int head_dim, int esize, int npad_max,
                      float* __restrict__ part, int64_t part_stride, unsigned long long* __restrict__ acc64,
                      int* status, int free_running, const AlphaOut alpha)
 {
@@ -85,7 +85,8 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     const uint32_t crank = cluster_ctarank();
     const uint32_t csize = gridDim.x;
     const int d = head_dim;
-    const int khalves = (d + 63) / 64;                    // 64 bf16 = one 128-byte swizzle row; a last partial box is zero-filled by TMA
+    const int khalves = (d * esize + 127) / 128;          // 128-byte swizzle rows (64 bf16 or 128 e4m3) per key; a last partial box is zero-filled by TMA
+    const int box_elems = 128 / esize;
     const float cscale = 1.4426950408889634f * rsqrtf(static_cast<float>(d));   // log2 domain
     const int tt0 = static_cast<int>(crank) * NTILE;
     uint8_t* Ks = dyn_smem;                               // [tile][khalf][128 rows x 128 B]
@@ -120,14 +121,14 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         mbar_expect_tx(bar_full, static_cast<uint32_t>(khalves) * (npad * 128 + live * 16384));
         for (int kh = 0; kh < khalves; ++kh)
             for (int c = 0; c < npad / 16; ++c)
-                tma_load_3d(smem_u32(Qs + kh * npad * 128 + c * 2048), &tmap_q, kh * 64, h,
+                tma_load_3d(smem_u32(Qs + kh * npad * 128 + c * 2048), &tmap_q, kh * box_elems, h,
                             s.seq_off + s.off_txt + c * 16, bar_full);
 #pragma unroll
         for (int t = 0; t < NTILE; ++t) {
             if (valid[t] <= 0) continue;
             const int row0 = tile_info(s, tt0 + t).row0;
             for (int kh = 0; kh < khalves; ++kh)
-                tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * 64, h / kv_group, row0, bar_full);
+                tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * box_elems, h / kv_group, row0, bar_full);
         }
     }
     if (tid < kMaxText) s_w[tid] = 0.f;
@@ -149,7 +150,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         }
         if (got) {
             tc_fence_after();
-            const uint32_t idesc = idesc_bf16_m128(npad);
+            const uint32_t idesc = idesc_by_size(esize, npad);
 #pragma unroll
             for (int t = 0; t < NTILE; ++t) {
                 if (valid[t] <= 0) continue;
@@ -157,7 +158,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
                     const int kh = kb >> 2, kin = kb & 3;          // 4 K-steps of 16 inside a 64-wide half
                     const uint64_t a = smem_desc_sw128(smem_u32(Ks + (t * khalves + kh) * 16384) + kin * 32);
                     const uint64_t b = smem_desc_sw128(smem_u32(Qs + kh * npad * 128) + kin * 32);
-                    umma_bf16(tmem_base + t * TCOL, a, b, idesc, kb > 0 ? 1u : 0u);
+                    umma_by_size(esize, tmem_base + t * TCOL, a, b, idesc, kb > 0 ? 1u : 0u);
                 }
             }
         }
@@ -291,11 +292,11 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
 }
 
 template <int TCOL, int NTILE>
-cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, const CUtensorMap* tq,
+cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tq,
                           const CUtensorMap* tk, int cluster, int npad, float* part, int64_t part_stride,
                           unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, cudaStream_t stream)
 {
-    const size_t smem = 1024 + static_cast<size_t>((head_dim + 63) / 64) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
+    const size_t smem = 1024 + static_cast<size_t>((head_dim * esize + 127) / 128) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
     auto kern = salience_fast_kernel<TCOL, NTILE>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
@@ -312,14 +313,14 @@ cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int he
     attr[1] = pdl_attribute();
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, kv_group, head_dim, npad, part, part_stride, acc64, status, free_running, alpha);
+    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, kv_group, head_dim, esize, npad, part, part_stride, acc64, status, free_running, alpha);
 }
 
 }  // namespace
 
 bool fast_salience_supported(int tiles_per_cta) { return tiles_per_cta >= 1 && tiles_per_cta <= 2; }
 
-cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, const CUtensorMap* tmap_q,
+cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
                                  bool free_running, AlphaOut alpha, cudaStream_t stream)
@@ -327,7 +328,7 @@ cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group,
     const int tcol = npad <= 16 ? 16 : (npad <= 32 ? 32 : 64);
 #define MVLA_FAST(TC, NTL)                                                                                      \
     if (tcol == TC && tiles_per_cta == NTL)                                                                     \
-        return launch_fast_t<TC, NTL>(bd, n_heads, kv_group, head_dim, tmap_q, tmap_k, cluster, npad, part, part_stride, \
+        return launch_fast_t<TC, NTL>(bd, n_heads, kv_group, head_dim, esize, tmap_q, tmap_k, cluster, npad, part, part_stride, \
                                       acc64, status, free_running ? 1 : 0, alpha, stream);
     MVLA_FAST(16, 1) MVLA_FAST(32, 1) MVLA_FAST(64, 1) MVLA_FAST(16, 2) MVLA_FAST(32, 2) MVLA_FAST(64, 2)
 #undef MVLA_FAST

@@ -25,7 +25,7 @@ template <typename T, bool UMMA>
 __global__ void __launch_bounds__(kThreads, 1)
 salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
                 const __grid_constant__ CUtensorMap tmap_k, const T* __restrict__ q,
-                const T* __restrict__ k, int n_heads, int kv_group, int head_dim, int tiles_per_cta, int npad,
+                const T* __restrict__ k, int n_heads, int kv_group, int head_dim, int esize, int tiles_per_cta, int npad,
                 float* __restrict__ part, int64_t part_stride, int* status, const AlphaOut alpha)
 {
     extern __shared__ uint8_t dyn_smem_raw[];
@@ -57,7 +57,8 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
     bool ok = true;
 
     if constexpr (UMMA) {
-        const int khalves = (d + 63) / 64;                    // 64 bf16 = one 128-byte swizzle row; a last partial box is zero-filled by TMA
+        const int khalves = (d * esize + 127) / 128;          // 128-byte swizzle rows (64 bf16 or 128 e4m3) per key; a last partial box is zero-filled by TMA
+        const int box_elems = 128 / esize;
         uint8_t* Ks = dyn_smem;                               // [tile][khalf][128 rows x 128 B]
         uint8_t* Qs = dyn_smem + static_cast<size_t>(tiles_per_cta) * khalves * 16384;   // [khalf][npad rows x 128 B]
         const uint32_t bar_full = smem_u32(&s_bar[0]), bar_mma = smem_u32(&s_bar[1]);
@@ -75,13 +76,13 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
             mbar_expect_tx(bar_full, bytes);
             for (int kh = 0; kh < khalves; ++kh)
                 for (int c = 0; c < npad / 16; ++c)
-                    tma_load_3d(smem_u32(Qs + kh * npad * 128 + c * 2048), &tmap_q, kh * 64, h,
+                    tma_load_3d(smem_u32(Qs + kh * npad * 128 + c * 2048), &tmap_q, kh * box_elems, h,
                                 s.seq_off + s.off_txt + c * 16, bar_full);
             for (int t = 0; t < tiles_per_cta; ++t) {
                 const TileInfo ti = tile_info(s, tt0 + t);
                 if (ti.valid <= 0) continue;
                 for (int kh = 0; kh < khalves; ++kh)
-                    tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * 64, hk, ti.row0, bar_full);
+                    tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * box_elems, hk, ti.row0, bar_full);
             }
         }
         if (warp == 1) tmem_alloc(smem_u32(&s_tmem), tmem_cols);
@@ -98,14 +99,14 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
             }
             if (got) {
                 tc_fence_after();
-                const uint32_t idesc = idesc_bf16_m128(npad);
+                const uint32_t idesc = idesc_by_size(esize, npad);
                 for (int t = 0; t < tiles_per_cta; ++t) {
                     if (tile_info(s, tt0 + t).valid <= 0) continue;
                     for (int kb = 0; kb < khalves * 4; ++kb) {     // columns past d are zeros
                         const int kh = kb >> 2, kin = kb & 3;      // 4 K-steps of 16 inside a 64-wide half
                         const uint64_t a = smem_desc_sw128(smem_u32(Ks + (t * khalves + kh) * 16384) + kin * 32);
                         const uint64_t b = smem_desc_sw128(smem_u32(Qs + kh * npad * 128) + kin * 32);
-                        umma_bf16(tmem_base + t * tcol, a, b, idesc, kb > 0 ? 1u : 0u);
+                        umma_by_size(esize, tmem_base + t * tcol, a, b, idesc, kb > 0 ? 1u : 0u);
                     }
                 }
             }
@@ -326,14 +327,14 @@ l1norm_kernel(const __grid_constant__ BatchDesc bd, int d_model, const T* __rest
 }
 
 template <typename T, bool UMMA>
-cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, const void* q, const void* k,
+cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const void* q, const void* k,
                               const CUtensorMap* tq, const CUtensorMap* tk, int tiles_per_cta, int cluster,
                               int npad, float* part, int64_t part_stride, int* status, AlphaOut alpha,
                               cudaStream_t stream)
 {
     size_t smem;
     if (UMMA)
-        smem = 1024 + static_cast<size_t>((head_dim + 63) / 64) * (static_cast<size_t>(tiles_per_cta) * 16384 + npad * 128);
+        smem = 1024 + static_cast<size_t>((head_dim * esize + 127) / 128) * (static_cast<size_t>(tiles_per_cta) * 16384 + npad * 128);
     else
         smem = 1024 + sizeof(float) * (static_cast<size_t>(npad) * head_dim + kKeyTile * (head_dim + 1) +
                                 static_cast<size_t>(tiles_per_cta) * npad * kKeyTile);
@@ -355,7 +356,7 @@ cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int kv_group, in
     cfg.numAttrs = 1;
     static const CUtensorMap zero_map = {};
     return cudaLaunchKernelEx(&cfg, kern, bd, tq ? *tq : zero_map, tk ? *tk : zero_map,
-                              static_cast<const T*>(q), static_cast<const T*>(k), n_heads, kv_group, head_dim,
+                              static_cast<const T*>(q), static_cast<const T*>(k), n_heads, kv_group, head_dim, esize,
                               tiles_per_cta, npad, part, part_stride, status, alpha);
 }
 
@@ -366,14 +367,19 @@ cudaError_t launch_salience(const BatchDesc& bd, int dtype, int n_heads, int kv_
                             bool use_umma, int tiles_per_cta, int cluster, int npad, float* part,
                             int64_t part_stride, int* status, AlphaOut alpha, cudaStream_t stream)
 {
+    if (dtype == MVLA_DTYPE_FP8_E4M3) {      // tensor cores only: there is no FMA path for 8-bit inputs
+        if (!use_umma) return cudaErrorInvalidConfiguration;
+        return launch_salience_t<uint8_t, true>(bd, n_heads, kv_group, head_dim, 1, q, k, tmap_q, tmap_k, tiles_per_cta,
+                                                cluster, npad, part, part_stride, status, alpha, stream);
+    }
     if (dtype == MVLA_DTYPE_BF16) {
         if (use_umma)
-            return launch_salience_t<__nv_bfloat16, true>(bd, n_heads, kv_group, head_dim, q, k, tmap_q, tmap_k, tiles_per_cta,
+            return launch_salience_t<__nv_bfloat16, true>(bd, n_heads, kv_group, head_dim, 2, q, k, tmap_q, tmap_k, tiles_per_cta,
                                                           cluster, npad, part, part_stride, status, alpha, stream);
-        return launch_salience_t<__nv_bfloat16, false>(bd, n_heads, kv_group, head_dim, q, k, nullptr, nullptr, tiles_per_cta,
+        return launch_salience_t<__nv_bfloat16, false>(bd, n_heads, kv_group, head_dim, 2, q, k, nullptr, nullptr, tiles_per_cta,
                                                        cluster, npad, part, part_stride, status, alpha, stream);
     }
-    return launch_salience_t<float, false>(bd, n_heads, kv_group, head_dim, q, k, nullptr, nullptr, tiles_per_cta, cluster,
+    return launch_salience_t<float, false>(bd, n_heads, kv_group, head_dim, 4, q, k, nullptr, nullptr, tiles_per_cta, cluster,
                                            npad, part, part_stride, status, alpha, stream);
 }
 

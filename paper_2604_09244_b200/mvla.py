@@ -22,7 +22,7 @@ ERR_CAPACITY, ERR_TIMEOUT, ERR_STATE = -5, -6, -7
 _ERR_NAMES = {-1: "MVLA_ERR_INVALID_ARG", -2: "MVLA_ERR_UNSUPPORTED", -3: "MVLA_ERR_OOM",
               -4: "MVLA_ERR_CUDA", -5: "MVLA_ERR_CAPACITY", -6: "MVLA_ERR_TIMEOUT",
               -7: "MVLA_ERR_STATE"}
-DTYPE_BF16, DTYPE_FP32 = 0, 1
+DTYPE_BF16, DTYPE_FP32, DTYPE_FP8_E4M3 = 0, 1, 2
 MODE_FIXED, MODE_ADAPTIVE, MODE_PATCH = 0, 1, 2
 LABEL_BG, LABEL_ROB, LABEL_OBJ = 0, 1, 2
 FLAG_RESET_STATE, FLAG_NO_STATE_UPDATE, FLAG_INPUTS_STABLE = 1, 2, 4
@@ -179,7 +179,8 @@ class PruneContext:
             device = torch.cuda.current_device()
         self.device = torch.device("cuda", device)
         self.torch_dtype = dtype
-        code = {torch.bfloat16: DTYPE_BF16, torch.float32: DTYPE_FP32}[dtype]
+        code = {torch.bfloat16: DTYPE_BF16, torch.float32: DTYPE_FP32, torch.float8_e4m3fn: DTYPE_FP8_E4M3}[dtype]
+        self.hidden_dtype = torch.bfloat16 if dtype == torch.float8_e4m3fn else dtype   # e4m3 is for q, k, v only
         self.cfg = Config(device, code, n_heads, head_dim, d_model, max_batch, max_text, max_2d,
                           max_3d, n_prune_points, n_state_slots, window_k, cold_start_full_keep,
                           salience_path, tau_2d, tau_3d, beta, eps_3d, floor_ratio, obj_2d_min, patch_path,
@@ -209,7 +210,7 @@ class PruneContext:
         c, dev, dt = self.cfg, self.device, self.torch_dtype
         mk = lambda *shape, dtype=dt: torch.empty(*shape, dtype=dtype, device=dev)
         return StepOutputs(
-            out_hidden=mk(rows, c.d_model) if hidden else None,
+            out_hidden=mk(rows, c.d_model, dtype=self.hidden_dtype) if hidden else None,
             out_k=mk(rows, c.n_kv_heads or c.n_heads, c.head_dim) if kv else None,
             out_v=mk(rows, c.n_kv_heads or c.n_heads, c.head_dim) if kv else None,
             kept_idx=mk(rows, dtype=torch.int32),
@@ -316,7 +317,7 @@ class PruneContext:
 def context_for(wl, *, max_batch=None, n_prune_points=1, n_state_slots=0, salience_path=SALIENCE_AUTO,
                 device=None, patch_path=None) -> PruneContext:
     """A context sized for a synthetic workload (see ``workloads``)."""
-    dt = {"bf16": torch.bfloat16, "fp32": torch.float32}[wl.dtype]
+    dt = {"bf16": torch.bfloat16, "fp32": torch.float32, "fp8": torch.float8_e4m3fn}[wl.dtype]
     return PruneContext(dtype=dt, n_heads=wl.n_heads, head_dim=wl.head_dim, d_model=wl.d_model,
                         max_batch=max_batch or len(wl.samples),
                         max_text=max(s.n_txt for s in wl.samples),
@@ -337,6 +338,8 @@ def to_device(arr, dtype: str, device) -> torch.Tensor:
     t = torch.from_numpy(arr)
     if dtype == "bf16":
         t = t.to(torch.bfloat16)      # exact: the values are already bf16-representable
+    elif dtype == "fp8":
+        t = t.to(torch.float8_e4m3fn)  # exact likewise
     return t.to(device).contiguous()
 
 

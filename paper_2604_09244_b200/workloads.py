@@ -51,7 +51,24 @@ def bf16_bits(x: np.ndarray) -> np.ndarray:
     return (x.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
 
 
+def round_to_e4m3(x: np.ndarray) -> np.ndarray:
+    """Round float32 values to the nearest 8-bit e4m3 value (finite format, largest magnitude 448, ties to
+    even, saturating); the result is float32 holding exactly representable e4m3 values."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).clamp(-448.0, 448.0)
+    return t.to(torch.float8_e4m3fn).to(torch.float32).numpy()
+
+
+def e4m3_bits(x: np.ndarray) -> np.ndarray:
+    """uint8 bit patterns of float32 values that are already e4m3-exact."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(torch.float8_e4m3fn)
+    return t.view(torch.uint8).numpy()
+
+
 def round_to_dtype(x: np.ndarray, dtype: str) -> np.ndarray:
+    if dtype == "fp8":
+        return round_to_e4m3(x)
     if dtype == "bf16":
         return round_to_bf16(x)
     if dtype == "fp32":
@@ -100,7 +117,7 @@ class Tensors:
 @dataclass
 class Workload:
     name: str
-    dtype: str                 # "bf16" | "fp32"
+    dtype: str                 # "bf16" | "fp32" | "fp8" (q, k, v in e4m3; hidden bf16)
     n_heads: int
     head_dim: int
     d_model: int
@@ -152,7 +169,8 @@ def _project(hidden: np.ndarray, w, H: int, d: int, dtype: str, H_kv: int = 0) -
     q = (hidden @ wq).reshape(S, H, d)
     k = (hidden @ wk).reshape(S, H_kv or H, d)
     v = (hidden @ wv).reshape(S, H_kv or H, d)
-    return Tensors(hidden=round_to_dtype(hidden, dtype), q=round_to_dtype(q, dtype),
+    # "fp8": q, k, v in e4m3, the hidden states stay bf16
+    return Tensors(hidden=round_to_dtype(hidden, "bf16" if dtype == "fp8" else dtype), q=round_to_dtype(q, dtype),
                    k=round_to_dtype(k, dtype), v=round_to_dtype(v, dtype))
 
 

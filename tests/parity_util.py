@@ -12,7 +12,9 @@ SALIENCE_ATOL = 1e-12
 
 def device_tensors(wl, step=0, device="cuda"):
     t = wl.steps[step]
-    return {name: mvla.to_device(getattr(t, name), wl.dtype, device) for name in ("q", "k", "v", "hidden")}
+    # with e4m3 q / k / v the hidden states stay bf16
+    return {name: mvla.to_device(getattr(t, name), "bf16" if (wl.dtype == "fp8" and name == "hidden") else wl.dtype, device)
+            for name in ("q", "k", "v", "hidden")}
 
 
 def diag_records(out, batch):
@@ -73,7 +75,11 @@ def check_compaction(wl_tensors_np, dev_out, s, kept_gpu, row0, dtype):
         src = getattr(wl_tensors_np, name)
         n = len(kept_gpu)
         got = out_t[row0:row0 + n]
-        if dtype == "bf16":
+        if dtype == "fp8" and name != "hidden":
+            got_bits = got.view(torch.uint8).cpu().numpy().reshape(n, -1)
+            src_bits = W.e4m3_bits(src[s.seq_off + np.asarray(kept_gpu)]).reshape(n, -1)
+            ref_bits = W.e4m3_bits(oracle.compact(src, s.seq_off, kept_gpu)).reshape(n, -1)
+        elif dtype in ("bf16", "fp8"):
             got_bits = got.view(torch.int16).cpu().numpy().view(np.uint16).reshape(n, -1)
             src_bits = W.bf16_bits(src[s.seq_off + np.asarray(kept_gpu)]).reshape(n, -1)
             ref_bits = W.bf16_bits(oracle.compact(src, s.seq_off, kept_gpu)).reshape(n, -1)

@@ -559,3 +559,32 @@ def test_head_sharded_step_two_ranks_emulated_on_one_gpu():
     assert np.array_equal(o.kept_idx[:n].cpu().numpy(), kept_by_rank[0])
     for c in ctxs + [full]:
         c.close()
+
+
+def test_fp8_keys_small_ragged_and_grouped():
+    # q, k, v in e4m3 (hidden bf16): ragged tiles, two samples, grouped key heads, head_dim 64 and 128
+    for d, hkv in ((128, 0), (64, 2)):
+        wl = W.small_workload(81, batch=2, D=256, H=4, d=d, dtype="fp8", n_txt=(7, 33), n_2d=(130, 70), n_3d=(150, 300),
+                              n_kv_heads=hkv)
+        ctx = mvla.context_for(wl)
+        dev = device_tensors(wl)
+        assert dev["k"].dtype == torch.float8_e4m3fn and dev["hidden"].dtype == torch.bfloat16
+        attn, l1 = ctx.salience(wl.samples, dev["q"], dev["k"], dev["hidden"])
+        torch.cuda.synchronize()
+        attn = attn.cpu().numpy()
+        t = wl.steps[0]
+        vis = 0
+        for s in wl.samples:
+            ref = oracle.salience_gqa(t.q, t.k, 4, hkv or 4, d, s)
+            assert_salience_close(attn[vis:vis + s.n_vis], ref, "e4m3 scores")
+            vis += s.n_vis
+        if not hkv:
+            run_and_check_step(ctx, wl, 0, [oracle.State(s.n_vis) for s in wl.samples])
+        ctx.close()
+
+
+def test_fp8_step_single_frame_shape():
+    wl = W.config2_single_frame(dtype="fp8")          # 32 text + 256 2D + 512 3D, D = 4096, 32 heads x 128
+    ctx = mvla.context_for(wl)
+    run_and_check_step(ctx, wl, 0, [oracle.State(s.n_vis) for s in wl.samples])
+    ctx.close()
