@@ -55,7 +55,7 @@ NCU_SOURCES = {
 NCU_DIGEST = {             # stage -> sha256 of its sources when the counters were taken
     "salience": "ffd62393d650c2e5efee3b5134b9c65f706d6194bcd7bab2db45ab591ca9d630",
     "select": "4d8d621fb08d123bffa8c27634f0c2082dc1552bbf6292d5b331160edb121b84",
-    "compact": "f4d0a99750e4b9890a6a22bd5e31e38a5e660da99bf48f72b03ede77da5636f0",
+    "compact": "27d2a238f0b0e282dbdbc78fc8456f3149d3b82f90688d8421ddd0830ffa6299",
     "patch_salience": "bc910990d2d34e5090584ef1d24d33ef11b19d0f6cdf72918256a3500f7fb1a7",
     "patch_select": "5e9cc17fa3b0a30e57bac3560d78233fc067a917a9373740935fea78df45dbe6",
 }

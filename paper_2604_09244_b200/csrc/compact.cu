@@ -6,6 +6,8 @@
 // then four stores.  The loads bypass L1 (read once), the stores are streaming.
 #include "common.cuh"
 
+#include <algorithm>
+
 namespace mvla {
 namespace {
 
@@ -39,46 +41,52 @@ compact_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ Com
                int32_t chunk_first, int32_t batch_total)
 {
     const int lane = threadIdx.x & 31;
-    const int64_t unit = static_cast<int64_t>(blockIdx.x) * kWarpsPerBlock + (threadIdx.x >> 5);
     const int per_row = a.seg_begin[3];
-    if (unit >= static_cast<int64_t>(chunk_rows) * per_row) return;
-    const int r = static_cast<int>(unit / per_row);       // output row inside this chunk
-    const int u = static_cast<int>(unit - static_cast<int64_t>(r) * per_row);
-    const int orow = chunk_row0 + r;
+    int64_t unit = static_cast<int64_t>(blockIdx.x) * kWarpsPerBlock + (threadIdx.x >> 5);
+    int64_t n_units = static_cast<int64_t>(chunk_rows) * per_row;
+    if (!out_offsets && unit >= n_units) return;
 
     asm volatile("griddepcontrol.wait;" ::: "memory");      // kept_idx comes from the kernel before this one
     // Only now may the next kernel become resident: by then this step's selection is complete.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    // which sample owns output row `orow` (samples are few: linear scan)
-    int b = 0;
-    if (out_offsets) {            // offsets known only on the device: scan the whole batch
-        if (orow >= out_offsets[batch_total]) return;      // the launch covered a capacity bound, not the row count
-        while (b + 1 < batch_total && orow >= out_offsets[b + 1]) ++b;
-        b -= chunk_first;
-        if (b < 0 || b >= bd.n) return;      // row belongs to another launch's samples
-    } else {
-        while (b + 1 < bd.n && orow >= bd.s[b + 1].out_off) ++b;
-    }
-    const int64_t srow = static_cast<int64_t>(bd.s[b].seq_off) + kept_idx[orow];
+    // Row count known only on the device: the launch covers a capacity bound with a bounded grid, and the
+    // warps stride over the rows that exist.
+    const int64_t stride = out_offsets ? static_cast<int64_t>(gridDim.x) * kWarpsPerBlock : n_units;
+    if (out_offsets) n_units = min(n_units, static_cast<int64_t>(out_offsets[batch_total] - chunk_row0) * per_row);
+    for (; unit < n_units; unit += stride) {
+        const int r = static_cast<int>(unit / per_row);       // output row inside this chunk
+        const int u = static_cast<int>(unit - static_cast<int64_t>(r) * per_row);
+        const int orow = chunk_row0 + r;
+        // which sample owns output row `orow` (samples are few: linear scan)
+        int b = 0;
+        if (out_offsets) {            // offsets known only on the device: scan the whole batch
+            while (b + 1 < batch_total && orow >= out_offsets[b + 1]) ++b;
+            b -= chunk_first;
+            if (b < 0 || b >= bd.n) continue;    // row belongs to another launch's samples
+        } else {
+            while (b + 1 < bd.n && orow >= bd.s[b + 1].out_off) ++b;
+        }
+        const int64_t srow = static_cast<int64_t>(bd.s[b].seq_off) + kept_idx[orow];
 
-    const int tsel = u >= a.seg_begin[2] ? 2 : (u >= a.seg_begin[1] ? 1 : 0);
-    const int seg = u - a.seg_begin[tsel];
-    const int rb = a.row_bytes[tsel];
-    const uint8_t* sp = a.src[tsel] + srow * rb + static_cast<int64_t>(seg) * kSegBytes;
-    uint8_t* dp = a.dst[tsel] + static_cast<int64_t>(orow) * rb + static_cast<int64_t>(seg) * kSegBytes;
-    const int nbytes = min(kSegBytes, rb - seg * kSegBytes);
-    const int nvec = nbytes >> 4;
+        const int tsel = u >= a.seg_begin[2] ? 2 : (u >= a.seg_begin[1] ? 1 : 0);
+        const int seg = u - a.seg_begin[tsel];
+        const int rb = a.row_bytes[tsel];
+        const uint8_t* sp = a.src[tsel] + srow * rb + static_cast<int64_t>(seg) * kSegBytes;
+        uint8_t* dp = a.dst[tsel] + static_cast<int64_t>(orow) * rb + static_cast<int64_t>(seg) * kSegBytes;
+        const int nbytes = min(kSegBytes, rb - seg * kSegBytes);
+        const int nvec = nbytes >> 4;
 
-    uint4 v[4];
+        uint4 v[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int idx = lane + i * 32;
-        if (idx < nvec) v[i] = ld_stream(reinterpret_cast<const uint4*>(sp) + idx);
-    }
+        for (int i = 0; i < 4; ++i) {
+            const int idx = lane + i * 32;
+            if (idx < nvec) v[i] = ld_stream(reinterpret_cast<const uint4*>(sp) + idx);
+        }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int idx = lane + i * 32;
-        if (idx < nvec) st_stream(reinterpret_cast<uint4*>(dp) + idx, v[i]);
+        for (int i = 0; i < 4; ++i) {
+            const int idx = lane + i * 32;
+            if (idx < nvec) st_stream(reinterpret_cast<uint4*>(dp) + idx, v[i]);
+        }
     }
 }
 
@@ -102,7 +110,8 @@ cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int
     a.seg_begin[3] = total;
     if (total == 0 || chunk_rows <= 0) return cudaSuccess;
     const int64_t units = static_cast<int64_t>(chunk_rows) * total;
-    const int64_t blocks = (units + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    int64_t blocks = (units + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    if (out_offsets) blocks = std::min<int64_t>(blocks, 148 * 32);     // capacity launch: a bounded grid strides over the rows that exist
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(blocks));
     cfg.blockDim = dim3(kWarpsPerBlock * 32);
