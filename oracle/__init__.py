@@ -112,6 +112,9 @@ def load(path: str):
                                         C.c_int32, C.POINTER(CState), ip, C.POINTER(CDiag),
                                         dp, dp, dp, dp]
         L.oracle_prune_step.restype = C.c_int32
+        L.oracle_decide_step.argtypes = [dp, dp, sp, pp, C.c_int32, C.POINTER(CState), ip,
+                                         C.POINTER(CDiag), dp, dp]
+        L.oracle_decide_step.restype = C.c_int32
         L.oracle_num_threads.argtypes = []
         L.oracle_num_threads.restype = C.c_int32
         # Alg. 1 patch by patch
@@ -328,6 +331,25 @@ def prune_step(q, k, hidden, n_heads, head_dim, d_model, s, params: CParams, mod
                                 mode, C.byref(state.c), kept.ctypes.data_as(C.POINTER(C.c_int32)),
                                 C.byref(dg), dp(attn), dp(l1), dp(ahat), dp(z))
     return StepResult(kept[:n].copy(), attn, l1 if mode == MODE_ADAPTIVE else None, ahat, z, dg.t,
+                      np.array(dg.x[:]), np.array(dg.mhat[:]), dg.c_s1, dg.c_s2, dg.c_final,
+                      dg.k_2d, dg.k_3d, bool(dg.near_half), bool(dg.near_gate))
+
+
+def decide_step(a, l1, s, params: CParams, mode: int, state: State) -> StepResult:
+    """Alg. 1 from the scores on: `a` [n_vis] attention scores, `l1` [n_vis] feature norms or None."""
+    a, ap = _f64(a)
+    lp = None
+    if l1 is not None:
+        l1, lp = _f64(l1)
+    cs = c_sample(s)
+    nv = cs.n_2d + cs.n_3d
+    kept = np.zeros(cs.n_txt + nv, dtype=np.int32)
+    ahat = np.zeros(nv); z = np.zeros(nv)
+    dg = CDiag()
+    dp = lambda v: v.ctypes.data_as(C.POINTER(C.c_double))
+    n = lib().oracle_decide_step(ap, lp, C.byref(cs), C.byref(params), mode, C.byref(state.c),
+                                 kept.ctypes.data_as(C.POINTER(C.c_int32)), C.byref(dg), dp(ahat), dp(z))
+    return StepResult(kept[:n].copy(), a.copy(), None if l1 is None else l1.copy(), ahat, z, dg.t,
                       np.array(dg.x[:]), np.array(dg.mhat[:]), dg.c_s1, dg.c_s2, dg.c_final,
                       dg.k_2d, dg.k_3d, bool(dg.near_half), bool(dg.near_gate))
 

@@ -258,26 +258,17 @@ void oracle_compact(const void *src, int64_t row_bytes, int32_t seq_off,
                (const char *)src + ((int64_t)seq_off + kept_idx[r]) * row_bytes, (size_t)row_bytes);
 }
 
-/* ---- Alg. 1 as a whole, for one sample ---- */
-int32_t oracle_prune_step(const float *q, const float *k, const float *hidden,
-                          int32_t n_heads, int32_t head_dim, int32_t d_model,
-                          const oracle_sample *s, const oracle_params *p, int32_t mode,
-                          oracle_state *st, int32_t *kept_idx, oracle_diag *diag,
-                          double *attn_out, double *l1_out, double *ahat_out, double *z_out)
+/* ---- Alg. 1 from the scores on: everything that follows the attention and the feature norms ---- */
+int32_t oracle_decide_step(const double *a, const double *l1, const oracle_sample *s,
+                           const oracle_params *p, int32_t mode, oracle_state *st,
+                           int32_t *kept_idx, oracle_diag *diag, double *ahat_out, double *z_out)
 {
     const int32_t n2 = s->n_2d, n3 = s->n_3d, nv = n2 + n3;
-    double *a = (double *)malloc((size_t)nv * sizeof(double));
     double *z = (double *)malloc((size_t)nv * sizeof(double));
-    double *l1 = NULL;
     double x[4];
     oracle_diag dg;
     memset(&dg, 0, sizeof dg);
 
-    oracle_salience(q, k, n_heads, head_dim, s, a);
-    if (mode == ORACLE_MODE_ADAPTIVE) {
-        l1 = (double *)malloc((size_t)nv * sizeof(double));
-        oracle_l1norm(hidden, d_model, s, l1);
-    }
     oracle_indicators(a, l1, n2, n3, x);
 
     /* action-iteration stage first (Alg. 1): smooth the per-token scores and the indicators */
@@ -286,6 +277,7 @@ int32_t oracle_prune_step(const float *q, const float *k, const float *hidden,
     oracle_state_update(t, p->window_k, p->beta, 4, x, st->mhat);
     st->t = t;
 
+    /* the later stages are written on the predicted (hatted) quantities */
     oracle_normalise(st->ahat, n2, n3, z);
     oracle_gates(st->mhat, p, &dg.c_s1, &dg.c_s2, &dg.c_final, &dg.near_gate);
 
@@ -303,11 +295,32 @@ int32_t oracle_prune_step(const float *q, const float *k, const float *hidden,
     memcpy(dg.x, x, sizeof x);
     memcpy(dg.mhat, st->mhat, sizeof x);
     if (diag) *diag = dg;
-    if (attn_out) memcpy(attn_out, a, (size_t)nv * sizeof(double));
-    if (l1_out && l1) memcpy(l1_out, l1, (size_t)nv * sizeof(double));
     if (ahat_out) memcpy(ahat_out, st->ahat, (size_t)nv * sizeof(double));
     if (z_out) memcpy(z_out, z, (size_t)nv * sizeof(double));
-    free(a); free(z); free(l1);
+    free(z);
+    return n_kept;
+}
+
+/* ---- Alg. 1 as a whole, for one sample: scores and norms, then the decisions above ---- */
+int32_t oracle_prune_step(const float *q, const float *k, const float *hidden,
+                          int32_t n_heads, int32_t head_dim, int32_t d_model,
+                          const oracle_sample *s, const oracle_params *p, int32_t mode,
+                          oracle_state *st, int32_t *kept_idx, oracle_diag *diag,
+                          double *attn_out, double *l1_out, double *ahat_out, double *z_out)
+{
+    const int32_t nv = s->n_2d + s->n_3d;
+    double *a = (double *)malloc((size_t)nv * sizeof(double));
+    double *l1 = NULL;
+
+    oracle_salience(q, k, n_heads, head_dim, s, a);
+    if (mode == ORACLE_MODE_ADAPTIVE) {
+        l1 = (double *)malloc((size_t)nv * sizeof(double));
+        oracle_l1norm(hidden, d_model, s, l1);
+    }
+    const int32_t n_kept = oracle_decide_step(a, l1, s, p, mode, st, kept_idx, diag, ahat_out, z_out);
+    if (attn_out) memcpy(attn_out, a, (size_t)nv * sizeof(double));
+    if (l1_out && l1) memcpy(l1_out, l1, (size_t)nv * sizeof(double));
+    free(a); free(l1);
     return n_kept;
 }
 

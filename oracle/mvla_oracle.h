@@ -122,7 +122,16 @@ int32_t oracle_select(const double *z, const oracle_sample *s, int32_t k_2d, int
 void oracle_compact(const void *src, int64_t row_bytes, int32_t seq_off,
                     const int32_t *kept_idx, int32_t n_kept, void *dst);
 
-/* The whole step for one sample.  hidden may be NULL in FIXED mode.
+/* Alg. 1 from the scores on (stages 1-4 and the selection): takes the attention scores a
+ * [n_2d + n_3d] and the feature norms l1 (NULL: the S1 pair stays 0.5 / 0.5) as they come out of
+ * oracle_salience / oracle_l1norm, advances the state, decides, and writes the kept positions.
+ * ahat_out / z_out / diag may be NULL.  Returns the kept count. */
+int32_t oracle_decide_step(const double *a, const double *l1, const oracle_sample *s,
+                           const oracle_params *p, int32_t mode, oracle_state *st,
+                           int32_t *kept_idx, oracle_diag *diag, double *ahat_out, double *z_out);
+
+/* The whole step for one sample: oracle_salience (+ oracle_l1norm in ADAPTIVE mode), then
+ * oracle_decide_step.  hidden may be NULL in FIXED mode.
  * attn_out / l1_out / ahat_out / z_out may be NULL.  Returns kept count. */
 int32_t oracle_prune_step(const float *q, const float *k, const float *hidden,
                           int32_t n_heads, int32_t head_dim, int32_t d_model,

@@ -49,6 +49,14 @@ MUTATIONS = {
     "text tokens dropped": ("for (int32_t i = 0; i < s->n_txt; ++i) kept_idx[n++] = s->off_txt + i;", ""),
     "compaction ignores the sample offset": ("(const char *)src + ((int64_t)seq_off + kept_idx[r]) * row_bytes",
                                              "(const char *)src + ((int64_t)kept_idx[r]) * row_bytes"),
+    "ranks on the scores of the step alone": ("oracle_normalise(st->ahat, n2, n3, z);", "oracle_normalise(a, n2, n3, z);"),
+    "gates on the indicators of the step alone": ("oracle_gates(st->mhat, p, &dg.c_s1,", "oracle_gates(x, p, &dg.c_s1,"),
+    "budget from the attention share of the step alone": ("oracle_budget_adaptive(s, p, st->mhat[3], dg.c_final,",
+                                                          "oracle_budget_adaptive(s, p, x[3], dg.c_final,"),
+    "whole step decides on zeroed scores": ("const int32_t n_kept = oracle_decide_step(a, l1, s, p, mode,",
+                                            "memset(a, 0, sizeof(double)); const int32_t n_kept = oracle_decide_step(a, l1, s, p, mode,"),
+    "whole step drops the norms": ("const int32_t n_kept = oracle_decide_step(a, l1, s, p, mode,",
+                                   "const int32_t n_kept = oracle_decide_step(a, NULL, s, p, mode,"),
     "cold start prunes": ("if (t == 1 && p->cold_start_full_keep) {", "if (0) {"),
     "state updated after the decision": ("const int32_t n_kept = oracle_select(z, s, k2, k3, kept_idx);",
                                          "const int32_t n_kept = oracle_select(attn_out ? attn_out : z, s, k2, k3, kept_idx);"),
@@ -82,6 +90,7 @@ PATCH_MUTATIONS = {
     "3D mask emits the 2D token": ("kept_idx[n] = s->off_3d + q; ++n; ++dg.k_3d;", "kept_idx[n] = s->off_2d + q; ++n; ++dg.k_3d;"),
     "baseline from the instantaneous shares": ("s3 += st->xhat[4 * q + 3];", "s3 += x[4 * q + 3];"),
     "clusters the 2D mass only": ("mass[q] = a[q] + a[P + q];", "mass[q] = a[q];"),
+    "patch rules on the shares of the step alone": ("const double *xh = st->xhat + 4 * q;", "const double *xh = x + 4 * q;"),
     "patch cold start prunes": ("if (cold) cf = ORACLE_SET_2D | ORACLE_SET_3D;", "if (0) cf = 0;"),
 }
 

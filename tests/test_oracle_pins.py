@@ -447,3 +447,89 @@ def test_cold_start_keeps_everything_then_prunes():
     r2 = oracle.run_workload_step(wl, 1, [st])[0]
     assert r2.t == 2 and len(r2.kept_idx) == s.n_txt + 20
     np.testing.assert_allclose(r2.ahat, 0.5 * (r1.attn + r2.attn), rtol=1e-14)
+
+
+# ---------------------------------------------------------------- Alg. 1 over several steps
+def multistep_worked():
+    out = {}
+    with open(os.path.join(GOLDEN, "alg1_multistep_worked.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            key, *vals = line.split()
+            out[key] = np.array([float(v) for v in vals])
+    return out
+
+
+def test_ranking_uses_the_predicted_scores_hand_worked():
+    # Alg. 1 stage 1 feeds the later stages: the kept tokens follow X^_t (Eq. 8, then Eq. 9), which here
+    # ranks the tokens the other way round from the step's own scores.
+    g = multistep_worked()
+    s = S(1, 2, 2, keep_2d=0.5, keep_3d=0.5)
+    p = oracle.c_params(window_k=3, beta=0.85, cold_start_full_keep=0)
+    st = oracle.State(4)
+    r1 = oracle.decide_step(g["R_a1"], None, s, p, oracle.MODE_FIXED, st)
+    assert r1.kept_idx.tolist() == g["R_kept1"].astype(int).tolist() and (r1.k_2d, r1.k_3d, r1.t) == (1, 1, 1)
+    r2 = oracle.decide_step(g["R_a2"], None, s, p, oracle.MODE_FIXED, st)
+    np.testing.assert_allclose(r2.ahat, g["R_ahat2"], rtol=1e-14)
+    np.testing.assert_allclose(r2.z, g["R_z2"], rtol=1e-14)
+    assert r2.kept_idx.tolist() == g["R_kept2"].astype(int).tolist()
+    assert np.argmax(g["R_a2"][:2]) == 1 and np.argmax(g["R_a2"][2:]) == 1      # the step alone says rows 1, 3
+    r3 = oracle.decide_step(g["R_a3"], None, s, p, oracle.MODE_FIXED, st)
+    np.testing.assert_allclose(r3.ahat, g["R_ahat3_ema"], rtol=1e-14)
+    assert r3.kept_idx.tolist() == g["R_kept3"].astype(int).tolist() and r3.t == 3
+
+
+def _case_g(g):
+    j = np.arange(10)
+    a1 = np.concatenate([(j + 1) * (1 - g["G_share1"][0]) / 55, (10 - j) * g["G_share1"][0] / 55])
+    a2 = np.concatenate([(10 - j) * (1 - g["G_share2"][0]) / 55, (j + 1) * g["G_share2"][0] / 55])
+    n1 = np.repeat(g["G_norm1"], 10)
+    n2 = np.repeat(g["G_norm2"], 10)
+    return a1, a2, n1, n2
+
+
+def test_gates_and_budget_use_the_predicted_indicators_hand_worked():
+    # Sec. 4.1 / 4.2 / 4.4 and the budget split act on M^ (Alg. 1 stages 2-4), with the defaults of Sec. 5.4
+    g = multistep_worked()
+    a1, a2, n1, n2 = _case_g(g)
+    s = S(1, 10, 10, keep_total=0.5)
+    p = oracle.c_params(cold_start_full_keep=0)
+    st = oracle.State(20)
+    r1 = oracle.decide_step(a1, n1, s, p, oracle.MODE_ADAPTIVE, st)
+    assert [r1.c_s1, r1.c_s2, r1.c_final] == g["G_sets1"].astype(int).tolist()
+    assert [r1.k_2d, r1.k_3d] == g["G_k1"].astype(int).tolist()
+    assert r1.kept_idx.tolist() == g["G_kept1"].astype(int).tolist()
+    r2 = oracle.decide_step(a2, n2, s, p, oracle.MODE_ADAPTIVE, st)
+    np.testing.assert_allclose(r2.mhat, g["G_mhat2"], rtol=1e-12)
+    np.testing.assert_allclose(r2.x, [0.7, 0.3, 0.38, 0.62], rtol=1e-12)          # the step's own indicators
+    assert [r2.c_s1, r2.c_s2, r2.c_final] == g["G_sets2"].astype(int).tolist()
+    assert [r2.k_2d, r2.k_3d] == g["G_k2"].astype(int).tolist()
+    assert r2.kept_idx.tolist() == g["G_kept2"].astype(int).tolist()
+    assert not r2.near_gate and not r2.near_half
+
+
+def test_whole_step_feeds_scores_and_norms_into_the_decisions():
+    # The same two steps through oracle_prune_step.  One head, one query q = (sqrt(d), 0, ...): the logit of
+    # key j is its first component, so keys (ln a_j, 0, ...) make the softmax return a_j itself; a constant
+    # hidden row c has the L1 norm D |c|.
+    g = multistep_worked()
+    d = D = 4
+    s = S(1, 10, 10, keep_total=0.5)
+    p = oracle.c_params(cold_start_full_keep=0)
+    st = oracle.State(20)
+    for a, nrm, kept, ks in zip(_case_g(g)[:2], _case_g(g)[2:], ("G_kept1", "G_kept2"), ("G_k1", "G_k2")):
+        q = np.zeros((21, 1, d), np.float32)
+        k = np.zeros((21, 1, d), np.float32)
+        q[20, 0, 0] = 2.0
+        k[:20, 0, 0] = np.log(a)
+        k[:20, 0, 1:] = 7.0                                   # orthogonal to q: must not matter
+        hidden = np.zeros((21, D), np.float32)
+        hidden[:20] = (nrm / D)[:, None] * np.array([1, -1, 1, -1])
+        r = oracle.prune_step(q, k, hidden, 1, d, D, s, p, oracle.MODE_ADAPTIVE, st)
+        np.testing.assert_allclose(r.attn, a, rtol=1e-6)
+        np.testing.assert_allclose(r.l1, nrm, rtol=1e-6)
+        assert [r.k_2d, r.k_3d] == g[ks].astype(int).tolist()
+        assert r.kept_idx.tolist() == g[kept].astype(int).tolist()
+    np.testing.assert_allclose(st.c.mhat[:], g["G_mhat2"], rtol=1e-6)

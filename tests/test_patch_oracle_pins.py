@@ -276,3 +276,26 @@ def test_patch_step_is_the_composition_of_its_parts():
     np.testing.assert_allclose(r.x, x, rtol=1e-15)
     r2 = oracle.patch_select(r.attn, x, u, s, p, oracle.PatchState(9))
     assert np.array_equal(r.kept_idx, r2.kept_idx) and np.array_equal(r.cand, r2.cand)
+
+
+def test_patch_rules_use_the_predicted_indicators_hand_worked():
+    # Alg. 1 stages 2-4 read X^_t (Eq. 8 at t = 2, Eq. 9 at t = 3 = k); every named patch is built so
+    # that its predicted share and the step's own share fall on opposite sides of a threshold.
+    g = {}
+    with open(os.path.join(GOLDEN, "alg1_multistep_worked.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                key, *vals = line.split()
+                g[key] = np.array([float(v) for v in vals])
+    s, a, _, u = _small_case()
+    p = oracle.c_patch_params(window_k=3, beta=0.85, cold_start_full_keep=0)
+    st = oracle.PatchState(4)
+    for t in (1, 2, 3):
+        r = oracle.patch_select(a, g[f"P_x{t}"].reshape(4, 4), u, s, p, st)
+        assert r.t == t and r.labels.tolist() == [0, 0, 1, 2]
+        assert r.cand.reshape(-1).tolist() == g[f"P_cand{t}"].astype(int).tolist(), t
+        assert r.kept_idx.tolist() == g[f"P_kept{t}"].astype(int).tolist(), t
+        if t > 1:
+            assert [r.mu_2d, r.mu_3d] == pytest.approx(g[f"P_mu{t}"].tolist(), rel=1e-13)
+    np.testing.assert_allclose(st.xhat[1], g["P_xhat3_p1"], rtol=1e-13)
