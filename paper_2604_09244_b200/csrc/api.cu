@@ -12,7 +12,13 @@
 
 using namespace mvla;
 
-namespace { constexpr int kSets = 6; }   // scratch sets = prune steps that may be in flight at once
+namespace {
+constexpr int kSets = 6;            // scratch sets = prune steps that may be in flight at once
+#ifndef MVLA_TAIL_CTAS_PER_SM
+#define MVLA_TAIL_CTAS_PER_SM 2
+#endif
+constexpr int kTailCtasPerSm = MVLA_TAIL_CTAS_PER_SM;   // grid of the selection + row copy kernel
+}
 
 struct mvla_ctx {
     mvla_config cfg;
@@ -26,11 +32,14 @@ struct mvla_ctx {
     float* part;                 // [H][max_batch * max_vis] per-head partial scores
     int64_t part_stride;
     float* l1_ws;                // [kSets][max_batch * max_vis] feature norms, one set per step in flight
-    float* ahat_state;           // [n_prune_points][n_slots][max_vis]
-    float* mhat_state;           // [n_prune_points][n_slots][4]
+    float* ahat_state;           // [n_prune_points][n_slots][2][max_vis]: the copy step t reads and the one it writes
+    float* mhat_state;           // [n_prune_points][n_slots][2][4]
     unsigned long long* acc64;   // [kSets][max_batch * max_vis] fixed-point score accumulators, zero between
                                  // calls; the sets rotate from step to step (a step's scoring may run beside
                                  // the selections of the steps before it)
+    int32_t* tail_list;          // [kSets][max_batch * (max_text + max_vis)] kept list as the copying CTAs read it (-1 between launches)
+    size_t rows_all;             // max_batch * (max_text + max_vis)
+    int sm_count;                // multiprocessors of the device
     size_t vis_all;              // max_batch * max_vis
     // patch-by-patch path (cfg.patch_path): attention copy [H][max_text][vis_all], per-patch smoothed
     // indicators [n_prune_points][n_slots][max_patch][4], and the scratch between its kernels
@@ -160,8 +169,12 @@ int32_t make_plan(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_
             const int t_prev = (flags & MVLA_FLAG_RESET_STATE) ? 0 : ctx->t_host[sidx];
             const int t = t_prev + 1;
             d.t = t;
-            d.state_off = sidx * ctx->max_vis;
-            d.mstate_off = sidx;
+            // two copies of every state: step t reads the one step t - 1 wrote, writes the other
+            d.state_off = (sidx * 2 + (t_prev & 1)) * ctx->max_vis;
+            d.state_off_w = (sidx * 2 + (t & 1)) * ctx->max_vis;
+            d.mstate_off = sidx * 2 + (t_prev & 1);
+            d.mstate_off_w = sidx * 2 + (t & 1);
+            d.slot_index = sidx;
             d.update_state = (flags & MVLA_FLAG_NO_STATE_UPDATE) ? 0 : 1;
             if (t <= 1) { d.c_prev = 0.f; d.c_new = 1.f; }                                   // X^_1 = X_1
             else if (t < c.window_k) {                                                        // Eq. 8
@@ -257,7 +270,8 @@ int32_t check_sticky(mvla_ctx* ctx)
 // fixed-point accumulators ctx->acc64 (*used_acc64 = true).
 int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, const void* k, int64_t rows,
                            const void* hidden, float* l1, unsigned long long* acc64, bool* used_acc64,
-                           bool free_running, cudaStream_t st, AlphaOut alpha = AlphaOut{nullptr, 0, 0})
+                           bool free_running, cudaStream_t st, AlphaOut alpha = AlphaOut{nullptr, 0, 0},
+                           int32_t* rearm = nullptr)
 {
     if (used_acc64) *used_acc64 = false;
     const mvla_config& c = ctx->cfg;
@@ -286,7 +300,7 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
         e = launch_salience_fast(bd, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, static_cast<int>(ctx->qk_elem), tq, tk,
                                  tiles_per_cta, cluster, npad,
                                  alpha.ptr && !acc64 ? nullptr : ctx->part,     // the patch path reads the attention copy only
-                                 ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, st);
+                                 ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, rearm, st);
         if (used_acc64) *used_acc64 = acc64 != nullptr;
     } else {
         e = launch_salience(bd, c.dtype, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, q, k, tq, tk, ctx->use_umma, tiles_per_cta,
@@ -633,6 +647,8 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (c.salience_path == MVLA_SALIENCE_FMA) ctx->use_umma = false;
     ctx->part = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
     ctx->acc64 = nullptr;
+    ctx->tail_list = nullptr;
+    ctx->sm_count = prop.multiProcessorCount;
     ctx->alpha_ws = ctx->xhat_patch = ctx->patch_x_ws = ctx->patch_attn_ws = nullptr;
     ctx->patch_sets = 1;
     ctx->nout_ws = nullptr;
@@ -666,10 +682,13 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     alloc(&ctx->l1_ws, kSets * vis_all);
     ctx->vis_all = vis_all;
     ctx->step_parity = 0;
-    alloc(&ctx->ahat_state, n_state * ctx->max_vis);
-    alloc(&ctx->mhat_state, n_state * 4);
+    alloc(&ctx->ahat_state, 2 * n_state * ctx->max_vis);
+    alloc(&ctx->mhat_state, 2 * n_state * 4);
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->acc64), kSets * vis_all * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(ctx->acc64, 0, kSets * vis_all * sizeof(unsigned long long));
+    ctx->rows_all = static_cast<size_t>(c.max_batch) * (c.max_text + ctx->max_vis);
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->tail_list), kSets * ctx->rows_all * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->tail_list, 0xFF, kSets * ctx->rows_all * sizeof(int32_t));
     if (c.patch_path) {
         const size_t alpha_n = static_cast<size_t>(c.n_heads) * c.max_text * vis_all;
         ctx->patch_sets = alpha_n * sizeof(float) * kSets <= (size_t(1) << 30) ? kSets : 1;   // at most 1 GiB of attention copies
@@ -719,6 +738,7 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     cudaFree(ctx->ahat_state);
     cudaFree(ctx->mhat_state);
     cudaFree(ctx->acc64);
+    cudaFree(ctx->tail_list);
     cudaFree(ctx->alpha_ws);
     cudaFree(ctx->xhat_patch);
     cudaFree(ctx->patch_x_ws);
@@ -950,8 +970,11 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         const int n = std::min(kMaxChunk, batch - first);
         const BatchDesc bd = chunk_of(plan, first, n);
         bool used_acc64 = false;
+        // the fused selection + copy kernel (below) wants its list words re-armed by the scoring kernel
+        const bool tail = !forked && select_copy_supported(bd);
         rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, l1_ws, acc64,
-                                &used_acc64, false, forked ? ctx->aux[par] : st);
+                                &used_acc64, false, forked ? ctx->aux[par] : st, AlphaOut{nullptr, 0, 0},
+                                tail ? ctx->tail_list + par * ctx->rows_all : nullptr);
         if (rc != MVLA_OK) return rc;
         cudaStream_t sel_stream = st;
         if (forked) {
@@ -970,6 +993,17 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         io.attn_out = out->attn; io.ahat_out = out->ahat; io.z_out = out->z; io.diag = out->diag;
         io.chunk_first = first; io.total_out = plan.total_out; io.write_total = first + n == batch;
         io.n_in_launch = n;
+        if (!forked && used_acc64 && select_copy_supported(bd)) {
+            // one kernel for selection and row copy: every CTA repeats its sample's selection, then copies
+            ctx->sel_valid[par] = false;             // this set was used outside the event chain
+            const bool copying = (job.src[0] && job.dst[0]) || (job.src[1] && job.dst[1]) || (job.src[2] && job.dst[2]);
+            (void)copying;
+            const cudaError_t e2 = launch_select_copy(bd, gp, io, job, ctx->tail_list + par * ctx->rows_all,
+                                                      ctx->status_dev,
+                                                      ctx->sm_count * kTailCtasPerSm - n, st);
+            if (e2 != cudaSuccess) return fail_cuda(ctx, e2);
+            continue;
+        }
         cudaError_t e = launch_select(bd, gp, io, sel_stream);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
         if (forked) {                                // join: the row copy, and whatever the caller enqueues next

@@ -26,8 +26,13 @@ struct SampleDev {
     int32_t budget;         // kept visual tokens (host known)
     int32_t k_2d_fixed;     // >= 0: host-decided split (FIXED mode or cold start); -1: split on device
     int32_t kmin_2d, kmin_3d;   // ADAPTIVE floors
-    int32_t state_off;      // offset of this (prune point, slot) in the per-token state array
-    int32_t mstate_off;     // index of this (prune point, slot) in the indicator state array (x4 floats)
+    // The smoothed state of a (prune point, slot) is kept twice: step t reads the copy that step t - 1
+    // wrote and writes the other one, so that several CTAs may read the previous state while one writes.
+    int32_t state_off;      // per-token state array: offset of the copy this step READS
+    int32_t state_off_w;    // ... and of the copy it WRITES
+    int32_t mstate_off;     // indicator state array (x4 floats): index of the copy this step reads
+    int32_t mstate_off_w;   // ... and writes
+    int32_t slot_index;     // prune point * slots + slot: addresses the per-patch state (updated in place by one CTA)
     int32_t t;              // 1-based action step this call is
     int32_t update_state;   // 0: dry run
     float c_prev, c_new;    // state update weights: xhat = c_prev * xhat + c_new * x
@@ -86,6 +91,8 @@ inline cudaLaunchAttribute pdl_attribute()
 // `part` is null too: only the attention copy is wanted).
 // `free_running`: the kernel does not wait for the kernel before it in its stream (the caller orders
 // everything it depends on with events).
+// `rearm`: when not null, words [out_off, out_off + n_out) of every sample are set to -1 (the kept list that
+// launch_select_copy's CTAs exchange, see there).
 // Optional copy of the attention itself for the patch-by-patch path:
 // ptr[(h * stride_h) + (i * stride_i) + vis_off + j] = alpha[h, i, j]   (null: not written).
 struct AlphaOut {
@@ -100,7 +107,7 @@ bool fast_salience_supported(int tiles_per_cta);
 cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
-                                 bool free_running, AlphaOut alpha, cudaStream_t stream);
+                                 bool free_running, AlphaOut alpha, int32_t* rearm, cudaStream_t stream);
 
 
 // Salience: per-head partial scores part[h][vis] (already scaled by 1/(H n_t)).
@@ -128,12 +135,48 @@ struct CompactJob {
     void* dst[3];
     int32_t row_bytes[3];
 };
+// The same as the kernels see it: rows cut into 2 KB segments (one warp moves one segment).
+constexpr int kSegBytes = 2048;     // 32 lanes x 4 x 16 B
+struct CompactArgs {
+    const uint8_t* src[3];
+    uint8_t* dst[3];
+    int32_t row_bytes[3];
+    int32_t segs[3];          // 2 KB segments per row
+    int32_t seg_begin[4];     // prefix sums of segs per row over the (up to) three tensors
+};
+inline CompactArgs compact_args(const CompactJob& job)
+{
+    CompactArgs a;
+    int total = 0;
+    for (int i = 0; i < 3; ++i) {
+        const bool on = job.src[i] && job.dst[i];
+        a.src[i] = static_cast<const uint8_t*>(job.src[i]);
+        a.dst[i] = static_cast<uint8_t*>(job.dst[i]);
+        a.row_bytes[i] = job.row_bytes[i];
+        a.segs[i] = on ? (job.row_bytes[i] + kSegBytes - 1) / kSegBytes : 0;
+        a.seg_begin[i] = total;
+        total += a.segs[i];
+    }
+    a.seg_begin[3] = total;
+    return a;
+}
 // Rows [chunk_row0, chunk_row0 + chunk_rows) of the output.  With `out_offsets` (device) the owning
 // sample of a row is looked up there over the whole batch and rows of samples outside this launch's
 // descriptors are skipped; without it the descriptors' host-computed out_off is used.
 cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int32_t* kept_idx,
                            int32_t chunk_rows, int32_t chunk_row0, const int32_t* out_offsets,
                            int32_t chunk_first, int32_t batch_total, cudaStream_t stream);
+
+// Tail of the fused step for samples of up to 2048 visual tokens: carry-over + budget + top-k (as in
+// launch_select) AND the row copy in one kernel.  One CTA per sample selects; the other CTAs copy the
+// text rows at once, then take the kept rows word by word from `list` as the selecting CTA writes them
+// (bounded waits, MVLA_ERR_TIMEOUT into `status` when one runs out): no kernel boundary, fence or flag lies
+// between selection and copy.  `list`: one int per output row of the batch, all -1 when the kernel starts
+// (the scoring kernel before it re-arms them, see launch_salience_fast).
+// `ctas`: copying CTAs to aim for (every sample gets at least one).
+bool select_copy_supported(const BatchDesc& bd);
+cudaError_t launch_select_copy(const BatchDesc& bd, const GateParams& gp, const SelectIO& io, const CompactJob& job,
+                               int32_t* list, int* status, int ctas, cudaStream_t stream);
 
 // ---- patch-by-patch path (Alg. 1 taken literally) ----
 struct PatchParams {

@@ -12,7 +12,6 @@ namespace mvla {
 namespace {
 
 constexpr int kWarpsPerBlock = 8;
-constexpr int kSegBytes = 2048;     // 32 lanes x 4 x 16 B
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p)
 {
@@ -25,14 +24,6 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v)
 {
     asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
-
-struct CompactArgs {
-    const uint8_t* src[3];
-    uint8_t* dst[3];
-    int32_t row_bytes[3];
-    int32_t segs[3];          // 2 KB segments per row
-    int32_t seg_begin[4];     // prefix sums of segs per row over the (up to) three tensors
-};
 
 // grid.x covers chunk_rows * segs_per_row_all warp-units.
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
@@ -96,18 +87,8 @@ cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int
                            int32_t chunk_rows, int32_t chunk_row0, const int32_t* out_offsets,
                            int32_t chunk_first, int32_t batch_total, cudaStream_t stream)
 {
-    CompactArgs a;
-    int total = 0;
-    for (int i = 0; i < 3; ++i) {
-        const bool on = job.src[i] && job.dst[i];
-        a.src[i] = static_cast<const uint8_t*>(job.src[i]);
-        a.dst[i] = static_cast<uint8_t*>(job.dst[i]);
-        a.row_bytes[i] = job.row_bytes[i];
-        a.segs[i] = on ? (job.row_bytes[i] + kSegBytes - 1) / kSegBytes : 0;
-        a.seg_begin[i] = total;
-        total += a.segs[i];
-    }
-    a.seg_begin[3] = total;
+    const CompactArgs a = compact_args(job);
+    const int total = a.seg_begin[3];
     if (total == 0 || chunk_rows <= 0) return cudaSuccess;
     const int64_t units = static_cast<int64_t>(chunk_rows) * total;
     int64_t blocks = (units + kWarpsPerBlock - 1) / kWarpsPerBlock;

@@ -48,9 +48,9 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         uint32_t ok;
         asm volatile("{\n\t.reg .pred p;\n\t"
-                     "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+                     "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
                      "selp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+                     : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
         if (ok) return true;
         if ((it & 63u) == 63u && global_ns() - t0 > 1000000000ull) break;
     }
@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(kFastThreads, 1)
 salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
                      const __grid_constant__ CUtensorMap tmap_k, int n_heads, int kv_group, int head_dim, int esize, int npad_max,
                      float* __restrict__ part, int64_t part_stride, unsigned long long* __restrict__ acc64,
-                     int* status, int free_running, const AlphaOut alpha)
+                     int* status, int free_running, const AlphaOut alpha, int32_t* __restrict__ rearm)
 {
     constexpr int CC = TCOL * NTILE;
     extern __shared__ uint8_t dyn_smem_raw[];
@@ -103,7 +103,6 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         any_live |= ti.valid > 0;
     }
 
-    pdl_trigger();
     if (tid == 0) {                           // the loads go out first; everything else overlaps with them
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);
@@ -141,6 +140,13 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = s_tmem;
+    // Thread 0 is past its wait for the kernel before this one, so whatever that kernel wrote is
+    // complete: the next kernel may become resident now and may read such data in its prologue.
+    pdl_trigger();
+    // One CTA per sample re-arms the words through which the kernel after this one hands the kept list from
+    // its selecting CTA to its copying CTAs (-1: not yet known).  Their last users finished long ago.
+    if (rearm && blockIdx.x == 0 && blockIdx.y == 0)
+        for (int i = tid; i < s.n_out; i += kFastThreads) rearm[s.out_off + i] = -1;
 
     if (tid == 0) {
         bool got = mbar_wait(bar_full, 0);
@@ -164,9 +170,14 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         }
         umma_commit(bar_mma);                 // arrives once every MMA issued above has finished
     }
-    __syncwarp();
-    bool ok = mbar_wait(bar_mma, 0);
-    if (!ok) *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
+    // Only thread 0 polls the barriers; the other threads park at the block barrier below (a hardware
+    // wait), so while a CTA waits for its predecessor, its loads or its MMAs it leaves the issue slots and
+    // the shared-memory pipe of the multiprocessor to the CTAs that share it.
+    bool ok = true;
+    if (tid == 0) {
+        ok = mbar_wait(bar_mma, 0);
+        if (!ok) *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
+    }
     ok = __syncthreads_and(ok) != 0;          // block-uniform from here on (aligned instructions follow)
     tc_fence_after();
 
@@ -243,9 +254,9 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         st_async_peer_f32x2(smem_u32(&s_peer[crank][i]), bar_x, r, s_loc[i]);
     }
     __syncwarp();
-    bool okx = mbar_wait_cluster(bar_x, 0);
-    if (!okx) *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
-    if (tid < npad) {
+    if (tid < npad) {                         // the warps that combine the pairs wait for them; the others park below
+        const bool okx = mbar_wait_cluster(bar_x, 0);
+        if (!okx) *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
         float gmax = -CUDART_INF_F;
         for (uint32_t r = 0; r < csize; ++r) gmax = fmaxf(gmax, s_peer[r][tid].x);
         float z = 0.f;
@@ -294,7 +305,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
 template <int TCOL, int NTILE>
 cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tq,
                           const CUtensorMap* tk, int cluster, int npad, float* part, int64_t part_stride,
-                          unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, cudaStream_t stream)
+                          unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, int32_t* rearm, cudaStream_t stream)
 {
     const size_t smem = 1024 + static_cast<size_t>((head_dim * esize + 127) / 128) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
     auto kern = salience_fast_kernel<TCOL, NTILE>;
@@ -313,7 +324,7 @@ cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int he
     attr[1] = pdl_attribute();
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, kv_group, head_dim, esize, npad, part, part_stride, acc64, status, free_running, alpha);
+    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, kv_group, head_dim, esize, npad, part, part_stride, acc64, status, free_running, alpha, rearm);
 }
 
 }  // namespace
@@ -323,13 +334,13 @@ bool fast_salience_supported(int tiles_per_cta) { return tiles_per_cta >= 1 && t
 cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
-                                 bool free_running, AlphaOut alpha, cudaStream_t stream)
+                                 bool free_running, AlphaOut alpha, int32_t* rearm, cudaStream_t stream)
 {
     const int tcol = npad <= 16 ? 16 : (npad <= 32 ? 32 : 64);
 #define MVLA_FAST(TC, NTL)                                                                                      \
     if (tcol == TC && tiles_per_cta == NTL)                                                                     \
         return launch_fast_t<TC, NTL>(bd, n_heads, kv_group, head_dim, esize, tmap_q, tmap_k, cluster, npad, part, part_stride, \
-                                      acc64, status, free_running ? 1 : 0, alpha, stream);
+                                      acc64, status, free_running ? 1 : 0, alpha, rearm, stream);
     MVLA_FAST(16, 1) MVLA_FAST(32, 1) MVLA_FAST(64, 1) MVLA_FAST(16, 2) MVLA_FAST(32, 2) MVLA_FAST(64, 2)
 #undef MVLA_FAST
     return cudaErrorInvalidConfiguration;

@@ -234,7 +234,7 @@ patch_select_kernel(const __grid_constant__ BatchDesc bd, const PatchParams pp, 
     const int pat_off = s.vis_off / 2;
     const bool carry = s.c_prev != 0.f;
     const bool cold = s.t == 1 && pp.cold_start_full_keep;
-    float4* state = reinterpret_cast<float4*>(io.xhat_state) + static_cast<int64_t>(s.mstate_off) * pp.max_patch;
+    float4* state = reinterpret_cast<float4*>(io.xhat_state) + static_cast<int64_t>(s.slot_index) * pp.max_patch;
     if (tid < 5) sm.cnt[tid] = 0;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");    // scores and indicators come from the kernel before this one

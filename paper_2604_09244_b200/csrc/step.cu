@@ -1,0 +1,212 @@
+// Tail of the fused prune step: carry-over, gates, budget split, top-k selection (Alg. 1 stages 1-4,
+// Eqs. 8-10) AND the compaction of the surviving rows (Sec. 4.4) in one kernel.
+//
+// A step on one sample is a chain of latencies, not a bandwidth problem: a kernel boundary costs a
+// microsecond or two, a device-wide fence about one.  Here one CTA per sample runs the selection and the
+// other CTAs of the grid copy rows:
+//   * while the scores are still being computed the copying CTAs move the text rows, whose output
+//     positions the host knows;
+//   * the selecting CTA writes every entry of the kept list as one 4-byte word into library scratch; a
+//     copying warp polls the word of the row it is to move (-1: not yet known) and starts the moment the
+//     word is there.  No fence, flag or barrier lies between the two roles: each word is its own signal;
+//   * what nobody waits for (smoothed state, indicators and diagnostics when the budgets came from the
+//     host, optional score outputs) is written after the list.
+// The scoring kernel that runs before this one re-arms the words, so nothing is left to do at the end.
+#include "common.cuh"
+#include "device_utils.cuh"
+#include "select_impl.cuh"
+
+#include <algorithm>
+
+namespace mvla {
+namespace {
+
+struct TailPlan {
+    int16_t cta0[kMaxChunk + 1];      // first CTA of every sample; cta0[n] = grid size
+};
+
+__device__ __forceinline__ uint4 ld_row(const uint4* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_row(uint4* p, const uint4& v)
+{
+    asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// Copies `n_rows` rows.  The work is cut into 2 KB segments of one row of one tensor; warp `w` of `nw`
+// takes segments w, w + nw, ... and keeps two of them (8 x 16 bytes per lane) in flight.
+// rows(i, src_row, dst_row): absolute source and destination row of the i-th row of the list; false: skip it.
+template <class RowFn>
+__device__ __forceinline__ void copy_rows(const CompactArgs& a, int n_rows, int w, int nw, int lane, RowFn rows)
+{
+    const int per_row = a.seg_begin[3];
+    const int n_units = n_rows * per_row;
+    for (int u0 = w; u0 < n_units; u0 += 2 * nw) {
+        uint4 v[2][4];
+        const uint4* sp[2];
+        uint4* dp[2];
+        int nvec[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int u = u0 + k * nw;
+            nvec[k] = 0;
+            sp[k] = nullptr;
+            dp[k] = nullptr;
+            if (u < n_units) {
+                const int r = u / per_row, g = u - r * per_row;
+                int64_t srow = 0, drow = 0;
+                if (!rows(r, srow, drow)) continue;
+                const int tsel = g >= a.seg_begin[2] ? 2 : (g >= a.seg_begin[1] ? 1 : 0);
+                const int seg = g - a.seg_begin[tsel];
+                const int rb = a.row_bytes[tsel];
+                sp[k] = reinterpret_cast<const uint4*>(a.src[tsel] + srow * rb + static_cast<int64_t>(seg) * kSegBytes);
+                dp[k] = reinterpret_cast<uint4*>(a.dst[tsel] + drow * rb + static_cast<int64_t>(seg) * kSegBytes);
+                nvec[k] = min(kSegBytes, rb - seg * kSegBytes) >> 4;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 2; ++k)
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (lane + i * 32 < nvec[k]) v[k][i] = ld_row(sp[k] + lane + i * 32);
+#pragma unroll
+        for (int k = 0; k < 2; ++k)
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (lane + i * 32 < nvec[k]) st_row(dp[k] + lane + i * 32, v[k][i]);
+    }
+}
+
+// One word of the kept list as the copiers see it: a 4-byte store is indivisible, so a copier that reads a
+// value >= 0 has the row it needs, with no fence, flag or barrier between the CTA that selects and the
+// CTAs that copy.  The words are -1 between launches.
+__device__ __forceinline__ int ld_relaxed_gpu(const int* p)
+{
+    int v;
+    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// grid: CTAs 0 .. n-1 select (CTA b for sample b of the launch), the CTAs after them copy; tp.cta0[b] is the
+// first copying CTA of sample b.  `list`: the kept list in library scratch (one word per output row of the
+// launch's samples, -1 = not yet known; the scoring kernel before this one has set them all to -1).
+// A selecting CTA always has a lower index than any copying CTA, so it is dispatched before them: a
+// copier that runs can count on its selector running too.  Its waits are bounded all the same.
+template <int NT, int CAP>
+__global__ void __launch_bounds__(NT)
+select_copy_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ TailPlan tp, const GateParams gp,
+                   const SelectIO io, const __grid_constant__ CompactArgs ca, int32_t* __restrict__ list, int* status)
+{
+    const int tid = threadIdx.x, lane = tid & 31;
+    if (static_cast<int>(blockIdx.x) < bd.n) {
+        // ---- selection of one sample, by one CTA
+        __shared__ SelectSmem<NT, CAP> sm;
+        const int b = blockIdx.x;
+        SelectRole role;
+        role.late_pdl = true;
+        if (tp.cta0[bd.n] > 0) role.kept_sm = list + bd.s[b].out_off;   // every word is its own "ready" signal
+        select_sample<NT, CAP>(bd.s[b], b, gp, io, sm, role);
+        return;
+    }
+    // ---- row copy
+    const int c = static_cast<int>(blockIdx.x) - bd.n;
+    int b = 0;
+    while (b + 1 < bd.n && c >= tp.cta0[b + 1]) ++b;
+    const int part = c - tp.cta0[b], nparts = tp.cta0[b + 1] - tp.cta0[b];
+    const SampleDev& s = bd.s[b];
+    const int w = part * (NT / 32) + (tid >> 5), nw = nparts * (NT / 32);
+
+    // Output position of the text rows: known on the host when the split is (FIXED budgets, cold start),
+    // or when the text segment lies before or behind both visual segments (then only the total counts).
+    const bool b2 = s.n_2d > 0 && s.off_2d < s.off_txt, b3 = s.n_3d > 0 && s.off_3d < s.off_txt;
+    int baset = -1;
+    if (s.k_2d_fixed >= 0) baset = (b2 ? s.k_2d_fixed : 0) + (b3 ? s.budget - s.k_2d_fixed : 0);
+    else if (b2 == b3) baset = b2 ? s.budget : 0;
+    const bool text_early = baset >= 0;
+    if (text_early)                                         // while the scores are still being computed
+        copy_rows(ca, s.n_txt, w, nw, lane, [&](int i, int64_t& srow, int64_t& drow) {
+            srow = static_cast<int64_t>(s.seq_off) + s.off_txt + i;
+            drow = static_cast<int64_t>(s.out_off) + baset + i;
+            return true;
+        });
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // keeps the chain of dependencies whole: the kernel after
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // this one may rely on the one before it being complete
+
+    {
+        const int n_rows = s.n_out - (text_early ? s.n_txt : 0);
+        const int32_t* kept = list + s.out_off;
+        const uint64_t t0 = global_ns();
+        copy_rows(ca, n_rows, w, nw, lane, [&](int i, int64_t& srow, int64_t& drow) {
+            const int r = (text_early && i >= baset) ? i + s.n_txt : i;       // skip the text rows copied before
+            int v = ld_relaxed_gpu(kept + r);               // the whole warp reads one word: one request
+            for (uint32_t it = 0; v < 0 && it < kSpinLimit; ++it) {
+                __nanosleep(20);
+                v = ld_relaxed_gpu(kept + r);
+                if ((it & 63u) == 63u && global_ns() - t0 > 1000000000ull) break;
+            }
+            if (v < 0) {                                    // gave up: report, leave the row alone
+                *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
+                return false;
+            }
+            srow = static_cast<int64_t>(s.seq_off) + v;
+            drow = static_cast<int64_t>(s.out_off) + r;
+            return true;
+        });
+    }
+}
+
+template <int NT, int CAP>
+cudaError_t launch_t(const BatchDesc& bd, const TailPlan& tp, const GateParams& gp, const SelectIO& io, const CompactArgs& ca,
+                     int32_t* list, int* status, cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(bd.n + tp.cta0[bd.n]));
+    cfg.blockDim = dim3(NT);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1] = {pdl_attribute()};
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, select_copy_kernel<NT, CAP>, bd, tp, gp, io, ca, list, status);
+}
+
+int max_vis_of(const BatchDesc& bd)
+{
+    int m = 0;
+    for (int b = 0; b < bd.n; ++b) m = std::max(m, bd.s[b].n_2d + bd.s[b].n_3d);
+    return m;
+}
+
+}  // namespace
+
+bool select_copy_supported(const BatchDesc& bd) { return max_vis_of(bd) <= 2048; }
+
+cudaError_t launch_select_copy(const BatchDesc& bd, const GateParams& gp, const SelectIO& io, const CompactJob& job,
+                               int32_t* list, int* status, int ctas, cudaStream_t stream)
+{
+    if (bd.n < 1 || !select_copy_supported(bd)) return cudaErrorInvalidConfiguration;
+    const CompactArgs ca = compact_args(job);
+    TailPlan tp;
+    int next = 0;
+    if (ca.seg_begin[3] > 0) {
+        // copying CTAs per sample in proportion to its kept rows, at least one each
+        ctas = std::min(std::max(ctas, bd.n), 30000);
+        int64_t rows = 0;
+        for (int b = 0; b < bd.n; ++b) rows += bd.s[b].n_out;
+        for (int b = 0; b < bd.n; ++b) {
+            tp.cta0[b] = static_cast<int16_t>(next);
+            const int64_t share = rows > 0 ? (static_cast<int64_t>(ctas) * bd.s[b].n_out + rows / 2) / rows : 1;
+            next += static_cast<int>(std::max<int64_t>(1, share));
+        }
+    } else {
+        for (int b = 0; b < bd.n; ++b) tp.cta0[b] = 0;       // nothing to copy: selection only
+    }
+    for (int b = bd.n; b <= kMaxChunk; ++b) tp.cta0[b] = static_cast<int16_t>(next);
+    if (max_vis_of(bd) <= 1024) return launch_t<512, 1024>(bd, tp, gp, io, ca, list, status, stream);
+    return launch_t<512, 2048>(bd, tp, gp, io, ca, list, status, stream);
+}
+
+}  // namespace mvla
