@@ -32,6 +32,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
            "-o", LIB] + [os.path.join(CSRC, f) for f in SOURCES] + ["-lcudart"]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
+    cmd += os.environ.get("MVLA_NVCC_FLAGS", "").split()       # extra compiler flags, e.g. -D tuning macros
     subprocess.run(cmd, check=True)
     return LIB
 

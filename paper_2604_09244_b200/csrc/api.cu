@@ -271,7 +271,7 @@ int32_t check_sticky(mvla_ctx* ctx)
 int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, const void* k, int64_t rows,
                            const void* hidden, float* l1, unsigned long long* acc64, bool* used_acc64,
                            bool free_running, cudaStream_t st, AlphaOut alpha = AlphaOut{nullptr, 0, 0},
-                           int32_t* rearm = nullptr)
+                           int32_t* rearm = nullptr, bool norms_beside = false)
 {
     if (used_acc64) *used_acc64 = false;
     const mvla_config& c = ctx->cfg;
@@ -292,8 +292,11 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
     }
     cudaError_t e;
     const bool fast = ctx->use_umma && fast_salience_supported(tiles_per_cta);
-    if (hidden && l1) {
-        e = launch_l1norm(bd, ctx->hidden_dtype, c.d_model, hidden, l1, st);
+    // The norms do not depend on the scores: with `norms_beside` (fast kernel only) they are launched AFTER
+    // the scoring kernel and run beside it instead of in front of it.
+    norms_beside = norms_beside && fast;
+    if (hidden && l1 && !norms_beside) {
+        e = launch_l1norm(bd, ctx->hidden_dtype, c.d_model, hidden, l1, false, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
     if (fast) {
@@ -308,6 +311,10 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
     }
     if (e == cudaErrorInvalidConfiguration) return MVLA_ERR_UNSUPPORTED;
     if (e != cudaSuccess) return fail_cuda(ctx, e);
+    if (hidden && l1 && norms_beside) {
+        e = launch_l1norm(bd, ctx->hidden_dtype, c.d_model, hidden, l1, true, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+    }
     return MVLA_OK;
 }
 
@@ -974,7 +981,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         const bool tail = !forked && select_copy_supported(bd);
         rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, l1_ws, acc64,
                                 &used_acc64, false, forked ? ctx->aux[par] : st, AlphaOut{nullptr, 0, 0},
-                                tail ? ctx->tail_list + par * ctx->rows_all : nullptr);
+                                tail ? ctx->tail_list + par * ctx->rows_all : nullptr, tail);
         if (rc != MVLA_OK) return rc;
         cudaStream_t sel_stream = st;
         if (forked) {

@@ -122,9 +122,11 @@ cudaError_t launch_salience(const BatchDesc& bd, int dtype, int n_heads, int kv_
 cudaError_t launch_head_reduce(const float* part, int64_t part_stride, int n_heads, int total_vis,
                                float* attn, cudaStream_t stream);
 
-// L1 feature norms of the visual rows.
+// L1 feature norms of the visual rows.  `beside_predecessor`: the kernel is launched right after a scoring
+// kernel that releases its dependents only once ITS predecessor is complete (launch_salience_fast): it then
+// runs beside the scoring kernel and completes after it.
 cudaError_t launch_l1norm(const BatchDesc& bd, int dtype, int d_model, const void* hidden,
-                          float* l1, cudaStream_t stream);
+                          float* l1, bool beside_predecessor, cudaStream_t stream);
 
 // Carry-over + budget + top-k + emission; one CTA per sample (io.n_in_launch = bd.n).
 cudaError_t launch_select(const BatchDesc& bd, const GateParams& gp, const SelectIO& io, cudaStream_t stream);

@@ -48,9 +48,9 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         uint32_t ok;
         asm volatile("{\n\t.reg .pred p;\n\t"
-                     "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+                     "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
                      "selp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
         if (ok) return true;
         if ((it & 63u) == 63u && global_ns() - t0 > 1000000000ull) break;
     }

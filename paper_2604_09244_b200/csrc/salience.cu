@@ -292,15 +292,25 @@ __global__ void head_reduce_kernel(const float* __restrict__ part, int64_t part_
 }
 
 // One warp per visual row; 16-byte loads; fixed reduction order.
+// Launched with programmatic serialization: the kernel after it may become resident at once, and this
+// kernel itself needs nothing from the kernel before it except that the hidden rows are final, which the
+// launch order guarantees (see the callers).  It therefore does its work first and waits for its
+// predecessor LAST, only so that "this kernel is complete" keeps implying "its predecessor is complete"
+// for whatever follows.
 template <typename T>
 __global__ void __launch_bounds__(256)
 l1norm_kernel(const __grid_constant__ BatchDesc bd, int d_model, const T* __restrict__ hidden,
-              float* __restrict__ l1)
+              float* __restrict__ l1, int early)
 {
+    if (early) pdl_trigger();
+    else pdl_wait();
     const SampleDev& s = bd.s[blockIdx.y];
     const int nv = s.n_2d + s.n_3d;
     const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (j >= nv) return;
+    if (j >= nv) {
+        if (early) pdl_wait();
+        return;
+    }
     const int lane = threadIdx.x & 31;
     const int row = s.seq_off + (j < s.n_2d ? s.off_2d + j : s.off_3d + (j - s.n_2d));
     constexpr int kVec = 16 / sizeof(T);
@@ -324,6 +334,7 @@ l1norm_kernel(const __grid_constant__ BatchDesc bd, int d_model, const T* __rest
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
     if (lane == 0) l1[s.vis_off + j] = acc;
+    if (early) pdl_wait();
 }
 
 template <typename T, bool UMMA>
@@ -398,17 +409,22 @@ cudaError_t launch_head_reduce(const float* part, int64_t part_stride, int n_hea
 }
 
 cudaError_t launch_l1norm(const BatchDesc& bd, int dtype, int d_model, const void* hidden, float* l1,
-                          cudaStream_t stream)
+                          bool beside_predecessor, cudaStream_t stream)
 {
     int max_nv = 0;
     for (int b = 0; b < bd.n; ++b) max_nv = max(max_nv, bd.s[b].n_2d + bd.s[b].n_3d);
     if (max_nv == 0) return cudaSuccess;
-    const dim3 grid((max_nv + 7) / 8, bd.n);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((max_nv + 7) / 8, bd.n);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1] = {pdl_attribute()};
+    cfg.attrs = attr;
+    cfg.numAttrs = beside_predecessor ? 1 : 0;
+    const int early = beside_predecessor ? 1 : 0;
     if (dtype == MVLA_DTYPE_BF16)
-        l1norm_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(bd, d_model, static_cast<const __nv_bfloat16*>(hidden), l1);
-    else
-        l1norm_kernel<float><<<grid, 256, 0, stream>>>(bd, d_model, static_cast<const float*>(hidden), l1);
-    return cudaGetLastError();
+        return cudaLaunchKernelEx(&cfg, l1norm_kernel<__nv_bfloat16>, bd, d_model, static_cast<const __nv_bfloat16*>(hidden), l1, early);
+    return cudaLaunchKernelEx(&cfg, l1norm_kernel<float>, bd, d_model, static_cast<const float*>(hidden), l1, early);
 }
 
 }  // namespace mvla

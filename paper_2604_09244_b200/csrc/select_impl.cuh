@@ -56,6 +56,7 @@ struct SelectSmem {
     alignas(16) uint32_t ext[NT / 32][4];    // per-warp smallest / largest key: min 2D, max 2D, min 3D, max 3D
     alignas(16) uint32_t cand_key[2][kCandMax];
     alignas(16) int cand_idx[2][kCandMax];
+    int cand_rank[2][kCandMax];              // rank of every listed key among the listed keys of its modality
     alignas(16) int ctl[8];                  // mode 2D, 3D; threshold bin 2D, 3D; keys to take from it 2D, 3D; budgets 2D, 3D
     int wtot[CAP / NT][NT / 32];             // emission: kept tokens (low half) and index-ranked ties (high half) per slice and warp
     int ncand[2];
@@ -141,11 +142,13 @@ __device__ __forceinline__ int block_exscan(int x, int* warp_tot, int* total)
 //              previous state and of the norms follow griddepcontrol.wait; true: those loads come first
 //              (the caller guarantees that they were written before this kernel could start), `before_wait`
 //              runs, and the next kernel is released only after the wait.
+//   l1_late  : with late_pdl: the norms come from the kernel right before this one after all (loaded after the wait).
 struct SelectRole {
     bool leader = true;
     int32_t* kept_sm = nullptr;
     bool clear_acc = true;
     bool late_pdl = false;
+    bool l1_late = false;
 };
 struct NoHook {
     __device__ void operator()() const {}
@@ -187,6 +190,7 @@ __device__ __forceinline__ void select_sample(const SampleDev& s, int b_local, c
     constexpr int NW = NT / 32;
     static_assert(EPT >= 1 && EPT * NT == CAP, "thread count must divide the capacity");
     static_assert(EPT * NW <= 128, "the emission prefix is taken by one warp, four entries per lane");
+    static_assert((2 * kCandMax * 8) % NT == 0 || NT % (2 * kCandMax * 8) == 0, "whole warps rank the listed keys");
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n2 = s.n_2d, n3 = s.n_3d, nv = n2 + n3;
     const int b_glob = io.chunk_first + b_local;
@@ -215,7 +219,7 @@ __device__ __forceinline__ void select_sample(const SampleDev& s, int b_local, c
             const int j = tid + e * NT;
             if (j < nv) {
                 if (carry) prev[e] = io.ahat_state[s.state_off + j];
-                if (gp.has_l1 && want_sums) nrm[e] = io.l1[s.vis_off + j];
+                if (gp.has_l1 && want_sums && !role.l1_late) nrm[e] = io.l1[s.vis_off + j];
             }
         }
         before_wait();
@@ -232,6 +236,8 @@ __device__ __forceinline__ void select_sample(const SampleDev& s, int b_local, c
             else if (!io.part) a[e] = io.attn[s.vis_off + j];
             if (!role.late_pdl) {
                 if (carry) prev[e] = io.ahat_state[s.state_off + j];
+                if (gp.has_l1 && want_sums) nrm[e] = io.l1[s.vis_off + j];
+            } else if (role.l1_late) {
                 if (gp.has_l1 && want_sums) nrm[e] = io.l1[s.vis_off + j];
             }
         }
@@ -369,9 +375,9 @@ __device__ __forceinline__ void select_sample(const SampleDev& s, int b_local, c
 
     // ---- 3./4. threshold bin per modality, refined while the bin is crowded
     // st[e]: 0 dropped, 1 kept, 2 undecided (in the threshold bin, or not yet examined)
-    int st[EPT];
+    int st[EPT], slot[EPT];
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) st[e] = (tid + e * NT) < nv ? 2 : 0;
+    for (int e = 0; e < EPT; ++e) { st[e] = (tid + e * NT) < nv ? 2 : 0; slot[e] = -1; }
     bool act2 = true, act3 = true;            // the modality still has a histogram pass to run
     int mode2 = SEL_NONE, mode3 = SEL_NONE, need2 = 0, need3 = 0, k2 = 0, k3 = 0;
 #pragma unroll 1
@@ -423,9 +429,9 @@ __device__ __forceinline__ void select_sample(const SampleDev& s, int b_local, c
                 else if (r > tbin) st[e] = 0;
                 else if (mode == SEL_BIN_ALL) st[e] = 1;
                 else if (mode == SEL_LIST) {
-                    const int slot = atomicAdd(&sm.ncand[is3 ? 1 : 0], 1);
-                    sm.cand_key[is3 ? 1 : 0][slot] = key[e];
-                    sm.cand_idx[is3 ? 1 : 0][slot] = tid + e * NT;
+                    slot[e] = atomicAdd(&sm.ncand[is3 ? 1 : 0], 1);
+                    sm.cand_key[is3 ? 1 : 0][slot[e]] = key[e];
+                    sm.cand_idx[is3 ? 1 : 0][slot[e]] = tid + e * NT;
                 }
             }
         }
@@ -441,27 +447,32 @@ __device__ __forceinline__ void select_sample(const SampleDev& s, int b_local, c
     }
     if (mode2 == SEL_LIST || mode3 == SEL_LIST) {              // rank the few keys of the threshold bin
         __syncthreads();                                                                   // ---- barrier D
+        // All pairs at once: 8 lanes share one listed key c1 and compare it with four others each (one
+        // 16-byte load of keys, one of indices); three shuffles add their counts.  No thread loops over
+        // the list, so no warp lags behind the others.
+        for (int wk = tid; wk < 2 * kCandMax * 8; wk += NT) {      // (modality, key, group of four)
+            const int m = wk / (kCandMax * 8), c1 = (wk >> 3) & (kCandMax - 1), g = wk & 7;
+            const int n = sm.ncand[m];
+            const uint32_t k1 = sm.cand_key[m][c1];
+            const int i1 = sm.cand_idx[m][c1];
+            const uint4 q = reinterpret_cast<const uint4*>(sm.cand_key[m])[g];
+            const int4 ix = reinterpret_cast<const int4*>(sm.cand_idx[m])[g];
+            const int c = 4 * g;                               // entries past n are stale: masked
+            int cnt = ((c < n) & ((q.x > k1) | ((q.x == k1) & (ix.x < i1)))) ? 1 : 0;
+            cnt += ((c + 1 < n) & ((q.y > k1) | ((q.y == k1) & (ix.y < i1)))) ? 1 : 0;
+            cnt += ((c + 2 < n) & ((q.z > k1) | ((q.z == k1) & (ix.z < i1)))) ? 1 : 0;
+            cnt += ((c + 3 < n) & ((q.w > k1) | ((q.w == k1) & (ix.w < i1)))) ? 1 : 0;
+            cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
+            cnt += __shfl_xor_sync(0xffffffffu, cnt, 2);
+            cnt += __shfl_xor_sync(0xffffffffu, cnt, 4);
+            if (g == 0) sm.cand_rank[m][c1] = cnt;
+        }
+        __syncthreads();
 #pragma unroll
         for (int e = 0; e < EPT; ++e) {
-            if (e * NT >= nv) break;
-            if (st[e] != 2) continue;
-            const int j = tid + e * NT;
-            const bool is3 = j >= n2;
-            if ((is3 ? mode3 : mode2) != SEL_LIST) continue;
-            const int n = sm.ncand[is3 ? 1 : 0];
-            const uint4* ck = reinterpret_cast<const uint4*>(sm.cand_key[is3 ? 1 : 0]);
-            const int4* ci = reinterpret_cast<const int4*>(sm.cand_idx[is3 ? 1 : 0]);
-            const uint32_t kk = key[e];
-            int rank = 0;
-            for (int c = 0; c < n; c += 4) {                   // entries past n are stale: masked
-                const uint4 q = ck[c >> 2];
-                const int4 ix = ci[c >> 2];
-                rank += ((q.x > kk) | ((q.x == kk) & (ix.x < j))) ? 1 : 0;
-                rank += ((c + 1 < n) & ((q.y > kk) | ((q.y == kk) & (ix.y < j)))) ? 1 : 0;
-                rank += ((c + 2 < n) & ((q.z > kk) | ((q.z == kk) & (ix.z < j)))) ? 1 : 0;
-                rank += ((c + 3 < n) & ((q.w > kk) | ((q.w == kk) & (ix.w < j)))) ? 1 : 0;
-            }
-            st[e] = rank < (is3 ? need3 : need2) ? 1 : 0;
+            if (slot[e] < 0) continue;
+            const bool is3 = (tid + e * NT) >= n2;
+            st[e] = sm.cand_rank[is3 ? 1 : 0][slot[e]] < (is3 ? need3 : need2) ? 1 : 0;
         }
     }
 

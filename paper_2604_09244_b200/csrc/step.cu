@@ -108,6 +108,7 @@ select_copy_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__
         const int b = blockIdx.x;
         SelectRole role;
         role.late_pdl = true;
+        role.l1_late = true;                                // the norms may come from a kernel that ran beside the scoring
         if (tp.cta0[bd.n] > 0) role.kept_sm = list + bd.s[b].out_off;   // every word is its own "ready" signal
         select_sample<NT, CAP>(bd.s[b], b, gp, io, sm, role);
         return;
