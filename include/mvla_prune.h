@@ -251,6 +251,18 @@ int32_t mvla_prune_step(mvla_ctx *ctx, int32_t prune_point, int32_t batch,
                         int32_t *total_kept_out, void *stream);
 
 /*
+ * Failure-detection self-test (the paper has no counterpart).  Every device-side wait of this library is
+ * bounded: when it runs out the kernel gives up, returns, and leaves MVLA_ERR_TIMEOUT in the context's status
+ * word; from then on every call on the context returns MVLA_ERR_TIMEOUT (sticky) and a new context must be
+ * created.  This call makes exactly that happen on purpose and harmlessly: one warp runs the library's
+ * wait for a kept-list word on a word that nothing ever sets, with a limit of `limit_us` microseconds
+ * (1 .. 1000000) instead of the second used in production.  Nothing hangs and nothing faults: the kernel
+ * ends by itself after `limit_us`.  Enqueues on `stream`, does not synchronise; once the stream has run
+ * it, the context is in the timed-out state.  Errors: INVALID_ARG, CUDA.
+ */
+int32_t mvla_selftest_wait_timeout(mvla_ctx *ctx, uint32_t limit_us, void *stream);
+
+/*
  * Salience scores without a context and without any allocation.  (The paper has no counterpart:
  * this is a packaging variant of mvla_salience, same arithmetic, same kernels.)
  *
@@ -265,9 +277,14 @@ int32_t mvla_prune_step(mvla_ctx *ctx, int32_t prune_point, int32_t batch,
  *   - all calls on a device share the array and it keeps the previous call's contents (every entry
  *     that is read is rewritten first, and the timeout flag is cleared by each call);
  *   - calls whose GPU work may overlap (two streams without ordering) race on it: serialise them;
- *   - the first call on a device looks up the array's device address; make that first call
- *     outside any stream capture.
- * device: CUDA ordinal; dtype, n_heads, head_dim as in mvla_config; samples: host array [batch];
+ *   - the first call on a device looks up the array's device address (host threads may race to be
+ *     first: the look-up is guarded by a mutex); with CUDA's lazy module loading that first call is also
+ *     when the driver loads the kernels and places the 512 KiB array on the device, so make one warm-up
+ *     call per device before the region in which nothing may be allocated begins, and outside any
+ *     stream capture.
+ * device: CUDA ordinal; dtype: MVLA_DTYPE_BF16 or MVLA_DTYPE_FP32 (no 8-bit inputs here); head_dim: 64 or
+ * 128 (the other head dims of mvla_config need a context); n_heads as in mvla_config, keys ungrouped;
+ * samples: host array [batch];
  * q, k: device, [rows, n_heads, head_dim], 16-byte aligned; attn_out: device, sum(n_vis) floats in
  * visual order, caller-owned.  Enqueues on `stream`, does not synchronise.  If a bounded
  * device-side wait gives up, every attn_out entry is NaN (there is no context to hold a status).

@@ -342,6 +342,16 @@ GateParams gate_params(const mvla_ctx* ctx, int32_t mode, bool has_l1)
     return gp;
 }
 
+// A launch of the step failed after the scoring kernel was enqueued: the fixed-point accumulators of the
+// chunk must not keep this step's sums (the selection that clears them will not run).
+void clear_accumulators(unsigned long long* acc64, const BatchDesc& bd, cudaStream_t st)
+{
+    const SampleDev& first = bd.s[0];
+    const SampleDev& last = bd.s[bd.n - 1];
+    const size_t n = static_cast<size_t>(last.vis_off + last.n_2d + last.n_3d - first.vis_off);
+    cudaMemsetAsync(acc64 + first.vis_off, 0, n * sizeof(unsigned long long), st);
+}
+
 // ---- overlap of neighbouring prune steps (MVLA_FLAG_INPUTS_STABLE) ----
 // With stable inputs, scoring and selection of a step go to the side stream of the step's scratch set
 // (`par`); only the row copy stays on the caller's stream.  What the side-stream work of step k must follow:
@@ -694,8 +704,9 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->acc64), kSets * vis_all * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(ctx->acc64, 0, kSets * vis_all * sizeof(unsigned long long));
     ctx->rows_all = static_cast<size_t>(c.max_batch) * (c.max_text + ctx->max_vis);
-    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->tail_list), kSets * ctx->rows_all * sizeof(int32_t));
-    if (e == cudaSuccess) e = cudaMemset(ctx->tail_list, 0xFF, kSets * ctx->rows_all * sizeof(int32_t));
+    // (+ 1: a word that no launch ever writes, for mvla_selftest_wait_timeout)
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->tail_list), (kSets * ctx->rows_all + 1) * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->tail_list, 0xFF, (kSets * ctx->rows_all + 1) * sizeof(int32_t));
     if (c.patch_path) {
         const size_t alpha_n = static_cast<size_t>(c.n_heads) * c.max_text * vis_all;
         ctx->patch_sets = alpha_n * sizeof(float) * kSets <= (size_t(1) << 30) ? kSets : 1;   // at most 1 GiB of attention copies
@@ -863,6 +874,19 @@ int32_t mvla_compact(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, c
     return MVLA_OK;
 }
 
+int32_t mvla_selftest_wait_timeout(mvla_ctx* ctx, uint32_t limit_us, void* stream)
+{
+    if (!ctx || limit_us < 1 || limit_us > 1000000u) return MVLA_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return MVLA_ERR_CUDA;
+    // the last word of the kept-list scratch is never an output row of any launch: it stays -1
+    const int32_t* never_set = ctx->tail_list + kSets * ctx->rows_all;
+    const cudaError_t e = launch_wait_probe(never_set, static_cast<uint64_t>(limit_us) * 1000ull, ctx->status_dev,
+                                            static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    return MVLA_OK;
+}
+
 int32_t mvla_patch_indicators(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const void* q, const void* k,
                               const void* hidden, int64_t rows, float* attn_out, float* x_out, void* stream)
 {
@@ -1008,11 +1032,17 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
             const cudaError_t e2 = launch_select_copy(bd, gp, io, job, ctx->tail_list + par * ctx->rows_all,
                                                       ctx->status_dev,
                                                       ctx->sm_count * kTailCtasPerSm - n, st);
-            if (e2 != cudaSuccess) return fail_cuda(ctx, e2);
+            if (e2 != cudaSuccess) {
+                clear_accumulators(acc64, bd, st);
+                return fail_cuda(ctx, e2);
+            }
             continue;
         }
         cudaError_t e = launch_select(bd, gp, io, sel_stream);
-        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        if (e != cudaSuccess) {
+            if (used_acc64) clear_accumulators(acc64, bd, sel_stream);
+            return fail_cuda(ctx, e);
+        }
         if (forked) {                                // join: the row copy, and whatever the caller enqueues next
             rc = join_selection(ctx, fp, par, sel_stream, st);
             if (rc != MVLA_OK) return rc;

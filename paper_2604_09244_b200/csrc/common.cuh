@@ -83,6 +83,9 @@ inline cudaLaunchAttribute pdl_attribute()
     return a;
 }
 
+// Multiprocessors of the current device (looked up once per device).
+int sm_count_of_current_device();
+
 // ---- launchers (each enqueues on `stream` and returns the launch status) ----
 
 // bf16 tensor-core salience with logits held in registers (one or two key tiles per CTA).  With
@@ -179,6 +182,10 @@ cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int
 bool select_copy_supported(const BatchDesc& bd);
 cudaError_t launch_select_copy(const BatchDesc& bd, const GateParams& gp, const SelectIO& io, const CompactJob& job,
                                int32_t* list, int* status, int ctas, cudaStream_t stream);
+
+// One warp runs the copying CTAs' bounded wait on `never_set` (a word that holds -1 and stays so) with the
+// given limit and reports MVLA_ERR_TIMEOUT into `status` when it runs out.
+cudaError_t launch_wait_probe(const int32_t* never_set, uint64_t limit_ns, int* status, cudaStream_t stream);
 
 // ---- patch-by-patch path (Alg. 1 taken literally) ----
 struct PatchParams {

@@ -83,6 +83,19 @@ compact_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ Com
 
 }  // namespace
 
+int sm_count_of_current_device()
+{
+    static int cached[64] = {};              // 0: not looked up yet (written once per device with the same value)
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int32_t* kept_idx,
                            int32_t chunk_rows, int32_t chunk_row0, const int32_t* out_offsets,
                            int32_t chunk_first, int32_t batch_total, cudaStream_t stream)
@@ -92,7 +105,8 @@ cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int
     if (total == 0 || chunk_rows <= 0) return cudaSuccess;
     const int64_t units = static_cast<int64_t>(chunk_rows) * total;
     int64_t blocks = (units + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    if (out_offsets) blocks = std::min<int64_t>(blocks, 148 * 32);     // capacity launch: a bounded grid strides over the rows that exist
+    if (out_offsets)      // capacity launch: a bounded grid strides over the rows that exist
+        blocks = std::min<int64_t>(blocks, static_cast<int64_t>(sm_count_of_current_device()) * 32);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(blocks));
     cfg.blockDim = dim3(kWarpsPerBlock * 32);

@@ -15,6 +15,7 @@
 #include "device_utils.cuh"
 #include "select_impl.cuh"
 #include "tmem_ld.cuh"
+#include "tmem_plan.h"
 
 #include <algorithm>
 #include <cstring>
@@ -135,6 +136,8 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     cluster_arrive_release();                 // publishes this CTA's barriers; matched by the wait before the first remote store
     uint32_t tmem_cols = 32;
     while (tmem_cols < static_cast<uint32_t>(CC)) tmem_cols <<= 1;
+    // blocks until the columns are free: the launcher has made sure that the CTAs resident on a multiprocessor
+    // never ask for more than its 512 columns together, so no CTA waits here for one that waits for it
     if (warp == 1) tmem_alloc(smem_u32(&s_tmem), tmem_cols);
     tc_fence_before();
     __syncthreads();
@@ -307,10 +310,18 @@ cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int he
                           const CUtensorMap* tk, int cluster, int npad, float* part, int64_t part_stride,
                           unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, int32_t* rearm, cudaStream_t stream)
 {
-    const size_t smem = 1024 + static_cast<size_t>((head_dim * esize + 127) / 128) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
+    size_t smem = 1024 + static_cast<size_t>((head_dim * esize + 127) / 128) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
     auto kern = salience_fast_kernel<TCOL, NTILE>;
+    // resident CTAs x tensor-memory columns must not exceed the 512 of a multiprocessor
+    const int tmem_cols = tmem_cols_for(TCOL * NTILE);
+    smem = smem_for_tmem(smem, tmem_cols);
+    if (smem == 0) return cudaErrorInvalidConfiguration;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
+    int resident = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kern, kFastThreads, smem);
+    if (e != cudaSuccess) return e;
+    if (resident * tmem_cols > kTmemColsPerSm) return cudaErrorInvalidConfiguration;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cluster, n_heads, bd.n);
     cfg.blockDim = dim3(kFastThreads);

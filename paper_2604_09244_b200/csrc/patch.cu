@@ -433,9 +433,10 @@ cudaError_t launch_patch_indicators(const BatchDesc& bd, int n_heads, AlphaOut a
     int max_p = 0;
     for (int b = 0; b < bd.n; ++b) max_p = max(max_p, bd.s[b].n_2d);
     if (max_p == 0) return cudaSuccess;
-    // as many patches per CTA as still give every SM a CTA (148 SMs)
+    // as many patches per CTA as still give every multiprocessor a CTA
     int pp = 8;
-    while (pp > 2 && static_cast<int64_t>(bd.n) * ((max_p + pp - 1) / pp) < 148) pp >>= 1;
+    const int sms = sm_count_of_current_device();
+    while (pp > 2 && static_cast<int64_t>(bd.n) * ((max_p + pp - 1) / pp) < sms) pp >>= 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((max_p + pp - 1) / pp, bd.n);
     cfg.blockDim = dim3(kIndThreads);

@@ -10,6 +10,7 @@
 // later in a fixed order so that the result does not depend on scheduling.
 #include "common.cuh"
 #include "device_utils.cuh"
+#include "tmem_plan.h"
 
 #include <math_constants.h>
 
@@ -85,6 +86,8 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
                     tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * box_elems, hk, ti.row0, bar_full);
             }
         }
+        // blocks until the columns are free: the launcher has made sure that the CTAs resident on a multiprocessor
+        // never ask for more than its 512 columns together, so no CTA waits here for one that waits for it
         if (warp == 1) tmem_alloc(smem_u32(&s_tmem), tmem_cols);
         tc_fence_before();
         __syncthreads();
@@ -351,8 +354,21 @@ cudaError_t launch_salience_t(const BatchDesc& bd, int n_heads, int kv_group, in
                                 static_cast<size_t>(tiles_per_cta) * npad * kKeyTile);
     if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
     auto kern = salience_kernel<T, UMMA>;
+    int tmem_cols = 0;
+    if (UMMA) {       // resident CTAs x tensor-memory columns must not exceed the 512 of a multiprocessor
+        const int tcol = npad <= 16 ? 16 : (npad <= 32 ? 32 : 64);
+        tmem_cols = tmem_cols_for(tiles_per_cta * tcol);
+        smem = smem_for_tmem(smem, tmem_cols);
+        if (smem == 0) return cudaErrorInvalidConfiguration;
+    }
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
+    if (UMMA) {
+        int resident = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kern, kThreads, smem);
+        if (e != cudaSuccess) return e;
+        if (resident * tmem_cols > kTmemColsPerSm) return cudaErrorInvalidConfiguration;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cluster, n_heads, bd.n);
     cfg.blockDim = dim3(kThreads);

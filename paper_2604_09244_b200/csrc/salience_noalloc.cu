@@ -21,6 +21,7 @@
 
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 
 namespace {
 
@@ -39,9 +40,11 @@ struct DeviceScratch {
     bool ready;
 };
 DeviceScratch g_dev[kMaxDevices] = {};
+std::mutex g_dev_mutex;          // host threads may make their first call on a device at the same time
 
 cudaError_t scratch_for_current_device(int dev, DeviceScratch** out)
 {
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
     DeviceScratch& d = g_dev[dev];
     if (!d.ready) {
         void *p = nullptr, *f = nullptr;

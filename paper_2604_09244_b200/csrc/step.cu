@@ -91,6 +91,26 @@ __device__ __forceinline__ int ld_relaxed_gpu(const int* p)
     return v;
 }
 
+// Bounded wait for one word of the kept list.  Returns the word, or -1 when `limit_ns` ran out.
+__device__ __forceinline__ int poll_word(const int* p, uint64_t t0, uint64_t limit_ns)
+{
+    int v = ld_relaxed_gpu(p);
+    for (uint32_t it = 0; v < 0 && it < kSpinLimit; ++it) {
+        __nanosleep(20);
+        v = ld_relaxed_gpu(p);
+        if ((it & 63u) == 63u && global_ns() - t0 > limit_ns) break;
+    }
+    return v;
+}
+
+// The same wait on a word that nothing ever sets, with a short limit: lets a test (or a health check) see
+// the whole failure path -- the wait gives up, the kernel returns, the status word holds the error --
+// without any kernel being made to hang.
+__global__ void wait_probe_kernel(const int* never_set, uint64_t limit_ns, int* status)
+{
+    if (poll_word(never_set, global_ns(), limit_ns) < 0) *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
+}
+
 // grid: CTAs 0 .. n-1 select (CTA b for sample b of the launch), the CTAs after them copy; tp.cta0[b] is the
 // first copying CTA of sample b.  `list`: the kept list in library scratch (one word per output row of the
 // launch's samples, -1 = not yet known; the scoring kernel before this one has set them all to -1).
@@ -143,12 +163,7 @@ select_copy_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__
         const uint64_t t0 = global_ns();
         copy_rows(ca, n_rows, w, nw, lane, [&](int i, int64_t& srow, int64_t& drow) {
             const int r = (text_early && i >= baset) ? i + s.n_txt : i;       // skip the text rows copied before
-            int v = ld_relaxed_gpu(kept + r);               // the whole warp reads one word: one request
-            for (uint32_t it = 0; v < 0 && it < kSpinLimit; ++it) {
-                __nanosleep(20);
-                v = ld_relaxed_gpu(kept + r);
-                if ((it & 63u) == 63u && global_ns() - t0 > 1000000000ull) break;
-            }
+            const int v = poll_word(kept + r, t0, 1000000000ull);   // the whole warp reads one word: one request
             if (v < 0) {                                    // gave up: report, leave the row alone
                 *reinterpret_cast<volatile int*>(status) = MVLA_ERR_TIMEOUT;
                 return false;
@@ -184,6 +199,12 @@ int max_vis_of(const BatchDesc& bd)
 }  // namespace
 
 bool select_copy_supported(const BatchDesc& bd) { return max_vis_of(bd) <= 2048; }
+
+cudaError_t launch_wait_probe(const int32_t* never_set, uint64_t limit_ns, int* status, cudaStream_t stream)
+{
+    wait_probe_kernel<<<1, 32, 0, stream>>>(never_set, limit_ns, status);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_select_copy(const BatchDesc& bd, const GateParams& gp, const SelectIO& io, const CompactJob& job,
                                int32_t* list, int* status, int ctas, cudaStream_t stream)

@@ -588,3 +588,82 @@ def test_fp8_step_single_frame_shape():
     ctx = mvla.context_for(wl)
     run_and_check_step(ctx, wl, 0, [oracle.State(s.n_vis) for s in wl.samples])
     ctx.close()
+
+
+# ------------------------------------------------------------------ fused tail: ties, guard bands, bounded waits
+def _duplicate_visual_rows(wl, group):
+    """Make groups of `group` neighbouring visual tokens identical (hidden, q, k, v): tokens of one 128-key
+    tile then get bit-identical scores, so the selection has to fall back on the index."""
+    t = wl.steps[0]
+    for s in wl.samples:
+        for off, n in ((s.off_2d, s.n_2d), (s.off_3d, s.n_3d)):
+            rows = s.seq_off + off + np.arange(n)
+            src = s.seq_off + off + (np.arange(n) // group) * group
+            for name in ("hidden", "q", "k", "v"):
+                getattr(t, name)[rows] = getattr(t, name)[src]
+
+
+@pytest.mark.parametrize("mode", [W.MODE_FIXED, W.MODE_ADAPTIVE])
+@pytest.mark.parametrize("sizes", [((200, 77), (300, 500)), ((900, 1000), (1100, 130))])   # <= 1024 and <= 2048 tokens
+@pytest.mark.parametrize("group", [8, 4096])                                                  # runs of 8; everything equal
+def test_step_with_equal_scores_straddling_the_budget(mode, sizes, group):
+    wl = W.small_workload(91, batch=2, D=256, H=2, d=64, dtype="bf16", mode=mode, n_txt=(9, 20), n_2d=sizes[0],
+                          n_3d=sizes[1], keep=(0.37, 0.21), keep_fixed=(0.33, 0.41))
+    _duplicate_visual_rows(wl, group)
+    ctx = mvla.context_for(wl)
+    out, refs = run_and_check_step(ctx, wl, 0, _fresh_states(wl))     # includes the exact stage-wise check
+    ahat = out.ahat.cpu().numpy()
+    assert len(np.unique(ahat)) < 0.6 * len(ahat), "the case was meant to hold many equal scores"
+    ctx.close()
+
+
+def test_step_leaves_the_bytes_behind_its_outputs_alone():
+    # stands in for a memory checker: capacity-sized output buffers are filled with a pattern, and whatever
+    # lies behind the rows / list entries the step reports must still hold it afterwards
+    wl = W.small_workload(93, batch=3, D=256, H=4, d=128, dtype="bf16", n_txt=(5, 19, 33), n_2d=(70, 130, 260),
+                          n_3d=(150, 37, 300), keep=(0.4, 0.3, 0.55))
+    ctx = mvla.context_for(wl)
+    dev = device_tensors(wl)
+    for flags in (0, mvla.FLAG_INPUTS_STABLE):
+        out = ctx.alloc_outputs(wl.samples, extras=True)
+        for t in (out.out_hidden, out.out_k, out.out_v):
+            t.view(torch.int16).fill_(0x5A5A)
+        out.kept_idx.fill_(-77)
+        ctx.prune_step(0, wl.samples, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"], flags=flags | mvla.FLAG_RESET_STATE,
+                       out=out)
+        torch.cuda.synchronize()
+        n = out.total_kept
+        assert 0 < n < out.kept_idx.numel() and int(out.out_offsets[-1]) == n
+        assert bool((out.kept_idx[n:] == -77).all()), "list entries past the total were written"
+        assert bool((out.kept_idx[:n] >= 0).all())
+        for t in (out.out_hidden, out.out_k, out.out_v):
+            assert bool((t[n:].view(torch.int16) == 0x5A5A).all()), "rows past the total were written"
+    ctx.close()
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_sticky():
+    # the wait is the one the row-copying CTAs use for a kept-list word; here it polls a word nothing sets,
+    # with a limit of 200 us: the kernel ends by itself, the status word holds the error
+    wl = W.small_workload(95, batch=1, D=256, H=2, d=64, dtype="bf16", n_txt=(5,), n_2d=(70,), n_3d=(150,))
+    dev = device_tensors(wl)
+    ctx = mvla.context_for(wl)
+    ctx.prune_step(0, wl.samples, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"])     # healthy before
+    torch.cuda.synchronize()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    ctx.selftest_wait_timeout(200)
+    t1.record()
+    torch.cuda.synchronize()
+    assert 0.15 < t0.elapsed_time(t1) < 50.0, "the wait must end by itself after about its limit"
+    for call in (lambda: ctx.prune_step(0, wl.samples, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"]),
+                 lambda: ctx.salience(wl.samples, dev["q"], dev["k"])):
+        with pytest.raises(mvla.MvlaError) as e:
+            call()
+        assert e.value.code == mvla.ERR_TIMEOUT                       # sticky: every later call reports it
+    ctx.close()
+    ctx2 = mvla.context_for(wl)                                       # a fresh context works
+    out, refs = run_and_check_step(ctx2, wl, 0, _fresh_states(wl))
+    with pytest.raises(mvla.MvlaError) as e:
+        ctx2.selftest_wait_timeout(0)                                 # the limit must be 1 us .. 1 s
+    assert e.value.code == mvla.ERR_INVALID_ARG
+    ctx2.close()

@@ -286,3 +286,25 @@ def test_pipelined_patch_steps_match_serial_steps():
         for x, y in zip(a, b):
             assert np.array_equal(x, y)
     assert serial[0][2].sum() > serial[-1][2].sum()      # the cold-start step kept everything, later steps prune
+
+
+def test_patch_step_leaves_the_bytes_behind_its_outputs_alone():
+    # the row copy of this path is launched over the capacity (the row count is known only on the device):
+    # rows and list entries past out_offsets[batch] must keep the pattern they were filled with
+    wl = W.patch_workload(17, batch=3, D=256, H=4, d=128, n_txt=(7, 20, 33), n_patch=(90, 200, 130))
+    ctx = mvla.context_for(wl)
+    dev = device_tensors(wl)
+    u = torch.from_numpy(wl.extra["rand_u"][0]).cuda()
+    out = ctx.alloc_outputs(wl.samples, extras=True, patch=True)
+    for t in (out.out_hidden, out.out_k, out.out_v):
+        t.view(torch.int16).fill_(0x5A5A)
+    out.kept_idx.fill_(-77)
+    ctx.prune_step(0, wl.samples, mvla.MODE_PATCH, dev["q"], dev["k"], dev["v"], dev["hidden"], rand_u=u, out=out,
+                   flags=mvla.FLAG_RESET_STATE)
+    torch.cuda.synchronize()
+    n = int(out.out_offsets[-1])
+    assert 0 < n < out.kept_idx.numel()
+    assert bool((out.kept_idx[n:] == -77).all()), "list entries past the total were written"
+    for t in (out.out_hidden, out.out_k, out.out_v):
+        assert bool((t[n:].view(torch.int16) == 0x5A5A).all()), "rows past the total were written"
+    ctx.close()
