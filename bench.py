@@ -7,13 +7,18 @@ A "step" is one fused prune step (`mvla_prune_step` through the C ABI) over one 
 synthetic input.  The default workload is the 7B-shaped single frame (32 text + 256 2D + 512 3D
 tokens, D=4096, 32 heads x 128, bf16, keep 40 % / 30 %).  Prints ONE JSON line.
 
-* `value`: visual tokens pruned per second, whole job, inputs resident in HBM.  The steps are
-  captured in CUDA graphs (one step per rotated input set) and replayed; CUDA events bracket the
-  K timed steps; inputs rotate over enough distinct sets to exceed L2.
+* `value`, `ms_per_step`, `latency_us`: EXACTLY --steps steps enqueued one after another in one stream (every
+  kernel waits for the work before it: what one request inside a prefill sees), inputs resident in HBM and
+  rotating over enough distinct sets to exceed L2, captured in CUDA graphs, bracketed by CUDA events.
+  `serial_us_per_step` gives p10 / median / p90 over replays of the same graph.
+* `overlapped`: the period of independent requests overlapping inside the library (MVLA_FLAG_INPUTS_STABLE).
+* `isolated_latency_us`: one step per graph launch with a device synchronise in between.
 * `e2e`: the same metric with the step's inputs copied from pinned host memory and its results
   copied back inside the timed region.
-* `roofline`: the dominant kernel's stage timed alone through its own C-ABI entry point.
-* `cpu_baseline` / `--impl reference`: the fp64 CPU oracle, as it stands, on the host cores.
+* `roofline`: the longer of the step's two kernels, timed as the step runs it.
+* `other_configs`: serial / overlapped step time of the other workloads (default run only).
+* `cpu_baseline` / `--impl reference`: the fp64 CPU oracle, as it stands, on the host cores (all, and one).
+* `--gpus N` without a launcher environment starts the N ranks itself (one process per GPU, replicas).
 """
 from __future__ import annotations
 
@@ -179,11 +184,13 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
-def time_oracle(wl, max_steps: int, max_seconds: float):
+def time_oracle(wl, max_steps: int, max_seconds: float, threads: int = 0):
     """The oracle as it stands: full prune steps (all samples) + compaction of hidden/K/V, repeated
-    `max_steps` times or until `max_seconds` of CPU work.  Returns (seconds per step, steps, cores)."""
-    import numpy as np
+    `max_steps` times or until `max_seconds` of CPU work.  `threads`: 0 = all the process may use.
+    Returns (seconds per step, steps, cores)."""
     import oracle
+    all_cores = len(os.sched_getaffinity(0))
+    oracle.set_num_threads(threads if threads > 0 else all_cores)
     t = wl.steps[-1]
     patch = wl.mode == 2
     p = oracle.patch_params_of(wl) if patch else oracle.params_of(wl)
@@ -206,7 +213,8 @@ def time_oracle(wl, max_steps: int, max_seconds: float):
         el = time.perf_counter() - t0
         if el >= max_seconds or n >= max_steps:
             break
-    cores = min(oracle.num_threads(), wl.n_heads, len(os.sched_getaffinity(0)))
+    cores = min(oracle.num_threads(), wl.n_heads, all_cores)
+    oracle.set_num_threads(all_cores)
     return el / n, n, cores
 
 
@@ -231,253 +239,356 @@ def run_reference(args, rank):
 
 
 # ----------------------------------------------------------------------------- GPU arm
-def run_ours(args, rank, local, world):
-    import numpy as np
-    import torch
-    from paper_2604_09244_b200 import dist as D
-    from paper_2604_09244_b200 import mvla
+class Harness:
+    """One workload resident on the device over rotating input / output sets, and the ways of timing it."""
 
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    wl, desc = make_workload(args.workload)
-    step_t = wl.steps[-1]
-    names = ("q", "k", "v", "hidden")
-    tdt = {"bf16": torch.bfloat16, "fp32": torch.float32, "fp8": torch.float8_e4m3fn}[wl.dtype]
-    host = {n: torch.from_numpy(getattr(step_t, n)).to(torch.bfloat16 if (wl.dtype == "fp8" and n == "hidden") else tdt).contiguous()
-            for n in names}
-    in_bytes = sum(t.numel() * t.element_size() for t in host.values())
+    def __init__(self, name, dev, world):
+        import numpy as np
+        import torch
+        from paper_2604_09244_b200 import mvla
+        self.np, self.torch, self.mvla, self.world, self.dev = np, torch, mvla, world, dev
+        self.wl, self.desc = make_workload(name)
+        wl = self.wl
+        step_t = wl.steps[-1]
+        self.names = ("q", "k", "v", "hidden")
+        tdt = {"bf16": torch.bfloat16, "fp32": torch.float32, "fp8": torch.float8_e4m3fn}[wl.dtype]
+        self.host = {n: torch.from_numpy(getattr(step_t, n)).to(torch.bfloat16 if (wl.dtype == "fp8" and n == "hidden") else tdt).contiguous()
+                     for n in self.names}
+        self.in_bytes = sum(t.numel() * t.element_size() for t in self.host.values())
+        # A single-frame workload is a stream of independent requests: each step starts a fresh smoothed
+        # state, and requests in flight at the same time hold distinct state slots, as the concurrent
+        # requests of a server do.  A workload with carry-over keeps its one episode (one slot per sample).
+        self.is_patch = wl.mode == 2
+        self.u_dev = torch.from_numpy(wl.extra["rand_u"][-1]).to(dev) if self.is_patch else None
+        self.n_req = 8 if not wl.cold_start_full_keep else 1
+        self.ctx = mvla.context_for(wl, n_state_slots=self.n_req * len(wl.samples))
+        probe = self.ctx.alloc_outputs(wl.samples, extras=False)
+        self.out_bytes_alloc = sum(t.numel() * t.element_size() for t in (probe.out_hidden, probe.out_k, probe.out_v))
+        # Enough distinct sets that the bytes a step actually touches (about its algorithmic bytes), summed
+        # over the sets, are at least twice the L2, so that no set can still be cached when its turn comes
+        # again -- and at least six: a step whose buffers were written by one of the five steps before it
+        # is ordered after them by the library.
+        self.probe_rows = sum(s.n_txt + s.n_2d + s.n_3d for s in wl.samples)
+        self.touched = algorithmic_bytes(wl, self.probe_rows // 3)["total"]
+        self.n_sets = min(64, max(6, int(np.ceil(2.0 * L2_BYTES / self.touched))))
+        self.sets = [{n: self.host[n].to(dev) for n in self.names} for _ in range(self.n_sets)]
+        self.outs = [probe] + [self.ctx.alloc_outputs(wl.samples, extras=False) for _ in range(self.n_sets - 1)]
+        self.cs = mvla.c_samples(wl.samples)
+        self.cs_req = [mvla.c_samples([dataclasses.replace(x, state_slot=x.state_slot + j * len(wl.samples))
+                                       for x in wl.samples]) for j in range(self.n_req)]
+        self.flags = mvla.FLAG_RESET_STATE if not wl.cold_start_full_keep else 0
+        if wl.cold_start_full_keep:      # absorb the cold-start step so that the timed steps prune
+            s0 = self.sets[0]
+            self.ctx.prune_step(0, self.cs, wl.mode, s0["q"], s0["k"], s0["v"], s0["hidden"], out=self.outs[0])
+            self.flags = mvla.FLAG_NO_STATE_UPDATE
+        o0 = self.step(0)
+        torch.cuda.synchronize()
+        # the patch-by-patch path decides its row count on the device (total_kept is then the capacity bound)
+        self.kept_rows = int(o0.out_offsets[-1]) if self.is_patch else o0.total_kept
+        # kernels of one step: scoring (+ norms) + selection-and-copy; the patch path has five
+        self.launches_per_step = 5 if self.is_patch else 2 + (1 if wl.mode == 1 else 0)
+        self.launches_per_step_overlapped = 5 if self.is_patch else 3 + (1 if wl.mode == 1 else 0)
+        self.per_graph = -(-56 // self.n_sets) * self.n_sets     # steps per graph: a whole number of rotations
 
-    # A single-frame workload is a stream of independent requests: each step starts a fresh smoothed
-    # state, and requests in flight at the same time hold distinct state slots, as the concurrent
-    # requests of a server do.  A workload with carry-over keeps its one episode (one slot per sample).
-    is_patch = wl.mode == 2
-    u_dev = torch.from_numpy(wl.extra["rand_u"][-1]).to(dev) if is_patch else None
-    n_req = 8 if not wl.cold_start_full_keep else 1
-    ctx = mvla.context_for(wl, n_state_slots=n_req * len(wl.samples))
-    probe = ctx.alloc_outputs(wl.samples, extras=False)
-    out_bytes_alloc = sum(t.numel() * t.element_size() for t in (probe.out_hidden, probe.out_k, probe.out_v))
-    # Enough distinct sets that the bytes a step actually touches (about its algorithmic bytes: the
-    # visual K rows, the text Q rows, the kept rows read and written), summed over the sets, are at
-    # least twice the L2, so that no set can still be cached when its turn comes again.
-    probe_rows = sum(s.n_txt + s.n_2d + s.n_3d for s in wl.samples)
-    touched = algorithmic_bytes(wl, probe_rows // 3)["total"]        # kept rows are a third to a half of the rows
-    # ... and at least six: a step whose buffers were written by one of the five steps before it is
-    # ordered after them by the library, which would time the serial path only.
-    n_sets = min(64, max(6, int(np.ceil(2.0 * L2_BYTES / touched))))
-    # distinct input sets: same values, distinct addresses (the cache cannot tell values apart)
-    sets = [{n: host[n].to(dev) for n in names} for _ in range(n_sets)]
-    outs = [probe] + [ctx.alloc_outputs(wl.samples, extras=False) for _ in range(n_sets - 1)]
-    cs = mvla.c_samples(wl.samples)
-    cs_req = [mvla.c_samples([dataclasses.replace(x, state_slot=x.state_slot + j * len(wl.samples))
-                              for x in wl.samples]) for j in range(n_req)]
-    flags = mvla.FLAG_RESET_STATE if not wl.cold_start_full_keep else 0
-    if wl.cold_start_full_keep:      # absorb the cold-start step so that the timed steps prune
-        ctx.prune_step(0, cs, wl.mode, sets[0]["q"], sets[0]["k"], sets[0]["v"], sets[0]["hidden"], out=outs[0])
-        flags = mvla.FLAG_NO_STATE_UPDATE
+    def step(self, i, extra=0):
+        s, o = self.sets[i % self.n_sets], self.outs[i % self.n_sets]
+        return self.ctx.prune_step(0, self.cs_req[i % self.n_req], self.wl.mode, s["q"], s["k"], s["v"], s["hidden"],
+                                   flags=self.flags | extra, out=o, rand_u=self.u_dev)
 
-    def step(i, extra=0):
-        s, o = sets[i % n_sets], outs[i % n_sets]
-        return ctx.prune_step(0, cs_req[i % n_req], wl.mode, s["q"], s["k"], s["v"], s["hidden"],
-                              flags=flags | extra, out=o, rand_u=u_dev)
-
-    o0 = step(0)
-    torch.cuda.synchronize()
-    # the patch-by-patch path decides its row count on the device (total_kept is then the capacity bound)
-    kept_rows = int(o0.out_offsets[-1]) if is_patch else o0.total_kept
-    # patch path: norms, scoring, indicators, select, row copy
-    launches_per_step = 5 if is_patch else 3 + (1 if wl.mode == 1 else 0)
-
-    # ---- device-resident timing: CUDA graphs of back-to-back steps over the rotating sets
-    per_graph = -(-200 // n_sets) * n_sets   # ~200 steps per graph: the pipeline of overlapping steps fills once per replay
-    replays = max(1, int(np.ceil(args.steps / per_graph)))
-    warm_replays = max(1, int(np.ceil(max(3, args.warmup) / per_graph)))
-    K = replays * per_graph
-
-    def capture(n_steps, extra):
+    def capture(self, n_steps, extra):
+        torch = self.torch
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
-            for i in range(min(n_steps, n_sets)):
-                step(i, extra)
+            for i in range(min(n_steps, self.n_sets)):
+                self.step(i, extra)
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             for i in range(n_steps):
-                step(i, extra)
+                self.step(i, extra)
         return g
 
-    def timed(g, n_replays, sampler=None):
-        for _ in range(warm_replays):
+    def timed_exact(self, extra, steps, warmup):
+        """EXACTLY `steps` timed steps after `warmup` (>= 3) untimed ones: whole graphs of per_graph steps
+        plus one shorter graph for the remainder.  Returns milliseconds for the `steps` steps (max over ranks)."""
+        from paper_2604_09244_b200 import dist as D
+        torch = self.torch
+        g = self.capture(self.per_graph, extra)
+        rem = steps % self.per_graph
+        g_rem = self.capture(rem, extra) if rem else None
+        for _ in range(max(1, -(-max(3, warmup) // self.per_graph))):
             g.replay()
+        if g_rem:
+            g_rem.replay()
         torch.cuda.synchronize()
-        D.barrier(world)
+        D.barrier(self.world)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         e0.record()
-        for _ in range(n_replays):
+        for _ in range(steps // self.per_graph):
             g.replay()
+        if g_rem:
+            g_rem.replay()
         e1.record()
         torch.cuda.synchronize()
-        D.barrier(world)
-        return D.max_over_ranks(e0.elapsed_time(e1), world, dev)
+        D.barrier(self.world)
+        return D.max_over_ranks(e0.elapsed_time(e1), self.world, self.dev), g
 
-    # The benchmark's inputs are static buffers and its output sets rotate, so the promise behind
-    # MVLA_FLAG_INPUTS_STABLE holds: neighbouring steps may overlap inside the library.
-    graph = capture(per_graph, mvla.FLAG_INPUTS_STABLE)
+    def distribution(self, g, min_seconds=0.25, min_replays=12):
+        """Per-step time of every replay of graph `g` (one event pair per replay): p10 / median / p90 in us."""
+        torch = self.torch
+        per = []
+        t_end = time.perf_counter() + min_seconds
+        while len(per) < min_replays or time.perf_counter() < t_end:
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(8)]
+            for a, b in evs:
+                a.record()
+                g.replay()
+                b.record()
+            torch.cuda.synchronize()
+            per += [a.elapsed_time(b) * 1e3 / self.per_graph for a, b in evs]
+            if len(per) > 4000:
+                break
+        per.sort()
+        q = lambda f: per[min(len(per) - 1, int(f * len(per)))]
+        return {"p10": q(0.10), "median": q(0.50), "p90": q(0.90), "replays": len(per), "steps_per_replay": self.per_graph}
+
+    def isolated(self, n=64):
+        torch = self.torch
+        g1 = self.capture(1, 0)
+        lat = []
+        for _ in range(n):
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            g1.replay()
+            b.record()
+            torch.cuda.synchronize()
+            lat.append(a.elapsed_time(b) * 1e3)
+        lat.sort()
+        return {"p10": lat[n // 10], "median": lat[n // 2], "p90": lat[(9 * n) // 10],
+                "how": "one step per graph launch, device synchronised between launches (includes the graph launch)"}
+
+    def kernel_times(self, replays=30):
+        """Duration of the step's kernels as the step runs them: one CUDA graph of one rotation of
+        (non-overlapped) steps with an event before each step, the library's stage event between its scoring
+        kernel(s) and its selection + copy kernel, and an event after it.  Returns mean microseconds."""
+        torch = self.torch
+        if self.is_patch:
+            return None
+        n = self.n_sets
+        ev = [[torch.cuda.Event(enable_timing=True, external=True) for _ in range(3)] for _ in range(n)]
+        for i in range(n):
+            self.step(i)
+        torch.cuda.synchronize()
+        for e3 in ev:                        # torch creates events lazily: record each once outside the capture
+            for e in e3:
+                e.record()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(n):
+                ev[i][0].record()
+                self.ctx.set_stage_event(ev[i][1])
+                self.step(i)
+                ev[i][2].record()
+        self.ctx.set_stage_event(None)
+        sc, tl = [], []
+        for r in range(replays + 2):
+            g.replay()
+            torch.cuda.synchronize()
+            if r >= 2:
+                sc += [e[0].elapsed_time(e[1]) * 1e3 for e in ev]
+                tl += [e[1].elapsed_time(e[2]) * 1e3 for e in ev]
+        sc.sort(); tl.sort()
+        trim = lambda v: sum(v[len(v) // 10: len(v) - len(v) // 10]) / max(1, len(v) - 2 * (len(v) // 10))
+        return {"scoring": trim(sc), "tail": trim(tl), "launches": len(sc)}
+
+    def e2e(self, steps):
+        """Pinned host inputs -> device, step, results -> pinned host, every step, inside the timed region."""
+        from paper_2604_09244_b200 import dist as D
+        torch, wl = self.torch, self.wl
+        pin_in = {n: self.host[n].pin_memory() for n in self.names}
+        stage_in = {n: torch.empty_like(self.host[n], device=self.dev) for n in self.names}
+        o, kr = self.outs[0], self.kept_rows
+        res_dev = [o.out_hidden[:kr], o.out_k[:kr], o.out_v[:kr], o.kept_idx[:kr], o.out_offsets, o.budgets]
+        res_host = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in res_dev]
+        u_pin = torch.from_numpy(wl.extra["rand_u"][-1]).pin_memory() if self.is_patch else None
+        u_stage = torch.empty_like(self.u_dev) if self.is_patch else None
+        h2d = self.in_bytes + (u_pin.numel() * 4 if self.is_patch else 0)
+        d2h = sum(t.numel() * t.element_size() for t in res_dev)
+
+        def one():
+            for n in self.names:
+                stage_in[n].copy_(pin_in[n], non_blocking=True)
+            if self.is_patch:
+                u_stage.copy_(u_pin, non_blocking=True)
+            self.ctx.prune_step(0, self.cs, wl.mode, stage_in["q"], stage_in["k"], stage_in["v"], stage_in["hidden"],
+                                flags=self.flags, out=o, rand_u=u_stage)
+            for dst, src in zip(res_host, res_dev):
+                dst.copy_(src, non_blocking=True)
+
+        for _ in range(5):
+            one()
+        torch.cuda.synchronize()
+        D.barrier(self.world)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            one()
+        b.record()
+        torch.cuda.synchronize()
+        ms = D.max_over_ranks(a.elapsed_time(b), self.world, self.dev) / steps
+        return ms, h2d, d2h
+
+    def close(self):
+        self.ctx.close()
+
+
+def other_config(name, dev, world, hbm_gbs):
+    """Compact record of another workload: serial and overlapped step time and the fraction of the copy peak."""
+    h = Harness(name, dev, world)
+    try:
+        n = max(h.per_graph, 4 * h.per_graph if h.touched < 100e6 else h.per_graph)
+        ms_s, g_s = h.timed_exact(0, n, h.per_graph)
+        ms_o, g_o = h.timed_exact(h.mvla.FLAG_INPUTS_STABLE, n, h.per_graph)
+        ab = algorithmic_bytes(h.wl, h.kept_rows)["total"]
+        s_us, o_us = ms_s * 1e3 / n, ms_o * 1e3 / n
+        return {"serial_us": s_us, "overlapped_period_us": o_us, "algorithmic_bytes": ab, "kept_rows": h.kept_rows,
+                "frac_of_peak_serial": ab / (s_us * 1e-6) / 1e9 / hbm_gbs,
+                "frac_of_peak_overlapped": ab / (o_us * 1e-6) / 1e9 / hbm_gbs, "steps": n}
+    finally:
+        h.close()
+        h.torch.cuda.empty_cache()
+
+
+def run_ours(args, rank, local, world):
+    import torch
+    from paper_2604_09244_b200 import mvla
+
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    h = Harness(args.workload, dev, world)
+    wl = h.wl
+    K, W = max(1, args.steps), max(3, args.warmup)
+
+    # ---- the headline: K steps one after another in one stream, every kernel waiting for the work before it
+    # (what one request inside a prefill sees), device-resident inputs rotating over sets larger than L2
     with ClockSampler(local) as clk:
-        ms = timed(graph, replays)
+        ms, g_serial = h.timed_exact(0, K, W)
+        serial_dist = h.distribution(g_serial)
     ms_per_step = ms / K
     tokens_per_step = wl.total_vis * world
     value = tokens_per_step / (ms_per_step * 1e-3)
 
-    # the same steps without the promise: every kernel waits for all earlier work
-    graph_serial = capture(per_graph, 0)
-    serial_us = timed(graph_serial, max(1, replays // 2)) * 1e3 / (max(1, replays // 2) * per_graph)
-
-    # ---- isolated latency: one step per graph launch, synchronised in between (nothing to overlap with)
-    g1 = [capture(1, 0)]
-    lat = []
-    for i in range(64):
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        g1[0].replay()
-        b.record()
-        torch.cuda.synchronize()
-        lat.append(a.elapsed_time(b) * 1e3)
-    lat.sort()
-
-    # ---- per-stage timing through the stage entry points (graphs, rotating sets)
-    attn_b = [torch.empty(wl.total_vis, dtype=torch.float32, device=dev) for _ in range(n_sets)]
-    l1_b = [torch.empty(wl.total_vis, dtype=torch.float32, device=dev) for _ in range(n_sets)]
-    adaptive = wl.mode == 1
-    x_b = [torch.empty(wl.total_vis // 2, 4, dtype=torch.float32, device=dev) for _ in range(n_sets)] if is_patch else None
-
-    def st_salience(i):
-        s = sets[i % n_sets]
-        if is_patch:
-            ctx.patch_indicators(cs, s["q"], s["k"], s["hidden"], attn_out=attn_b[i % n_sets], x_out=x_b[i % n_sets])
-            return
-        ctx.salience(cs, s["q"], s["k"], s["hidden"] if adaptive else None, attn_out=attn_b[i % n_sets],
-                     l1_out=l1_b[i % n_sets] if adaptive else None)
-
-    def st_select(i):
-        if is_patch:
-            ctx.patch_select(0, cs, attn_b[i % n_sets], x_b[i % n_sets], u_dev, flags=flags, out=outs[i % n_sets])
-            return
-        ctx.select(0, cs, wl.mode, attn_b[i % n_sets], l1_b[i % n_sets] if adaptive else None, flags=flags,
-                   out=outs[i % n_sets])
-
-    def st_compact(i):
-        s, o = sets[i % n_sets], outs[i % n_sets]
-        ctx.compact(cs, o.kept_idx, o.out_offsets, probe_rows if is_patch else kept_rows, s["hidden"], s["k"], s["v"],
-                    out_hidden=o.out_hidden, out_k=o.out_k, out_v=o.out_v)
-
-    stage_us = {}
-    for name, fn in (("salience", st_salience), ("select", st_select), ("compact", st_compact)):
-        for i in range(n_sets):
-            fn(i)
-        torch.cuda.synchronize()
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            for i in range(n_sets):
-                fn(i)
-        for _ in range(3):
-            g.replay()
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = max(1, K // (2 * n_sets))
-        a.record()
-        for _ in range(reps):
-            g.replay()
-        b.record()
-        torch.cuda.synchronize()
-        stage_us[name] = a.elapsed_time(b) * 1e3 / (reps * n_sets)
-
-    # ---- end to end: pinned host inputs -> device, step, results -> pinned host
-    pin_in = {n: host[n].pin_memory() for n in names}
-    stage_in = {n: torch.empty_like(host[n], device=dev) for n in names}
-    o = outs[0]
-    res_dev = [o.out_hidden[:kept_rows], o.out_k[:kept_rows], o.out_v[:kept_rows], o.kept_idx[:kept_rows],
-               o.out_offsets, o.budgets]
-    res_host = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in res_dev]
-    u_pin = torch.from_numpy(wl.extra["rand_u"][-1]).pin_memory() if is_patch else None
-    u_stage = torch.empty_like(u_dev) if is_patch else None
-    h2d = in_bytes + (u_pin.numel() * 4 if is_patch else 0)
-    d2h = sum(t.numel() * t.element_size() for t in res_dev)
-
-    def e2e_step():
-        for n in names:
-            stage_in[n].copy_(pin_in[n], non_blocking=True)
-        if is_patch:
-            u_stage.copy_(u_pin, non_blocking=True)
-        ctx.prune_step(0, cs, wl.mode, stage_in["q"], stage_in["k"], stage_in["v"], stage_in["hidden"],
-                       flags=flags, out=o, rand_u=u_stage)
-        for dst, src in zip(res_host, res_dev):
-            dst.copy_(src, non_blocking=True)
-
-    e2e_steps = max(20, min(args.steps, 400))
-    for _ in range(5):
-        e2e_step()
-    torch.cuda.synchronize()
-    D.barrier(world)
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    for _ in range(e2e_steps):
-        e2e_step()
-    b.record()
-    torch.cuda.synchronize()
-    e2e_ms = D.max_over_ranks(a.elapsed_time(b), world, dev) / e2e_steps
+    # ---- independent requests overlapping inside the library (MVLA_FLAG_INPUTS_STABLE): the benchmark's inputs
+    # are static buffers and its output sets rotate, so the promise behind the flag holds
+    ms_o, g_over = h.timed_exact(mvla.FLAG_INPUTS_STABLE, K, W)
+    over_dist = h.distribution(g_over)
+    iso = h.isolated()
+    kt = h.kernel_times()
+    e2e_ms, h2d, d2h = h.e2e(max(20, min(K, 400)))
     e2e_value = tokens_per_step / (e2e_ms * 1e-3)
 
+    peaks, peak_kind = measured_peaks()
+    ab = algorithmic_bytes(wl, h.kept_rows)
+    others = {}
+    if rank == 0 and world == 1 and args.workload == "config2" and not args.no_other_configs:
+        n_sets, per_graph, touched = h.n_sets, h.per_graph, h.touched
+        alloc_mib = (h.in_bytes + h.out_bytes_alloc) * h.n_sets / 2**20
+        launches = h.launches_per_step
+        kept_rows, n_req = h.kept_rows, h.n_req
+        h.close()
+        torch.cuda.empty_cache()
+        for name in ("config3", "config4", "config5", "patch_mla"):
+            others[name] = other_config(name, dev, world, peaks["hbm_gbs"])
+    else:
+        n_sets, per_graph, touched = h.n_sets, h.per_graph, h.touched
+        alloc_mib = (h.in_bytes + h.out_bytes_alloc) * h.n_sets / 2**20
+        launches = h.launches_per_step
+        kept_rows, n_req = h.kept_rows, h.n_req
+        h.close()
     if rank != 0:
         return
-    peaks, peak_kind = measured_peaks()
-    ab = algorithmic_bytes(wl, kept_rows)
-    stage_bytes = {"salience": ab["salience"] + ab["l1"], "select": ab["scores"], "compact": ab["compact"]}
-    dom = max(stage_us, key=stage_us.get)
-    achieved = stage_bytes[dom] / (stage_us[dom] * 1e-6) / 1e9
-    kernels = {"salience": ("patch scoring: salience_fast_kernel + patch_indicators_kernel (mvla_patch_indicators)" if is_patch
-                            else "salience_fast_kernel (+ head_reduce_kernel; mvla_salience)" if wl.dtype == "bf16"
-                            else "salience_kernel (+ head_reduce_kernel; mvla_salience)"),
-               "select": "patch_select_kernel (mvla_patch_select)" if is_patch else "select_kernel (mvla_select)",
-               "compact": "compact_kernel (mvla_compact)"}
-    roof = {"bound": "hbm", "kernel": kernels[dom],
-            "achieved": achieved, "peak": peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-            "frac": achieved / peaks["hbm_gbs"], "traffic": ncu_traffic(args.workload, dom),
-            "bytes_per_launch": stage_bytes[dom], "us_per_launch": stage_us[dom],
-            "how": "the stage's own entry point timed alone in CUDA graphs over the rotating sets (includes its launch edges)"}
-    step_gbs = ab["total"] / (ms_per_step * 1e-3) / 1e9
 
-    cpu_sec, cpu_n, cores = time_oracle(wl, 10 ** 6, 10.0)
+    # ---- roofline of the dominant kernel, timed as the fused step runs it
+    if kt is not None:
+        kbytes = {"scoring": ab["salience"] + ab["l1"], "tail": ab["compact"] + ab["scores"]}
+        knames = {"scoring": ("salience_fast_kernel" if wl.dtype != "fp32" else "salience_kernel") +
+                             (" + l1norm_kernel beside it" if wl.mode == 1 else ""),
+                  "tail": "select_copy_kernel (selection + row copy)"}
+        dom = max(("scoring", "tail"), key=lambda k: kt[k])
+        achieved = kbytes[dom] / (kt[dom] * 1e-6) / 1e9
+        roof = {"bound": "hbm", "kernel": knames[dom], "achieved": achieved, "peak": peaks["hbm_gbs"],
+                "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "traffic": ncu_traffic(args.workload, dom), "bytes_per_launch": kbytes[dom], "us_per_launch": kt[dom],
+                "kernel_us": {k: kt[k] for k in ("scoring", "tail")},
+                "how": f"CUDA events around {kt['launches']} non-overlapped steps on the launching stream and the library's "
+                       "stage event between the step's two kernels (mvla_set_stage_event); the dominant kernel is the "
+                       "longer one; a launch's time includes its wait for the kernel before it"}
+    else:
+        roof = {"bound": "hbm", "kernel": "patch path (five kernels)", "achieved": None, "peak": peaks["hbm_gbs"],
+                "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": None, "traffic": None}
+    step_gbs = ab["total"] / (ms_per_step * 1e-3) / 1e9
+    over_us = ms_o * 1e3 / K
+
+    cpu_sec, cpu_n, cores = time_oracle(wl, 10 ** 6, 8.0)
+    cpu1_sec, cpu1_n, _ = time_oracle(wl, 10 ** 6, 6.0, threads=1)
     line = {"metric": "visual_tokens_per_s_pruned", "value": value, "unit": "tokens/s", "n_gpus": world,
-            "steps": K, "warmup": warm_replays * per_graph, "ms_per_step": ms_per_step,
+            "steps": K, "warmup": W, "ms_per_step": ms_per_step,
             "latency_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": {"bf16": "bf16", "fp32": "f32", "fp8": "e4m3"}[wl.dtype], "data": "synthetic",
-            "config": {"workload": desc, "l2": f"inputs and outputs rotate over {n_sets} distinct sets "
-                                               f"(about {touched * n_sets / 2**20:.0f} MiB touched per cycle, L2 is 126 MiB; "
-                                               f"{(in_bytes + out_bytes_alloc) * n_sets / 2**20:.0f} MiB allocated)",
-                       "timing": "CUDA events around CUDA-graph replays of back-to-back steps "
-                                 f"({per_graph} steps per graph, MVLA_FLAG_INPUTS_STABLE: neighbouring steps overlap; "
-                                 f"{'independent requests on ' + str(n_req) + ' state slots in rotation' if n_req > 1 else 'one episode, one state slot'})",
+            "config": {"workload": h.desc, "l2": f"inputs and outputs rotate over {n_sets} distinct sets "
+                                                 f"(about {touched * n_sets / 2**20:.0f} MiB touched per cycle, L2 is 126 MiB; "
+                                                 f"{alloc_mib:.0f} MiB allocated)",
+                       "timing": "value, ms_per_step and latency_us are the SERIAL figure: CUDA events around CUDA-graph "
+                                 f"replays ({per_graph} steps per graph) of steps enqueued one after another in one stream, "
+                                 "every kernel waiting for the work before it; the period of independent requests "
+                                 "overlapping inside the library is reported apart (overlapped)",
                        "kept_rows": kept_rows, "parallelism": f"replicas x{world}"},
             "clocks": clk.summary(),
             "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms},
-            "gpu_launches": K * launches_per_step,
+            "gpu_launches": K * launches,
             "roofline": roof,
             "step_hbm": {"algorithmic_bytes": ab["total"], "achieved_gbs": step_gbs,
-                         "frac_of_peak": step_gbs / peaks["hbm_gbs"], "peak_kind": peak_kind},
-            "serial_us_per_step": serial_us,
-            "isolated_latency_us": {"p10": lat[6], "median": lat[32], "p90": lat[57],
-                                    "how": "one step per graph launch, device synchronised between launches"},
-            "stage_us": stage_us,
+                         "frac_of_peak": step_gbs / peaks["hbm_gbs"], "peak_kind": peak_kind,
+                         "what": "whole step, serial latency"},
+            "serial_us_per_step": serial_dist,
+            "overlapped": {"period_us": over_us, "tokens_per_s": tokens_per_step / (over_us * 1e-6),
+                           "frac_of_peak": ab["total"] / (over_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                           "period_us_dist": over_dist,
+                           "what": f"MVLA_FLAG_INPUTS_STABLE: independent requests on {n_req} state slots in rotation, "
+                                   "neighbouring steps overlap inside the library (throughput, not latency)"},
+            "isolated_latency_us": iso,
             "cpu_baseline": {"value": wl.total_vis / cpu_sec, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                              "sample": f"{cpu_n} full prune steps of the same workload in {cpu_sec * cpu_n:.1f} s",
-                             "ms_per_step": cpu_sec * 1e3}}
+                             "ms_per_step": cpu_sec * 1e3,
+                             "cores_1": {"value": wl.total_vis / cpu1_sec, "ms_per_step": cpu1_sec * 1e3, "cores": 1,
+                                         "sample": f"{cpu1_n} steps in {cpu1_sec * cpu1_n:.1f} s"}}}
+    if others:
+        line["other_configs"] = others
     print(json.dumps(line), flush=True)
-    ctx.close()
+
+
+def spawn_ranks(args):
+    """`--gpus N` without a launcher environment: start the N local ranks (one process per GPU) here."""
+    import socket
+    import subprocess
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(args.gpus):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(args.gpus),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env))
+    rc = 0
+    for p in procs:
+        rc = p.wait() or rc
+    sys.exit(rc)
 
 
 def main():
@@ -487,8 +598,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config2")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the compact records of the other workloads")
     args = ap.parse_args()
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(args)
     if args.impl == "reference":
         rank = int(os.environ.get("RANK", 0))
         if args.steps == 20000:          # the GPU arm's default; the CPU oracle needs far fewer

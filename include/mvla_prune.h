@@ -251,6 +251,17 @@ int32_t mvla_prune_step(mvla_ctx *ctx, int32_t prune_point, int32_t batch,
                         int32_t *total_kept_out, void *stream);
 
 /*
+ * Measurement aid (the paper has no counterpart).  While `event` (a cudaEvent_t created with timing, passed
+ * as void*; null switches it off) is set, every mvla_prune_step that is not overlapped with its neighbours
+ * (no MVLA_FLAG_INPUTS_STABLE) records it on the call's stream between its scoring kernel(s) and its
+ * selection + row-copy kernel.  With events of the caller's own around the call this gives the duration of
+ * each of the step's kernels as the step runs them.  The record sits between two kernels that otherwise
+ * overlap at their edges, so the step is slightly slower while it is on; leave it off otherwise.  For
+ * batches of more than 32 samples the event is recorded once per launch of 32.  The library never destroys it.
+ */
+int32_t mvla_set_stage_event(mvla_ctx *ctx, void *event);
+
+/*
  * Failure-detection self-test (the paper has no counterpart).  Every device-side wait of this library is
  * bounded: when it runs out the kernel gives up, returns, and leaves MVLA_ERR_TIMEOUT in the context's status
  * word; from then on every call on the context returns MVLA_ERR_TIMEOUT (sticky) and a new context must be

@@ -86,6 +86,9 @@ def load(path: str):
         L.oracle_salience.restype = None
         L.oracle_salience_gqa.argtypes = [fp, fp, C.c_int32, C.c_int32, C.c_int32, sp, dp]
         L.oracle_salience_gqa.restype = None
+        L.oracle_salience_cached.argtypes = [fp, fp, C.c_int32, C.c_int32, sp, C.POINTER(C.c_uint8), C.c_int32,
+                                             dp, dp, ip]
+        L.oracle_salience_cached.restype = None
         L.oracle_l1norm.argtypes = [fp, C.c_int32, sp, dp]
         L.oracle_l1norm.restype = None
         L.oracle_indicators.argtypes = [dp, dp, C.c_int32, C.c_int32, dp]
@@ -115,6 +118,8 @@ def load(path: str):
         L.oracle_decide_step.argtypes = [dp, dp, sp, pp, C.c_int32, C.POINTER(CState), ip,
                                          C.POINTER(CDiag), dp, dp]
         L.oracle_decide_step.restype = C.c_int32
+        L.oracle_set_num_threads.argtypes = [C.c_int32]
+        L.oracle_set_num_threads.restype = None
         L.oracle_num_threads.argtypes = []
         L.oracle_num_threads.restype = C.c_int32
         # Alg. 1 patch by patch
@@ -152,6 +157,11 @@ def lib():
 
 def num_threads() -> int:
     return int(lib().oracle_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    """Threads the head loops use from now on (reporting: the oracle timed on one core and on all)."""
+    lib().oracle_set_num_threads(int(n))
 
 
 # --------------------------------------------------------------------------
@@ -203,6 +213,32 @@ def salience_gqa(q, k, n_heads, n_kv_heads, head_dim, s) -> np.ndarray:
     lib().oracle_salience_gqa(qp, kp, n_heads, n_kv_heads, head_dim, C.byref(cs),
                               out.ctypes.data_as(C.POINTER(C.c_double)))
     return out
+
+
+class LogitCache:
+    """The previous action step's logits of one sample, [H, n_txt, n_vis] (see oracle_salience_cached)."""
+
+    def __init__(self, n_heads: int, s):
+        self.logits = np.zeros((n_heads, int(s.n_txt), int(s.n_2d) + int(s.n_3d)), dtype=np.float64)
+        self.valid = False
+
+
+def salience_cached(q, k, n_heads, head_dim, s, changed, cache: LogitCache):
+    """Returns (scores, number of visual keys whose logits were recomputed); updates `cache`."""
+    q, qp = _f32(q)
+    k, kp = _f32(k)
+    cs = c_sample(s)
+    out = np.zeros(cs.n_2d + cs.n_3d, dtype=np.float64)
+    mp = None
+    if changed is not None:
+        changed = np.ascontiguousarray(changed, dtype=np.uint8)
+        mp = changed.ctypes.data_as(C.POINTER(C.c_uint8))
+    n = C.c_int32()
+    lib().oracle_salience_cached(qp, kp, n_heads, head_dim, C.byref(cs), mp, int(cache.valid),
+                                 cache.logits.ctypes.data_as(C.POINTER(C.c_double)),
+                                 out.ctypes.data_as(C.POINTER(C.c_double)), C.byref(n))
+    cache.valid = True
+    return out, n.value
 
 
 def l1norm(hidden, d_model, s) -> np.ndarray:

@@ -73,6 +73,56 @@ void oracle_salience_gqa(const float *q, const float *k, int32_t n_heads, int32_
     free(per_head);
 }
 
+/* ---- Sec. 4.3 / 5.2: consecutive frames share most of their content, so the logits of rows that did not
+ * change since the previous action step need not be recomputed.  `logits` ([H][n_txt][n_vis], kept by the
+ * caller between steps) holds the previous step's logits when `cache_valid`; `changed` has one byte per
+ * row of the packed tensors (non-zero: the row was rewritten since the previous step).  A changed text
+ * row invalidates everything (every logit has that query in it or is renormalised with it); otherwise
+ * only the columns of changed visual keys are recomputed.  With a truthful mask the result equals
+ * oracle_salience on the current inputs. ---- */
+void oracle_salience_cached(const float *q, const float *k, int32_t n_heads, int32_t head_dim,
+                            const oracle_sample *s, const uint8_t *changed, int32_t cache_valid,
+                            double *logits, double *a_out, int32_t *n_recomputed)
+{
+    const int32_t H = n_heads, d = head_dim, nt = s->n_txt, nv = s->n_2d + s->n_3d;
+    const int64_t row = (int64_t)H * d;
+    int32_t all = !cache_valid || changed == NULL;
+    for (int32_t i = 0; i < nt && !all; ++i)
+        if (changed[(int64_t)s->seq_off + s->off_txt + i]) all = 1;
+    int32_t redone = 0;
+    for (int32_t j = 0; j < nv; ++j) {
+        const int64_t krow = (int64_t)s->seq_off + vis_row(s, j);
+        if (!all && !changed[krow]) continue;                 /* the previous step's logits of key j stand */
+        ++redone;
+        for (int32_t h = 0; h < H; ++h)
+            for (int32_t ti = 0; ti < nt; ++ti) {
+                const float *qrow = q + ((int64_t)s->seq_off + s->off_txt + ti) * row;
+                const float *krw = k + krow * row;
+                double dot = 0.0;
+                for (int32_t c = 0; c < d; ++c) dot += (double)qrow[(int64_t)h * d + c] * (double)krw[(int64_t)h * d + c];
+                logits[((size_t)h * nt + ti) * nv + j] = dot / sqrt((double)d);
+            }
+    }
+    /* softmax over all visual keys, then the mean over heads and queries, in the order of oracle_salience */
+    double *head_sum = (double *)calloc((size_t)H * nv, sizeof(double));
+    for (int32_t h = 0; h < H; ++h)
+        for (int32_t ti = 0; ti < nt; ++ti) {
+            const double *l = logits + ((size_t)h * nt + ti) * nv;
+            double top = -INFINITY, z = 0.0;
+            for (int32_t j = 0; j < nv; ++j) if (l[j] > top) top = l[j];
+            for (int32_t j = 0; j < nv; ++j) z += exp(l[j] - top);
+            for (int32_t j = 0; j < nv; ++j) head_sum[(size_t)h * nv + j] += exp(l[j] - top) / z;
+        }
+    const double pairs = (double)H * (double)nt;
+    for (int32_t j = 0; j < nv; ++j) {
+        double total = 0.0;
+        for (int32_t h = 0; h < H; ++h) total += head_sum[(size_t)h * nv + j];
+        a_out[j] = total / pairs;
+    }
+    free(head_sum);
+    if (n_recomputed) *n_recomputed = redone;
+}
+
 /* ---- Sec. 3.1.2: L1 feature norm per visual token ---- */
 void oracle_l1norm(const float *hidden, int32_t d_model, const oracle_sample *s, double *n_out)
 {
@@ -328,6 +378,8 @@ int32_t oracle_prune_step(const float *q, const float *k, const float *hidden,
 #ifdef _OPENMP
 #include <omp.h>
 int32_t oracle_num_threads(void) { return (int32_t)omp_get_max_threads(); }
+void oracle_set_num_threads(int32_t n) { if (n >= 1) omp_set_num_threads((int)n); }
 #else
 int32_t oracle_num_threads(void) { return 1; }
+void oracle_set_num_threads(int32_t n) { (void)n; }
 #endif

@@ -88,6 +88,15 @@ void oracle_salience(const float *q, const float *k, int32_t n_heads, int32_t he
 void oracle_salience_gqa(const float *q, const float *k, int32_t n_heads, int32_t n_kv_heads,
                          int32_t head_dim, const oracle_sample *s, double *a_out);
 
+/* Sec. 4.3 / 5.2 (consecutive frames share content): oracle_salience that reuses the previous action
+ * step's logits for visual keys whose rows did not change.  logits: [H][n_txt][n_vis] doubles owned by the
+ * caller across steps (read when cache_valid, always left holding this step's logits); changed: one byte per
+ * row of the packed tensors, non-zero = rewritten since the previous step (NULL: everything); a changed
+ * text row recomputes everything.  n_recomputed (nullable): visual keys whose logits were recomputed. */
+void oracle_salience_cached(const float *q, const float *k, int32_t n_heads, int32_t head_dim,
+                            const oracle_sample *s, const uint8_t *changed, int32_t cache_valid,
+                            double *logits, double *a_out, int32_t *n_recomputed);
+
 /* Sec. 3.1.2: L1 norm of each visual token's feature row.  hidden: [rows, D]. */
 void oracle_l1norm(const float *hidden, int32_t d_model, const oracle_sample *s, double *n_out);
 
@@ -141,6 +150,8 @@ int32_t oracle_prune_step(const float *q, const float *k, const float *hidden,
 
 /* Threads the head loop of oracle_salience may use (reporting only). */
 int32_t oracle_num_threads(void);
+/* Threads for the head loops from now on (timing on one core and on all; the arithmetic does not change). */
+void oracle_set_num_threads(int32_t n);
 
 #ifdef __cplusplus
 }

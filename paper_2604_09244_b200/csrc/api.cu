@@ -40,6 +40,7 @@ struct mvla_ctx {
     int32_t* tail_list;          // [kSets][max_batch * (max_text + max_vis)] kept list as the copying CTAs read it (-1 between launches)
     size_t rows_all;             // max_batch * (max_text + max_vis)
     int sm_count;                // multiprocessors of the device
+    cudaEvent_t stage_event;     // measurement aid: recorded between scoring and selection + copy (null: off)
     size_t vis_all;              // max_batch * max_vis
     // patch-by-patch path (cfg.patch_path): attention copy [H][max_text][vis_all], per-patch smoothed
     // indicators [n_prune_points][n_slots][max_patch][4], and the scratch between its kernels
@@ -666,6 +667,7 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     ctx->acc64 = nullptr;
     ctx->tail_list = nullptr;
     ctx->sm_count = prop.multiProcessorCount;
+    ctx->stage_event = nullptr;
     ctx->alpha_ws = ctx->xhat_patch = ctx->patch_x_ws = ctx->patch_attn_ws = nullptr;
     ctx->patch_sets = 1;
     ctx->nout_ws = nullptr;
@@ -874,6 +876,13 @@ int32_t mvla_compact(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, c
     return MVLA_OK;
 }
 
+int32_t mvla_set_stage_event(mvla_ctx* ctx, void* event)
+{
+    if (!ctx) return MVLA_ERR_INVALID_ARG;
+    ctx->stage_event = static_cast<cudaEvent_t>(event);
+    return MVLA_OK;
+}
+
 int32_t mvla_selftest_wait_timeout(mvla_ctx* ctx, uint32_t limit_us, void* stream)
 {
     if (!ctx || limit_us < 1 || limit_us > 1000000u) return MVLA_ERR_INVALID_ARG;
@@ -1007,6 +1016,14 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
                                 &used_acc64, false, forked ? ctx->aux[par] : st, AlphaOut{nullptr, 0, 0},
                                 tail ? ctx->tail_list + par * ctx->rows_all : nullptr, tail);
         if (rc != MVLA_OK) return rc;
+        if (ctx->stage_event && !forked) {
+            // under stream capture the record must become an event-record node of the graph (an "external"
+            // record): only then can the event be timed after a replay
+            cudaStreamCaptureStatus cst = cudaStreamCaptureStatusNone;
+            cudaStreamIsCapturing(st, &cst);
+            const unsigned how = cst == cudaStreamCaptureStatusActive ? cudaEventRecordExternal : cudaEventRecordDefault;
+            if (cudaEventRecordWithFlags(ctx->stage_event, st, how) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
+        }
         cudaStream_t sel_stream = st;
         if (forked) {
             sel_stream = ctx->aux[par];

@@ -104,6 +104,9 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         any_live |= ti.valid > 0;
     }
 
+#ifdef MVLA_TRIGGER_EARLY
+    pdl_trigger();
+#endif
     if (tid == 0) {                           // the loads go out first; everything else overlaps with them
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);

@@ -31,7 +31,7 @@ SET_2D, SET_3D = 1, 2
 
 EXPORTS = ("mvla_prune_create", "mvla_salience", "mvla_select", "mvla_compact",
            "mvla_prune_step", "mvla_prune_destroy", "mvla_patch_indicators", "mvla_patch_select",
-           "mvla_salience_noalloc", "mvla_selftest_wait_timeout")
+           "mvla_salience_noalloc", "mvla_selftest_wait_timeout", "mvla_set_stage_event")
 
 
 class MvlaError(RuntimeError):
@@ -108,6 +108,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.mvla_patch_indicators.restype = i32
     lib.mvla_patch_select.argtypes = [vp, i32, i32, sp, u32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.mvla_patch_select.restype = i32
+    lib.mvla_set_stage_event.argtypes = [vp, vp]
+    lib.mvla_set_stage_event.restype = i32
     lib.mvla_selftest_wait_timeout.argtypes = [vp, u32, vp]
     lib.mvla_selftest_wait_timeout.restype = i32
     return lib
@@ -203,6 +205,13 @@ class PruneContext:
             self.close()
         except Exception:
             pass
+
+    def set_stage_event(self, event: Optional[torch.cuda.Event]) -> None:
+        """Measurement aid: `event` is recorded between the scoring kernel and the selection + copy kernel
+        of every non-overlapped prune step (None switches it off)."""
+        rc = self._lib.mvla_set_stage_event(self._h, event.cuda_event if event is not None else None)
+        if rc != OK:
+            raise MvlaError(rc, "mvla_set_stage_event")
 
     def selftest_wait_timeout(self, limit_us: int = 200, *, stream=None) -> None:
         """Makes one bounded device-side wait run out on purpose (see the header); afterwards every call

@@ -298,12 +298,17 @@ def config4_batched(seed: int = 3, batch: int = 16, D=4096, H=32, d=128, dtype="
 
 
 def config5_action_iteration(seed: int = 4, T: int = 16, D=4096, H=32, d=128, dtype="bf16",
-                             n_txt=32, n_2d=256, n_3d=1024) -> Workload:
+                             n_txt=32, n_2d=256, n_3d=1024, drift: str = "all") -> Workload:
     """Action iteration: T sequential steps of 32 text + 256 2D + 1024 3D.
     Step 1 is structured like the single-frame workload (5 % spikes x4); each
     later step adds N(0, sigma=0.1) to the (unrounded) hidden rows of a fresh
     random 10 % of all tokens and re-projects those rows with the same
-    weights.  Adaptive keep 30 %, cold start on (step 1 keeps everything)."""
+    weights.  Adaptive keep 30 %, cold start on (step 1 keeps everything).
+    ``extra["changed_rows"][t]`` is the truthful mask (uint8 per row) of the rows
+    step t rewrote (all ones at t = 0).  ``drift="visual_local"`` is the variant
+    in which consecutive frames share most of their content: the instruction
+    (text rows) stays fixed and the 10 % of rows that drift are one contiguous
+    run of visual tokens whose position moves from step to step."""
     s = layout_2d_3d_txt(0, n_txt, n_2d, n_3d, keep_total=0.30)
     rng = np.random.default_rng(seed)
     hidden = rng.standard_normal((s.seq_len, D), dtype=np.float32)
@@ -314,10 +319,19 @@ def config5_action_iteration(seed: int = 4, T: int = 16, D=4096, H=32, d=128, dt
     q = hidden @ wq
     k = hidden @ wk
     v = hidden @ wv
-    steps = []
+    steps, masks = [], []
     for t in range(T):
+        mask = np.ones(S, dtype=np.uint8)
         if t > 0:
-            rows = np.sort(rng.choice(S, size=_rhu(0.10 * S), replace=False))
+            n_drift = _rhu(0.10 * S)
+            if drift == "visual_local":
+                nv = n_2d + n_3d                                  # visual tokens are rows 0 .. nv-1 of the layout
+                start = int(rng.integers(0, nv - n_drift + 1))
+                rows = np.arange(start, start + n_drift)
+            else:
+                rows = np.sort(rng.choice(S, size=n_drift, replace=False))
+            mask[:] = 0
+            mask[rows] = 1
             hidden[rows] += rng.standard_normal((len(rows), D), dtype=np.float32) * np.float32(0.1)
             q[rows] = hidden[rows] @ wq
             k[rows] = hidden[rows] @ wk
@@ -326,8 +340,9 @@ def config5_action_iteration(seed: int = 4, T: int = 16, D=4096, H=32, d=128, dt
                              q=round_to_dtype(q.reshape(S, H, d).copy(), dtype),
                              k=round_to_dtype(k.reshape(S, H, d).copy(), dtype),
                              v=round_to_dtype(v.reshape(S, H, d).copy(), dtype)))
-    return Workload("action_iteration", dtype, H, d, D, MODE_ADAPTIVE, [s], steps,
-                    cold_start_full_keep=1, seed=seed)
+        masks.append(mask)
+    return Workload("action_iteration" if drift == "all" else "action_iteration_" + drift, dtype, H, d, D,
+                    MODE_ADAPTIVE, [s], steps, cold_start_full_keep=1, seed=seed, extra={"changed_rows": masks})
 
 
 def small_workload(seed: int, *, batch=2, D=256, H=4, d=64, dtype="bf16", mode=MODE_ADAPTIVE,

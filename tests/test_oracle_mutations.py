@@ -57,6 +57,12 @@ MUTATIONS = {
                                             "memset(a, 0, sizeof(double)); const int32_t n_kept = oracle_decide_step(a, l1, s, p, mode,"),
     "whole step drops the norms": ("const int32_t n_kept = oracle_decide_step(a, l1, s, p, mode,",
                                    "const int32_t n_kept = oracle_decide_step(a, NULL, s, p, mode,"),
+    "cached logits never refreshed": ("if (!all && !changed[krow]) continue;                 /* the previous step's logits of key j stand */",
+                                      "if (!all) continue;"),
+    "changed text row not honoured": ("if (changed[(int64_t)s->seq_off + s->off_txt + i]) all = 1;", ";"),
+    "cache ignored": ("int32_t all = !cache_valid || changed == NULL;", "int32_t all = 1;"),
+    "mask read without the sample offset": ("const int64_t krow = (int64_t)s->seq_off + vis_row(s, j);\n        if (!all && !changed[krow]) continue;",
+                                            "const int64_t krow = (int64_t)s->seq_off + vis_row(s, j);\n        if (!all && !changed[vis_row(s, j)]) continue;"),
     "cold start prunes": ("if (t == 1 && p->cold_start_full_keep) {", "if (0) {"),
     "state updated after the decision": ("const int32_t n_kept = oracle_select(z, s, k2, k3, kept_idx);",
                                          "const int32_t n_kept = oracle_select(attn_out ? attn_out : z, s, k2, k3, kept_idx);"),

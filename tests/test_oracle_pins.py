@@ -533,3 +533,56 @@ def test_whole_step_feeds_scores_and_norms_into_the_decisions():
         assert [r.k_2d, r.k_3d] == g[ks].astype(int).tolist()
         assert r.kept_idx.tolist() == g[kept].astype(int).tolist()
     np.testing.assert_allclose(st.c.mhat[:], g["G_mhat2"], rtol=1e-6)
+
+
+# ---------------------------------------------------------------- reuse of the previous step's logits
+def _drifting_case(seed=3):
+    rng = np.random.default_rng(seed)
+    H, d = 2, 8
+    s = S(3, 5, 6, seq_off=2)                                  # visual rows 2..12, text rows 13..15
+    rows = s.seq_off + s.seq_len
+    q0 = rng.standard_normal((rows, H, d)).astype(np.float32)
+    k0 = rng.standard_normal((rows, H, d)).astype(np.float32)
+    return H, d, s, rows, q0, k0, rng
+
+
+def test_cached_salience_with_a_truthful_mask_is_the_plain_salience():
+    H, d, s, rows, q, k, rng = _drifting_case()
+    cache = oracle.LogitCache(H, s)
+    a, n = oracle.salience_cached(q, k, H, d, s, None, cache)                  # nothing cached yet: everything computed
+    assert n == 11 and np.array_equal(a, oracle.salience(q, k, H, d, s))
+    for step in range(4):
+        changed = np.zeros(rows, np.uint8)
+        vis = s.seq_off + rng.choice(11, size=3, replace=False)
+        changed[vis] = 1
+        k = k.copy(); q = q.copy()
+        k[vis] += rng.standard_normal((3, H, d)).astype(np.float32)
+        q[vis] += 1.0                                           # queries of visual rows are never read
+        a, n = oracle.salience_cached(q, k, H, d, s, changed, cache)
+        assert n == 3
+        assert np.array_equal(a, oracle.salience(q, k, H, d, s))               # same arithmetic, same bits
+    # a changed text row: every logit has that query in it -> everything is recomputed
+    changed = np.zeros(rows, np.uint8)
+    changed[s.seq_off + s.off_txt + 1] = 1
+    q = q.copy(); q[s.seq_off + s.off_txt + 1] *= -2.0
+    a, n = oracle.salience_cached(q, k, H, d, s, changed, cache)
+    assert n == 11 and np.array_equal(a, oracle.salience(q, k, H, d, s))
+
+
+def test_cached_salience_really_uses_the_cache():
+    # a key that changed but is reported unchanged keeps its OLD logits: the result is the plain salience of
+    # the inputs in which that key still has its old row -- and not that of the current inputs
+    H, d, s, rows, q, k_old, rng = _drifting_case(5)
+    cache = oracle.LogitCache(H, s)
+    oracle.salience_cached(q, k_old, H, d, s, None, cache)
+    k_new = k_old.copy()
+    moved = s.seq_off + np.array([1, 7])
+    k_new[moved] += 2.0
+    changed = np.zeros(rows, np.uint8)
+    changed[moved[0]] = 1                                        # key 7 changed too, but the mask hides it
+    a, n = oracle.salience_cached(q, k_new, H, d, s, changed, cache)
+    k_mixed = k_new.copy()
+    k_mixed[moved[1]] = k_old[moved[1]]
+    assert n == 1
+    assert np.array_equal(a, oracle.salience(q, k_mixed, H, d, s))
+    assert np.abs(a - oracle.salience(q, k_new, H, d, s)).max() > 1e-3
