@@ -262,6 +262,21 @@ int32_t mvla_prune_step(mvla_ctx *ctx, int32_t prune_point, int32_t batch,
 int32_t mvla_set_stage_event(mvla_ctx *ctx, void *event);
 
 /*
+ * Measurement aid (the paper has no counterpart): time stamps taken by the step's own kernels.  An event
+ * between two kernels of a step removes their overlap and costs microseconds inside a CUDA graph, so it
+ * cannot time them as the step runs them; a handful of stores of the global nanosecond timer can.  While
+ * `device_buffer` (device memory, 2 x 4096 x 2 uint64, zero-filled by the caller; null switches it off) is
+ * set, every non-overlapped mvla_prune_step on shapes the fused kernels cover makes CTA c (linear index,
+ * c < 4096) of its scoring kernel write buffer[0][c][0] = the time it was free to start its loads (its
+ * predecessor complete) and buffer[0][c][1] = the time it ended, and CTA c of its selection + row-copy kernel
+ * the same into buffer[1][c][..] (start: past its wait for the scoring kernel; the selecting CTAs, which come
+ * first, report the time the kept list was written as both).  Entries of CTAs that do not exist stay as they
+ * were.  The pointer is read when the step is enqueued (or captured), so every captured step can have a buffer
+ * of its own.  For batches of more than 32 samples the launches of 32 share the buffer.
+ */
+int32_t mvla_set_kernel_stamps(mvla_ctx *ctx, uint64_t *device_buffer);
+
+/*
  * Failure-detection self-test (the paper has no counterpart).  Every device-side wait of this library is
  * bounded: when it runs out the kernel gives up, returns, and leaves MVLA_ERR_TIMEOUT in the context's status
  * word; from then on every call on the context returns MVLA_ERR_TIMEOUT (sticky) and a new context must be

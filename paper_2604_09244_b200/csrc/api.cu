@@ -41,6 +41,7 @@ struct mvla_ctx {
     size_t rows_all;             // max_batch * (max_text + max_vis)
     int sm_count;                // multiprocessors of the device
     cudaEvent_t stage_event;     // measurement aid: recorded between scoring and selection + copy (null: off)
+    unsigned long long* stamps;  // measurement aid: device buffer [2][kStampSlots][2] of per-CTA time stamps (null: off)
     size_t vis_all;              // max_batch * max_vis
     // patch-by-patch path (cfg.patch_path): attention copy [H][max_text][vis_all], per-patch smoothed
     // indicators [n_prune_points][n_slots][max_patch][4], and the scratch between its kernels
@@ -272,7 +273,7 @@ int32_t check_sticky(mvla_ctx* ctx)
 int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, const void* k, int64_t rows,
                            const void* hidden, float* l1, unsigned long long* acc64, bool* used_acc64,
                            bool free_running, cudaStream_t st, AlphaOut alpha = AlphaOut{nullptr, 0, 0},
-                           int32_t* rearm = nullptr, bool norms_beside = false)
+                           int32_t* rearm = nullptr, bool norms_beside = false, unsigned long long* stamps = nullptr)
 {
     if (used_acc64) *used_acc64 = false;
     const mvla_config& c = ctx->cfg;
@@ -304,7 +305,7 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
         e = launch_salience_fast(bd, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, static_cast<int>(ctx->qk_elem), tq, tk,
                                  tiles_per_cta, cluster, npad,
                                  alpha.ptr && !acc64 ? nullptr : ctx->part,     // the patch path reads the attention copy only
-                                 ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, rearm, st);
+                                 ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, rearm, stamps, st);
         if (used_acc64) *used_acc64 = acc64 != nullptr;
     } else {
         e = launch_salience(bd, c.dtype, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, q, k, tq, tk, ctx->use_umma, tiles_per_cta,
@@ -668,6 +669,7 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     ctx->tail_list = nullptr;
     ctx->sm_count = prop.multiProcessorCount;
     ctx->stage_event = nullptr;
+    ctx->stamps = nullptr;
     ctx->alpha_ws = ctx->xhat_patch = ctx->patch_x_ws = ctx->patch_attn_ws = nullptr;
     ctx->patch_sets = 1;
     ctx->nout_ws = nullptr;
@@ -883,6 +885,13 @@ int32_t mvla_set_stage_event(mvla_ctx* ctx, void* event)
     return MVLA_OK;
 }
 
+int32_t mvla_set_kernel_stamps(mvla_ctx* ctx, uint64_t* device_buffer)
+{
+    if (!ctx || (reinterpret_cast<uintptr_t>(device_buffer) & 7u)) return MVLA_ERR_INVALID_ARG;
+    ctx->stamps = reinterpret_cast<unsigned long long*>(device_buffer);
+    return MVLA_OK;
+}
+
 int32_t mvla_selftest_wait_timeout(mvla_ctx* ctx, uint32_t limit_us, void* stream)
 {
     if (!ctx || limit_us < 1 || limit_us > 1000000u) return MVLA_ERR_INVALID_ARG;
@@ -1014,7 +1023,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         const bool tail = !forked && select_copy_supported(bd);
         rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, l1_ws, acc64,
                                 &used_acc64, false, forked ? ctx->aux[par] : st, AlphaOut{nullptr, 0, 0},
-                                tail ? ctx->tail_list + par * ctx->rows_all : nullptr, tail);
+                                tail ? ctx->tail_list + par * ctx->rows_all : nullptr, tail, tail ? ctx->stamps : nullptr);
         if (rc != MVLA_OK) return rc;
         if (ctx->stage_event && !forked) {
             // under stream capture the record must become an event-record node of the graph (an "external"
@@ -1047,8 +1056,8 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
             const bool copying = (job.src[0] && job.dst[0]) || (job.src[1] && job.dst[1]) || (job.src[2] && job.dst[2]);
             (void)copying;
             const cudaError_t e2 = launch_select_copy(bd, gp, io, job, ctx->tail_list + par * ctx->rows_all,
-                                                      ctx->status_dev,
-                                                      ctx->sm_count * kTailCtasPerSm - n, st);
+                                                      ctx->status_dev, ctx->sm_count * kTailCtasPerSm - n,
+                                                      ctx->stamps ? ctx->stamps + 2 * kStampSlots : nullptr, st);
             if (e2 != cudaSuccess) {
                 clear_accumulators(acc64, bd, st);
                 return fail_cuda(ctx, e2);

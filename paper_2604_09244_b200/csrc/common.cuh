@@ -15,7 +15,8 @@ constexpr int kKeyTile = 128;        // visual keys per tile = rows of one MMA
 constexpr int kMaxCluster = 8;       // portable cluster size
 constexpr int kMaxText = 64;
 constexpr int kMaxVis = 4096;
-constexpr uint32_t kSpinLimit = 1u << 22;   // bounded device-side waits (each try sleeps, see wait loops)
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr unsigned kStampSlots = 4096;      // CTAs per kernel that leave time stamps when asked to (mvla_set_kernel_stamps)   // bounded device-side waits (each try sleeps, see wait loops)
 
 // Device-side view of one sample; everything the host can compute is computed there.
 struct SampleDev {
@@ -94,6 +95,8 @@ int sm_count_of_current_device();
 // `part` is null too: only the attention copy is wanted).
 // `free_running`: the kernel does not wait for the kernel before it in its stream (the caller orders
 // everything it depends on with events).
+// `stamps`: when not null, CTA c (linear index, below kStampSlots) writes the global timer when it was free to
+// start its loads to stamps[2 c] and when it ended to stamps[2 c + 1].
 // `rearm`: when not null, words [out_off, out_off + n_out) of every sample are set to -1 (the kept list that
 // launch_select_copy's CTAs exchange, see there).
 // Optional copy of the attention itself for the patch-by-patch path:
@@ -110,7 +113,8 @@ bool fast_salience_supported(int tiles_per_cta);
 cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
-                                 bool free_running, AlphaOut alpha, int32_t* rearm, cudaStream_t stream);
+                                 bool free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* stamps,
+                                 cudaStream_t stream);
 
 
 // Salience: per-head partial scores part[h][vis] (already scaled by 1/(H n_t)).
@@ -178,10 +182,11 @@ cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int
 // (bounded waits, MVLA_ERR_TIMEOUT into `status` when one runs out): no kernel boundary, fence or flag lies
 // between selection and copy.  `list`: one int per output row of the batch, all -1 when the kernel starts
 // (the scoring kernel before it re-arms them, see launch_salience_fast).
-// `ctas`: copying CTAs to aim for (every sample gets at least one).
+// `ctas`: copying CTAs to aim for (every sample gets at least one).  `stamps`: as in launch_salience_fast
+// (start: past the wait for the kernel before; the selecting CTA's end is when the list is written).
 bool select_copy_supported(const BatchDesc& bd);
 cudaError_t launch_select_copy(const BatchDesc& bd, const GateParams& gp, const SelectIO& io, const CompactJob& job,
-                               int32_t* list, int* status, int ctas, cudaStream_t stream);
+                               int32_t* list, int* status, int ctas, unsigned long long* stamps, cudaStream_t stream);
 
 // One warp runs the copying CTAs' bounded wait on `never_set` (a word that holds -1 and stays so) with the
 // given limit and reports MVLA_ERR_TIMEOUT into `status` when it runs out.

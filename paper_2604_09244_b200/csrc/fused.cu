@@ -65,7 +65,8 @@ __global__ void __launch_bounds__(kFastThreads, 1)
 salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
                      const __grid_constant__ CUtensorMap tmap_k, int n_heads, int kv_group, int head_dim, int esize, int npad_max,
                      float* __restrict__ part, int64_t part_stride, unsigned long long* __restrict__ acc64,
-                     int* status, int free_running, const AlphaOut alpha, int32_t* __restrict__ rearm)
+                     int* status, int free_running, const AlphaOut alpha, int32_t* __restrict__ rearm,
+                     unsigned long long* __restrict__ stamps)
 {
     constexpr int CC = TCOL * NTILE;
     extern __shared__ uint8_t dyn_smem_raw[];
@@ -104,9 +105,6 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         any_live |= ti.valid > 0;
     }
 
-#ifdef MVLA_TRIGGER_EARLY
-    pdl_trigger();
-#endif
     if (tid == 0) {                           // the loads go out first; everything else overlaps with them
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);
@@ -118,6 +116,10 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         // Inputs may come from the kernel before this one -- unless the host has established (stable
         // inputs, scratch ordered by events) that nothing this kernel touches depends on it.
         if (!free_running) pdl_wait();
+        if (stamps) {                         // measurement aid: when this CTA was free to start its loads
+            const unsigned cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+            if (cta < kStampSlots) stamps[2 * cta] = global_ns();
+        }
         int live = 0;
 #pragma unroll
         for (int t = 0; t < NTILE; ++t) live += valid[t] > 0;
@@ -306,12 +308,17 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);    // the warp that allocated
+    if (stamps && tid == 0) {
+        const unsigned cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+        if (cta < kStampSlots) stamps[2 * cta + 1] = global_ns();
+    }
 }
 
 template <int TCOL, int NTILE>
 cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tq,
                           const CUtensorMap* tk, int cluster, int npad, float* part, int64_t part_stride,
-                          unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, int32_t* rearm, cudaStream_t stream)
+                          unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* stamps,
+                          cudaStream_t stream)
 {
     size_t smem = 1024 + static_cast<size_t>((head_dim * esize + 127) / 128) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
     auto kern = salience_fast_kernel<TCOL, NTILE>;
@@ -338,7 +345,7 @@ cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int he
     attr[1] = pdl_attribute();
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, kv_group, head_dim, esize, npad, part, part_stride, acc64, status, free_running, alpha, rearm);
+    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, kv_group, head_dim, esize, npad, part, part_stride, acc64, status, free_running, alpha, rearm, stamps);
 }
 
 }  // namespace
@@ -348,13 +355,14 @@ bool fast_salience_supported(int tiles_per_cta) { return tiles_per_cta >= 1 && t
 cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
-                                 bool free_running, AlphaOut alpha, int32_t* rearm, cudaStream_t stream)
+                                 bool free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* stamps,
+                                 cudaStream_t stream)
 {
     const int tcol = npad <= 16 ? 16 : (npad <= 32 ? 32 : 64);
 #define MVLA_FAST(TC, NTL)                                                                                      \
     if (tcol == TC && tiles_per_cta == NTL)                                                                     \
         return launch_fast_t<TC, NTL>(bd, n_heads, kv_group, head_dim, esize, tmap_q, tmap_k, cluster, npad, part, part_stride, \
-                                      acc64, status, free_running ? 1 : 0, alpha, rearm, stream);
+                                      acc64, status, free_running ? 1 : 0, alpha, rearm, stamps, stream);
     MVLA_FAST(16, 1) MVLA_FAST(32, 1) MVLA_FAST(64, 1) MVLA_FAST(16, 2) MVLA_FAST(32, 2) MVLA_FAST(64, 2)
 #undef MVLA_FAST
     return cudaErrorInvalidConfiguration;

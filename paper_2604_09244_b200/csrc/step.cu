@@ -119,7 +119,8 @@ __global__ void wait_probe_kernel(const int* never_set, uint64_t limit_ns, int* 
 template <int NT, int CAP>
 __global__ void __launch_bounds__(NT)
 select_copy_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ TailPlan tp, const GateParams gp,
-                   const SelectIO io, const __grid_constant__ CompactArgs ca, int32_t* __restrict__ list, int* status)
+                   const SelectIO io, const __grid_constant__ CompactArgs ca, int32_t* __restrict__ list, int* status,
+                   unsigned long long* __restrict__ stamps)
 {
     const int tid = threadIdx.x, lane = tid & 31;
     if (static_cast<int>(blockIdx.x) < bd.n) {
@@ -130,7 +131,10 @@ select_copy_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__
         role.late_pdl = true;
         role.l1_late = true;                                // the norms may come from a kernel that ran beside the scoring
         if (tp.cta0[bd.n] > 0) role.kept_sm = list + bd.s[b].out_off;   // every word is its own "ready" signal
-        select_sample<NT, CAP>(bd.s[b], b, gp, io, sm, role);
+        select_sample<NT, CAP>(bd.s[b], b, gp, io, sm, role, [&]() {}, [&]() {
+            if (stamps && tid == 0 && blockIdx.x < kStampSlots) stamps[2 * blockIdx.x + 1] = global_ns();
+        });
+        if (stamps && tid == 0 && blockIdx.x < kStampSlots) stamps[2 * blockIdx.x] = stamps[2 * blockIdx.x + 1];   // placeholder start, see the copiers
         return;
     }
     // ---- row copy
@@ -156,6 +160,7 @@ select_copy_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__
         });
     asm volatile("griddepcontrol.wait;" ::: "memory");      // keeps the chain of dependencies whole: the kernel after
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // this one may rely on the one before it being complete
+    if (stamps && tid == 0 && blockIdx.x < kStampSlots) stamps[2 * blockIdx.x] = global_ns();
 
     {
         const int n_rows = s.n_out - (text_early ? s.n_txt : 0);
@@ -173,11 +178,15 @@ select_copy_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__
             return true;
         });
     }
+    if (stamps && blockIdx.x < kStampSlots) {
+        __syncthreads();
+        if (tid == 0) stamps[2 * blockIdx.x + 1] = global_ns();
+    }
 }
 
 template <int NT, int CAP>
 cudaError_t launch_t(const BatchDesc& bd, const TailPlan& tp, const GateParams& gp, const SelectIO& io, const CompactArgs& ca,
-                     int32_t* list, int* status, cudaStream_t stream)
+                     int32_t* list, int* status, unsigned long long* stamps, cudaStream_t stream)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(bd.n + tp.cta0[bd.n]));
@@ -186,7 +195,7 @@ cudaError_t launch_t(const BatchDesc& bd, const TailPlan& tp, const GateParams& 
     cudaLaunchAttribute attr[1] = {pdl_attribute()};
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, select_copy_kernel<NT, CAP>, bd, tp, gp, io, ca, list, status);
+    return cudaLaunchKernelEx(&cfg, select_copy_kernel<NT, CAP>, bd, tp, gp, io, ca, list, status, stamps);
 }
 
 int max_vis_of(const BatchDesc& bd)
@@ -207,7 +216,7 @@ cudaError_t launch_wait_probe(const int32_t* never_set, uint64_t limit_ns, int* 
 }
 
 cudaError_t launch_select_copy(const BatchDesc& bd, const GateParams& gp, const SelectIO& io, const CompactJob& job,
-                               int32_t* list, int* status, int ctas, cudaStream_t stream)
+                               int32_t* list, int* status, int ctas, unsigned long long* stamps, cudaStream_t stream)
 {
     if (bd.n < 1 || !select_copy_supported(bd)) return cudaErrorInvalidConfiguration;
     const CompactArgs ca = compact_args(job);
@@ -227,8 +236,8 @@ cudaError_t launch_select_copy(const BatchDesc& bd, const GateParams& gp, const 
         for (int b = 0; b < bd.n; ++b) tp.cta0[b] = 0;       // nothing to copy: selection only
     }
     for (int b = bd.n; b <= kMaxChunk; ++b) tp.cta0[b] = static_cast<int16_t>(next);
-    if (max_vis_of(bd) <= 1024) return launch_t<512, 1024>(bd, tp, gp, io, ca, list, status, stream);
-    return launch_t<512, 2048>(bd, tp, gp, io, ca, list, status, stream);
+    if (max_vis_of(bd) <= 1024) return launch_t<512, 1024>(bd, tp, gp, io, ca, list, status, stamps, stream);
+    return launch_t<512, 2048>(bd, tp, gp, io, ca, list, status, stamps, stream);
 }
 
 }  // namespace mvla

@@ -31,7 +31,7 @@ SET_2D, SET_3D = 1, 2
 
 EXPORTS = ("mvla_prune_create", "mvla_salience", "mvla_select", "mvla_compact",
            "mvla_prune_step", "mvla_prune_destroy", "mvla_patch_indicators", "mvla_patch_select",
-           "mvla_salience_noalloc", "mvla_selftest_wait_timeout", "mvla_set_stage_event")
+           "mvla_salience_noalloc", "mvla_selftest_wait_timeout", "mvla_set_stage_event", "mvla_set_kernel_stamps")
 
 
 class MvlaError(RuntimeError):
@@ -108,6 +108,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.mvla_patch_indicators.restype = i32
     lib.mvla_patch_select.argtypes = [vp, i32, i32, sp, u32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.mvla_patch_select.restype = i32
+    lib.mvla_set_kernel_stamps.argtypes = [vp, vp]
+    lib.mvla_set_kernel_stamps.restype = i32
     lib.mvla_set_stage_event.argtypes = [vp, vp]
     lib.mvla_set_stage_event.restype = i32
     lib.mvla_selftest_wait_timeout.argtypes = [vp, u32, vp]
@@ -212,6 +214,17 @@ class PruneContext:
         rc = self._lib.mvla_set_stage_event(self._h, event.cuda_event if event is not None else None)
         if rc != OK:
             raise MvlaError(rc, "mvla_set_stage_event")
+
+    STAMP_SLOTS = 4096
+
+    def set_kernel_stamps(self, buf: Optional[torch.Tensor]) -> None:
+        """Measurement aid: `buf` (int64 device tensor [2, 4096, 2], zero-filled; None switches it off) receives
+        the start / end time stamps of the CTAs of the step's two kernels (see the header)."""
+        if buf is not None:
+            assert buf.dtype == torch.int64 and buf.numel() == 2 * self.STAMP_SLOTS * 2 and buf.is_contiguous()
+        rc = self._lib.mvla_set_kernel_stamps(self._h, _ptr(buf))
+        if rc != OK:
+            raise MvlaError(rc, "mvla_set_kernel_stamps")
 
     def selftest_wait_timeout(self, limit_us: int = 200, *, stream=None) -> None:
         """Makes one bounded device-side wait run out on purpose (see the header); afterwards every call
