@@ -113,6 +113,12 @@ typedef struct mvla_config {
     int32_t n_kv_heads;        /* grouped-query attention: k and v are [rows, n_kv_heads, head_dim] and query head h
                                   reads key head h / (n_heads / n_kv_heads); 0 -> n_heads.  Must divide n_heads.
                                   Not available together with patch_path */
+    int32_t logit_cache;       /* 1: keep the raw logits of the last step of every (prune point, slot), so that a step
+                                  which says which rows changed (mvla_tensors.changed_rows) recomputes only those
+                                  (Sec. 4.3 / 5.2: consecutive frames share most of their content).
+                                  n_prune_points x slots x n_heads x (max_2d + max_3d) x round16(max_text) floats.
+                                  bf16 / e4m3 tensor-core path, samples of up to 2048 visual tokens, budgeted modes */
+    int32_t reserved0;
 } mvla_config;
 
 /* One batch element (host array).  Offsets are rows relative to seq_off; the three segments
@@ -160,6 +166,13 @@ typedef struct mvla_tensors {
     int64_t rows;              /* rows allocated in each tensor (bounds the TMA descriptors) */
     const float *rand_u;       /* MVLA_MODE_PATCH: one uniform number in [0, 1) per patch, samples back to back
                                   (the draws of the background rule); NULL otherwise */
+    const uint8_t *changed_rows; /* HOST array, one byte per row of the packed tensors, or NULL.  Non-zero: the caller
+                                  rewrote this row of q / k since the previous step on the sample's state.  Read during
+                                  the call (not afterwards).  Used only by contexts created with logit_cache: visual
+                                  keys are handled in tiles of 128 per modality, and a tile none of whose rows changed
+                                  takes its logits from the previous step instead of K (half the bytes, no MMA); a
+                                  changed text row, a reset state, a different sample shape, NULL or the first step
+                                  recompute everything.  A mask that hides a change silently reuses stale logits. */
 } mvla_tensors;
 
 /* Outputs of the fused step (device pointers, caller-owned). */
@@ -260,6 +273,13 @@ int32_t mvla_prune_step(mvla_ctx *ctx, int32_t prune_point, int32_t batch,
  * batches of more than 32 samples the event is recorded once per launch of 32.  The library never destroys it.
  */
 int32_t mvla_set_stage_event(mvla_ctx *ctx, void *event);
+
+/*
+ * Key tiles that mvla_prune_step recomputed and reused so far on this context (cumulative; contexts created
+ * with logit_cache; either pointer may be null).  Host-side counters: the decision is taken on the host from
+ * the caller's changed_rows.
+ */
+int32_t mvla_logit_cache_stats(mvla_ctx *ctx, int64_t *tiles_computed, int64_t *tiles_reused);
 
 /*
  * Measurement aid (the paper has no counterpart): time stamps taken by the step's own kernels.  An event

@@ -40,6 +40,12 @@ struct mvla_ctx {
     int32_t* tail_list;          // [kSets][max_batch * (max_text + max_vis)] kept list as the copying CTAs read it (-1 between launches)
     size_t rows_all;             // max_batch * (max_text + max_vis)
     int sm_count;                // multiprocessors of the device
+    // reuse of the previous step's logits (cfg.logit_cache)
+    float* lcache;               // [n_prune_points * n_slots][H][max_vis][cache_cols] raw dot products
+    int cache_cols;              // round16(max_text)
+    struct CacheSig { bool valid; int32_t n_txt, n_2d, n_3d; };
+    std::vector<CacheSig> cache_sig;   // per (prune point, slot): does the cache hold the last step's logits, and of what shape
+    int64_t tiles_computed, tiles_reused;
     cudaEvent_t stage_event;     // measurement aid: recorded between scoring and selection + copy (null: off)
     unsigned long long* stamps;  // measurement aid: device buffer [2][kStampSlots][2] of per-CTA time stamps (null: off)
     size_t vis_all;              // max_batch * max_vis
@@ -165,6 +171,8 @@ int32_t make_plan(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_
         d.vis_off = vis_off;
         vis_off += nv;
         d.k_2d_fixed = -1;
+        d.cache_state = -1;
+        d.tile_compute = 0xFFFFFFFFu;
         d.t = 1; d.update_state = 0; d.c_prev = 0.f; d.c_new = 1.f;
         if (with_state) {
             const int sidx = prune_point * ctx->n_slots + in.state_slot;
@@ -273,7 +281,8 @@ int32_t check_sticky(mvla_ctx* ctx)
 int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, const void* k, int64_t rows,
                            const void* hidden, float* l1, unsigned long long* acc64, bool* used_acc64,
                            bool free_running, cudaStream_t st, AlphaOut alpha = AlphaOut{nullptr, 0, 0},
-                           int32_t* rearm = nullptr, bool norms_beside = false, unsigned long long* stamps = nullptr)
+                           int32_t* rearm = nullptr, bool norms_beside = false, unsigned long long* stamps = nullptr,
+                           bool with_cache = false)
 {
     if (used_acc64) *used_acc64 = false;
     const mvla_config& c = ctx->cfg;
@@ -305,7 +314,8 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
         e = launch_salience_fast(bd, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, static_cast<int>(ctx->qk_elem), tq, tk,
                                  tiles_per_cta, cluster, npad,
                                  alpha.ptr && !acc64 ? nullptr : ctx->part,     // the patch path reads the attention copy only
-                                 ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, rearm, stamps, st);
+                                 ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, rearm, stamps,
+                                 with_cache ? ctx->lcache : nullptr, ctx->max_vis, ctx->cache_cols, st);
         if (used_acc64) *used_acc64 = acc64 != nullptr;
     } else {
         e = launch_salience(bd, c.dtype, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, q, k, tq, tk, ctx->use_umma, tiles_per_cta,
@@ -633,6 +643,9 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     if (c.dtype != MVLA_DTYPE_BF16 && c.dtype != MVLA_DTYPE_FP32 && c.dtype != MVLA_DTYPE_FP8_E4M3) return MVLA_ERR_UNSUPPORTED;
     if (c.dtype == MVLA_DTYPE_FP8_E4M3 && (c.salience_path == MVLA_SALIENCE_FMA || c.patch_path)) return MVLA_ERR_UNSUPPORTED;
     if (c.salience_path != MVLA_SALIENCE_AUTO && c.salience_path != MVLA_SALIENCE_FMA) return MVLA_ERR_INVALID_ARG;
+    if (c.logit_cache != 0 && c.logit_cache != 1) return MVLA_ERR_INVALID_ARG;
+    if (c.logit_cache && (c.dtype == MVLA_DTYPE_FP32 || c.salience_path == MVLA_SALIENCE_FMA || c.patch_path))
+        return MVLA_ERR_UNSUPPORTED;          // the cache lives in the tensor-core scoring kernel of the budgeted path
     if ((c.patch_path != 0 && c.patch_path != 1) || c.kmeans_max_iter < 0 || !(c.obj_2d_min >= 0.0 && c.obj_2d_min <= 1.0))
         return MVLA_ERR_INVALID_ARG;
     if (c.head_dim < 64 || c.head_dim > 256 || c.head_dim % 32 != 0) return MVLA_ERR_UNSUPPORTED;
@@ -670,6 +683,9 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     ctx->sm_count = prop.multiProcessorCount;
     ctx->stage_event = nullptr;
     ctx->stamps = nullptr;
+    ctx->lcache = nullptr;
+    ctx->cache_cols = (c.max_text + 15) / 16 * 16;
+    ctx->tiles_computed = ctx->tiles_reused = 0;
     ctx->alpha_ws = ctx->xhat_patch = ctx->patch_x_ws = ctx->patch_attn_ws = nullptr;
     ctx->patch_sets = 1;
     ctx->nout_ws = nullptr;
@@ -711,6 +727,10 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     // (+ 1: a word that no launch ever writes, for mvla_selftest_wait_timeout)
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->tail_list), (kSets * ctx->rows_all + 1) * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->tail_list, 0xFF, (kSets * ctx->rows_all + 1) * sizeof(int32_t));
+    if (c.logit_cache) {
+        ctx->cache_sig.assign(n_state, mvla_ctx::CacheSig{false, 0, 0, 0});
+        alloc(&ctx->lcache, n_state * static_cast<size_t>(c.n_heads) * ctx->max_vis * ctx->cache_cols);
+    }
     if (c.patch_path) {
         const size_t alpha_n = static_cast<size_t>(c.n_heads) * c.max_text * vis_all;
         ctx->patch_sets = alpha_n * sizeof(float) * kSets <= (size_t(1) << 30) ? kSets : 1;   // at most 1 GiB of attention copies
@@ -761,6 +781,7 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     cudaFree(ctx->mhat_state);
     cudaFree(ctx->acc64);
     cudaFree(ctx->tail_list);
+    cudaFree(ctx->lcache);
     cudaFree(ctx->alpha_ws);
     cudaFree(ctx->xhat_patch);
     cudaFree(ctx->patch_x_ws);
@@ -885,6 +906,14 @@ int32_t mvla_set_stage_event(mvla_ctx* ctx, void* event)
     return MVLA_OK;
 }
 
+int32_t mvla_logit_cache_stats(mvla_ctx* ctx, int64_t* tiles_computed, int64_t* tiles_reused)
+{
+    if (!ctx) return MVLA_ERR_INVALID_ARG;
+    if (tiles_computed) *tiles_computed = ctx->tiles_computed;
+    if (tiles_reused) *tiles_reused = ctx->tiles_reused;
+    return MVLA_OK;
+}
+
 int32_t mvla_set_kernel_stamps(mvla_ctx* ctx, uint64_t* device_buffer)
 {
     if (!ctx || (reinterpret_cast<uintptr_t>(device_buffer) & 7u)) return MVLA_ERR_INVALID_ARG;
@@ -986,6 +1015,45 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     for (int i = 0; i < 3; ++i) { job.src[i] = src[i]; job.dst[i] = dst[i]; job.row_bytes[i] = kv_bytes; }
     job.row_bytes[0] = static_cast<int32_t>(ctx->cfg.d_model * ctx->elem);
 
+    // Reuse of the previous step's logits: which key tiles of which sample must be computed (host decision
+    // from the caller's changed_rows), for steps that are not overlapped with their neighbours.
+    const bool cache_on = ctx->lcache != nullptr && !(flags & MVLA_FLAG_INPUTS_STABLE);
+    for (int b = 0; b < batch; ++b) {
+        SampleDev& d = plan.s[b];
+        d.cache_state = -1;
+        d.tile_compute = 0xFFFFFFFFu;
+        if (!ctx->lcache) continue;
+        const mvla_sample& sm = samples[b];
+        const int sidx = prune_point * ctx->n_slots + sm.state_slot;
+        mvla_ctx::CacheSig& sig = ctx->cache_sig[sidx];
+        const int tiles = tiles_of(d);
+        const bool fits = sm.n_2d + sm.n_3d <= 2048 && batch <= kMaxChunk;
+        if (!cache_on || !fits || (flags & MVLA_FLAG_NO_STATE_UPDATE)) {
+            // the step runs without the cache; a dry run leaves it as it is, anything else makes it stale
+            if (!(flags & MVLA_FLAG_NO_STATE_UPDATE)) sig.valid = false;
+            continue;
+        }
+        d.cache_state = sidx;
+        bool all = !sig.valid || (flags & MVLA_FLAG_RESET_STATE) || !in->changed_rows || sig.n_txt != sm.n_txt ||
+                   sig.n_2d != sm.n_2d || sig.n_3d != sm.n_3d;
+        const uint8_t* ch = in->changed_rows ? in->changed_rows + sm.seq_off : nullptr;
+        for (int i = 0; i < sm.n_txt && !all; ++i) all = ch[sm.off_txt + i] != 0;   // a changed query changes every logit
+        if (!all) {
+            uint32_t mask = 0;
+            const int t2 = (sm.n_2d + kKeyTile - 1) / kKeyTile;
+            for (int t = 0; t < tiles; ++t) {
+                const int off = t < t2 ? sm.off_2d + t * kKeyTile : sm.off_3d + (t - t2) * kKeyTile;
+                const int n = t < t2 ? std::min(kKeyTile, sm.n_2d - t * kKeyTile) : std::min(kKeyTile, sm.n_3d - (t - t2) * kKeyTile);
+                bool any = false;
+                for (int i = 0; i < n && !any; ++i) any = ch[off + i] != 0;
+                if (any) mask |= 1u << t;
+            }
+            d.tile_compute = mask;
+        }
+        for (int t = 0; t < tiles; ++t) ((d.tile_compute >> t) & 1u ? ctx->tiles_computed : ctx->tiles_reused) += 1;
+        sig = mvla_ctx::CacheSig{true, sm.n_txt, sm.n_2d, sm.n_3d};
+    }
+
     // scratch set of this step
     ctx->step_parity = (ctx->step_parity + 1u) % kSets;
     unsigned long long* acc64 = ctx->acc64 + ctx->step_parity * ctx->vis_all;
@@ -1023,7 +1091,8 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         const bool tail = !forked && select_copy_supported(bd);
         rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, l1_ws, acc64,
                                 &used_acc64, false, forked ? ctx->aux[par] : st, AlphaOut{nullptr, 0, 0},
-                                tail ? ctx->tail_list + par * ctx->rows_all : nullptr, tail, tail ? ctx->stamps : nullptr);
+                                tail ? ctx->tail_list + par * ctx->rows_all : nullptr, tail, tail ? ctx->stamps : nullptr,
+                                cache_on);
         if (rc != MVLA_OK) return rc;
         if (ctx->stage_event && !forked) {
             // under stream capture the record must become an event-record node of the graph (an "external"

@@ -34,6 +34,9 @@ struct SampleDev {
     int32_t mstate_off;     // indicator state array (x4 floats): index of the copy this step reads
     int32_t mstate_off_w;   // ... and writes
     int32_t slot_index;     // prune point * slots + slot: addresses the per-patch state (updated in place by one CTA)
+    // reuse of the previous step's logits (Sec. 4.3 / 5.2); cache_state < 0: off for this sample
+    int32_t cache_state;    // which (prune point, slot) block of the logit cache
+    uint32_t tile_compute;  // bit t: key tile t must be computed from K (and its logits stored); clear: reuse the cached logits
     int32_t t;              // 1-based action step this call is
     int32_t update_state;   // 0: dry run
     float c_prev, c_new;    // state update weights: xhat = c_prev * xhat + c_new * x
@@ -95,6 +98,8 @@ int sm_count_of_current_device();
 // `part` is null too: only the attention copy is wanted).
 // `free_running`: the kernel does not wait for the kernel before it in its stream (the caller orders
 // everything it depends on with events).
+// `lcache`: logit cache [state][head][cache_vis][cache_cols] fp32 (raw dot products), or null; which tiles are
+// computed and stored and which are read back is in the descriptors (cache_state, tile_compute).
 // `stamps`: when not null, CTA c (linear index, below kStampSlots) writes the global timer when it was free to
 // start its loads to stamps[2 c] and when it ended to stamps[2 c + 1].
 // `rearm`: when not null, words [out_off, out_off + n_out) of every sample are set to -1 (the kept list that
@@ -114,7 +119,7 @@ cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
                                  bool free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* stamps,
-                                 cudaStream_t stream);
+                                 float* lcache, int cache_vis, int cache_cols, cudaStream_t stream);
 
 
 // Salience: per-head partial scores part[h][vis] (already scaled by 1/(H n_t)).

@@ -66,7 +66,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
                      const __grid_constant__ CUtensorMap tmap_k, int n_heads, int kv_group, int head_dim, int esize, int npad_max,
                      float* __restrict__ part, int64_t part_stride, unsigned long long* __restrict__ acc64,
                      int* status, int free_running, const AlphaOut alpha, int32_t* __restrict__ rearm,
-                     unsigned long long* __restrict__ stamps)
+                     unsigned long long* __restrict__ stamps, float* __restrict__ lcache, int cache_vis, int cache_cols)
 {
     constexpr int CC = TCOL * NTILE;
     extern __shared__ uint8_t dyn_smem_raw[];
@@ -96,14 +96,19 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     const uint32_t bar_full = smem_u32(&s_bar[0]), bar_mma = smem_u32(&s_bar[1]), bar_x = smem_u32(&s_bar[2]);
 
     int valid[NTILE], vis0[NTILE];
+    bool from_k[NTILE];                       // the tile's logits come from K (TMA + MMA); false: from the logit cache
     bool any_live = false;
+    const bool caching = lcache != nullptr && s.cache_state >= 0;
 #pragma unroll
     for (int t = 0; t < NTILE; ++t) {
         const TileInfo ti = tile_info(s, tt0 + t);
         valid[t] = ti.valid;
         vis0[t] = ti.vis0;
         any_live |= ti.valid > 0;
+        from_k[t] = !caching || ((s.tile_compute >> (tt0 + t)) & 1u) != 0;
     }
+    // row of this thread's key in the cache: [state][head][visual index][column]
+    const int64_t cache_row0 = caching ? ((static_cast<int64_t>(s.cache_state) * n_heads + h) * cache_vis) * cache_cols : 0;
 
     if (tid == 0) {                           // the loads go out first; everything else overlaps with them
         prefetch_tensormap(&tmap_q);
@@ -120,17 +125,18 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
             const unsigned cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
             if (cta < kStampSlots) stamps[2 * cta] = global_ns();
         }
-        int live = 0;
+        int live = 0;                         // key tiles to fetch: those that exist and do not come from the cache
 #pragma unroll
-        for (int t = 0; t < NTILE; ++t) live += valid[t] > 0;
-        mbar_expect_tx(bar_full, static_cast<uint32_t>(khalves) * (npad * 128 + live * 16384));
-        for (int kh = 0; kh < khalves; ++kh)
+        for (int t = 0; t < NTILE; ++t) live += valid[t] > 0 && from_k[t];
+        // (no tile to compute: nothing is fetched, both barriers below complete at once)
+        mbar_expect_tx(bar_full, live > 0 ? static_cast<uint32_t>(khalves) * (npad * 128 + live * 16384) : 0u);
+        for (int kh = 0; kh < khalves && live > 0; ++kh)
             for (int c = 0; c < npad / 16; ++c)
                 tma_load_3d(smem_u32(Qs + kh * npad * 128 + c * 2048), &tmap_q, kh * box_elems, h,
                             s.seq_off + s.off_txt + c * 16, bar_full);
 #pragma unroll
         for (int t = 0; t < NTILE; ++t) {
-            if (valid[t] <= 0) continue;
+            if (valid[t] <= 0 || !from_k[t]) continue;
             const int row0 = tile_info(s, tt0 + t).row0;
             for (int kh = 0; kh < khalves; ++kh)
                 tma_load_3d(smem_u32(Ks + (t * khalves + kh) * 16384), &tmap_k, kh * box_elems, h / kv_group, row0, bar_full);
@@ -167,7 +173,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
             const uint32_t idesc = idesc_by_size(esize, npad);
 #pragma unroll
             for (int t = 0; t < NTILE; ++t) {
-                if (valid[t] <= 0) continue;
+                if (valid[t] <= 0 || !from_k[t]) continue;
                 for (int kb = 0; kb < khalves * 4; ++kb) {     // columns past d are zeros: they add nothing
                     const int kh = kb >> 2, kin = kb & 3;          // 4 K-steps of 16 inside a 64-wide half
                     const uint64_t a = smem_desc_sw128(smem_u32(Ks + (t * khalves + kh) * 16384) + kin * 32);
@@ -196,6 +202,25 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     } else {
 #pragma unroll
         for (int i = 0; i < CC; ++i) L[i] = 0.f;
+    }
+    // Logit cache: a computed tile leaves its raw dot products for the next action step, a reused tile takes
+    // the previous step's instead (128 bytes per key and head at 32 queries: half a key row, and no MMA).
+    if (caching && ok) {
+#pragma unroll
+        for (int t = 0; t < NTILE; ++t) {
+            if (tid >= valid[t]) continue;
+            float4* row = reinterpret_cast<float4*>(lcache + cache_row0 + static_cast<int64_t>(vis0[t] + tid) * cache_cols);
+#pragma unroll
+            for (int i = 0; i < TCOL / 4; ++i) {
+                if (4 * i >= npad) break;
+                if (from_k[t]) {
+                    row[i] = make_float4(L[t * TCOL + 4 * i], L[t * TCOL + 4 * i + 1], L[t * TCOL + 4 * i + 2], L[t * TCOL + 4 * i + 3]);
+                } else {
+                    const float4 v = __ldcg(row + i);
+                    L[t * TCOL + 4 * i] = v.x; L[t * TCOL + 4 * i + 1] = v.y; L[t * TCOL + 4 * i + 2] = v.z; L[t * TCOL + 4 * i + 3] = v.w;
+                }
+            }
+        }
     }
     // The registers keep the raw dot products; the scale enters with the exponent below (one FFMA).  Keys
     // past the end of a ragged tile are masked; a full tile needs no pass over the registers at all, and
@@ -318,7 +343,7 @@ template <int TCOL, int NTILE>
 cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tq,
                           const CUtensorMap* tk, int cluster, int npad, float* part, int64_t part_stride,
                           unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* stamps,
-                          cudaStream_t stream)
+                          float* lcache, int cache_vis, int cache_cols, cudaStream_t stream)
 {
     size_t smem = 1024 + static_cast<size_t>((head_dim * esize + 127) / 128) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
     auto kern = salience_fast_kernel<TCOL, NTILE>;
@@ -345,7 +370,7 @@ cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int he
     attr[1] = pdl_attribute();
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, kv_group, head_dim, esize, npad, part, part_stride, acc64, status, free_running, alpha, rearm, stamps);
+    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, kv_group, head_dim, esize, npad, part, part_stride, acc64, status, free_running, alpha, rearm, stamps, lcache, cache_vis, cache_cols);
 }
 
 }  // namespace
@@ -356,13 +381,13 @@ cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
                                  bool free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* stamps,
-                                 cudaStream_t stream)
+                                 float* lcache, int cache_vis, int cache_cols, cudaStream_t stream)
 {
     const int tcol = npad <= 16 ? 16 : (npad <= 32 ? 32 : 64);
 #define MVLA_FAST(TC, NTL)                                                                                      \
     if (tcol == TC && tiles_per_cta == NTL)                                                                     \
         return launch_fast_t<TC, NTL>(bd, n_heads, kv_group, head_dim, esize, tmap_q, tmap_k, cluster, npad, part, part_stride, \
-                                      acc64, status, free_running ? 1 : 0, alpha, rearm, stamps, stream);
+                                      acc64, status, free_running ? 1 : 0, alpha, rearm, stamps, lcache, cache_vis, cache_cols, stream);
     MVLA_FAST(16, 1) MVLA_FAST(32, 1) MVLA_FAST(64, 1) MVLA_FAST(16, 2) MVLA_FAST(32, 2) MVLA_FAST(64, 2)
 #undef MVLA_FAST
     return cudaErrorInvalidConfiguration;

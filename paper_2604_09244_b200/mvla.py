@@ -31,7 +31,8 @@ SET_2D, SET_3D = 1, 2
 
 EXPORTS = ("mvla_prune_create", "mvla_salience", "mvla_select", "mvla_compact",
            "mvla_prune_step", "mvla_prune_destroy", "mvla_patch_indicators", "mvla_patch_select",
-           "mvla_salience_noalloc", "mvla_selftest_wait_timeout", "mvla_set_stage_event", "mvla_set_kernel_stamps")
+           "mvla_salience_noalloc", "mvla_selftest_wait_timeout", "mvla_set_stage_event", "mvla_set_kernel_stamps",
+           "mvla_logit_cache_stats")
 
 
 class MvlaError(RuntimeError):
@@ -49,7 +50,8 @@ class Config(C.Structure):
                 ("salience_path", C.c_int32),
                 ("tau_2d", C.c_double), ("tau_3d", C.c_double), ("beta", C.c_double),
                 ("eps_3d", C.c_double), ("floor_ratio", C.c_double), ("obj_2d_min", C.c_double),
-                ("patch_path", C.c_int32), ("kmeans_max_iter", C.c_int32), ("n_kv_heads", C.c_int32)]
+                ("patch_path", C.c_int32), ("kmeans_max_iter", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("logit_cache", C.c_int32), ("reserved0", C.c_int32)]
 
 
 class CSample(C.Structure):
@@ -67,7 +69,7 @@ class CDiag(C.Structure):
 
 class CTensors(C.Structure):
     _fields_ = [("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("hidden", C.c_void_p),
-                ("rows", C.c_int64), ("rand_u", C.c_void_p)]
+                ("rows", C.c_int64), ("rand_u", C.c_void_p), ("changed_rows", C.c_void_p)]
 
 
 class COutputs(C.Structure):
@@ -108,6 +110,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.mvla_patch_indicators.restype = i32
     lib.mvla_patch_select.argtypes = [vp, i32, i32, sp, u32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.mvla_patch_select.restype = i32
+    lib.mvla_logit_cache_stats.argtypes = [vp, C.POINTER(i64), C.POINTER(i64)]
+    lib.mvla_logit_cache_stats.restype = i32
     lib.mvla_set_kernel_stamps.argtypes = [vp, vp]
     lib.mvla_set_kernel_stamps.restype = i32
     lib.mvla_set_stage_event.argtypes = [vp, vp]
@@ -178,7 +182,7 @@ class PruneContext:
                  beta: float = 0.85, window_k: int = 7, eps_3d: float = 0.02,
                  floor_ratio: float = 0.10, cold_start_full_keep: int = 1,
                  salience_path: int = SALIENCE_AUTO, device: Optional[int] = None, patch_path: int = 0,
-                 obj_2d_min: float = 0.5, kmeans_max_iter: int = 32, n_kv_heads: int = 0):
+                 obj_2d_min: float = 0.5, kmeans_max_iter: int = 32, n_kv_heads: int = 0, logit_cache: int = 0):
         self._h = C.c_void_p()
         self._lib = lib()
         if device is None:
@@ -190,7 +194,7 @@ class PruneContext:
         self.cfg = Config(device, code, n_heads, head_dim, d_model, max_batch, max_text, max_2d,
                           max_3d, n_prune_points, n_state_slots, window_k, cold_start_full_keep,
                           salience_path, tau_2d, tau_3d, beta, eps_3d, floor_ratio, obj_2d_min, patch_path,
-                          kmeans_max_iter, n_kv_heads)
+                          kmeans_max_iter, n_kv_heads, logit_cache, 0)
         rc = self._lib.mvla_prune_create(C.byref(self.cfg), C.byref(self._h))
         if rc != OK:
             self._h = C.c_void_p()
@@ -216,6 +220,14 @@ class PruneContext:
             raise MvlaError(rc, "mvla_set_stage_event")
 
     STAMP_SLOTS = 4096
+
+    def logit_cache_stats(self):
+        """(key tiles recomputed, key tiles reused) by prune_step so far."""
+        a, b = C.c_int64(0), C.c_int64(0)
+        rc = self._lib.mvla_logit_cache_stats(self._h, C.byref(a), C.byref(b))
+        if rc != OK:
+            raise MvlaError(rc, "mvla_logit_cache_stats")
+        return a.value, b.value
 
     def set_kernel_stamps(self, buf: Optional[torch.Tensor]) -> None:
         """Measurement aid: `buf` (int64 device tensor [2, 4096, 2], zero-filled; None switches it off) receives
@@ -326,12 +338,18 @@ class PruneContext:
         return out
 
     def prune_step(self, prune_point, samples, mode, q, k, v, hidden, *, flags=0,
-                   out: StepOutputs = None, stream=None, rand_u=None) -> StepOutputs:
+                   out: StepOutputs = None, stream=None, rand_u=None, changed_rows=None) -> StepOutputs:
         cs = samples if isinstance(samples, C.Array) else c_samples(samples)
         if out is None:
             out = self.alloc_outputs(cs, hidden=hidden is not None, kv=v is not None, extras=True,
                                      patch=mode == MODE_PATCH)
-        tin = CTensors(_ptr(q), _ptr(k), _ptr(v), _ptr(hidden), q.shape[0], _ptr(rand_u))
+        ch = None
+        if changed_rows is not None:         # host bytes, read during the call
+            import numpy as np
+            changed_rows = np.ascontiguousarray(changed_rows, dtype=np.uint8)
+            assert changed_rows.shape[0] == q.shape[0], "one byte per row of the packed tensors"
+            ch = changed_rows.ctypes.data
+        tin = CTensors(_ptr(q), _ptr(k), _ptr(v), _ptr(hidden), q.shape[0], _ptr(rand_u), ch)
         tout = COutputs(_ptr(out.out_hidden), _ptr(out.out_k), _ptr(out.out_v), _ptr(out.kept_idx),
                         _ptr(out.out_offsets), _ptr(out.budgets), _ptr(out.attn), _ptr(out.ahat),
                         _ptr(out.z), _ptr(out.diag), _ptr(out.patch_x), _ptr(out.patch_xhat),
@@ -346,7 +364,7 @@ class PruneContext:
 
 
 def context_for(wl, *, max_batch=None, n_prune_points=1, n_state_slots=0, salience_path=SALIENCE_AUTO,
-                device=None, patch_path=None) -> PruneContext:
+                device=None, patch_path=None, logit_cache=0) -> PruneContext:
     """A context sized for a synthetic workload (see ``workloads``)."""
     dt = {"bf16": torch.bfloat16, "fp32": torch.float32, "fp8": torch.float8_e4m3fn}[wl.dtype]
     return PruneContext(dtype=dt, n_heads=wl.n_heads, head_dim=wl.head_dim, d_model=wl.d_model,
@@ -361,7 +379,7 @@ def context_for(wl, *, max_batch=None, n_prune_points=1, n_state_slots=0, salien
                         patch_path=int(wl.mode == MODE_PATCH) if patch_path is None else patch_path,
                         obj_2d_min=wl.extra.get("obj_2d_min", 0.5),
                         kmeans_max_iter=wl.extra.get("kmeans_max_iter", 32),
-                        n_kv_heads=wl.extra.get("n_kv_heads", 0))
+                        n_kv_heads=wl.extra.get("n_kv_heads", 0), logit_cache=logit_cache)
 
 
 def to_device(arr, dtype: str, device) -> torch.Tensor:

@@ -92,13 +92,13 @@ def check_compaction(wl_tensors_np, dev_out, s, kept_gpu, row0, dtype):
         assert np.array_equal(got_bits, ref_bits), f"{name}: differs from the oracle's compaction"
 
 
-def run_and_check_step(ctx, wl, step, states, *, prune_point=0, flags=0, dev=None, samples=None):
+def run_and_check_step(ctx, wl, step, states, *, prune_point=0, flags=0, dev=None, samples=None, changed_rows=None):
     """One fused GPU step against the oracle on the same inputs.  `states`: oracle State per sample.
     Returns (gpu outputs, list of oracle StepResult)."""
     dev = dev or device_tensors(wl, step)
     samples = samples or wl.samples
     out = ctx.prune_step(prune_point, samples, wl.mode, dev["q"], dev["k"], dev["v"], dev["hidden"],
-                         flags=flags)
+                         flags=flags, changed_rows=changed_rows)
     torch.cuda.synchronize()
     refs = oracle.run_workload_step(wl, step, states)
     offs = out.out_offsets.cpu().numpy()

@@ -26,10 +26,10 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_struct_sizes_match_the_header_layout():
-    assert C.sizeof(mvla.Config) == 14 * 4 + 6 * 8 + 4 * 4      # three int32 and padding after the doubles
+    assert C.sizeof(mvla.Config) == 14 * 4 + 6 * 8 + 6 * 4      # five int32 and a reserved one after the doubles
     assert C.sizeof(mvla.CSample) == 8 * 4 + 3 * 8
     assert C.sizeof(mvla.CDiag) == 64
-    assert C.sizeof(mvla.CTensors) == 6 * 8
+    assert C.sizeof(mvla.CTensors) == 7 * 8
     assert C.sizeof(mvla.COutputs) == 14 * 8
     assert C.sizeof(mvla.CPatchDiag) == 64
 

@@ -8,7 +8,7 @@ import torch
 import oracle
 from paper_2604_09244_b200 import mvla
 from paper_2604_09244_b200 import workloads as W
-from parity_util import (assert_salience_close, check_compaction, check_kept_against_oracle,
+from parity_util import (SALIENCE_RTOL, assert_salience_close, check_compaction, check_kept_against_oracle,
                          check_stagewise_exact, device_tensors, diag_records, run_and_check_step)
 
 pytestmark = pytest.mark.gpu
@@ -667,3 +667,51 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_sticky():
         ctx2.selftest_wait_timeout(0)                                 # the limit must be 1 us .. 1 s
     assert e.value.code == mvla.ERR_INVALID_ARG
     ctx2.close()
+
+
+# ------------------------------------------------------------------ reuse of the previous action step's logits
+@pytest.mark.parametrize("drift,T", [("all", 16), ("visual_local", 8)])
+def test_action_iteration_reusing_the_previous_steps_logits(drift, T):
+    # every step is judged against the FULL oracle on the step's own inputs: with a truthful mask the reuse
+    # must not be visible in the results
+    wl = W.config5_action_iteration(T=T, drift=drift)
+    ctx = mvla.context_for(wl, logit_cache=1)
+    states = _fresh_states(wl)
+    per_step = []
+    for t in range(T):
+        before = ctx.logit_cache_stats()
+        run_and_check_step(ctx, wl, t, states, flags=mvla.FLAG_RESET_STATE if t == 0 else 0,
+                           changed_rows=wl.extra["changed_rows"][t] if t > 0 else None)
+        after = ctx.logit_cache_stats()
+        per_step.append((after[0] - before[0], after[1] - before[1]))
+    assert per_step[0] == (10, 0)                                     # 2 image + 8 point tiles, nothing to reuse yet
+    assert all(c + r == 10 for c, r in per_step)
+    if drift == "visual_local":                                       # one run of 131 rows: two or three tiles change
+        assert all(1 <= c <= 3 for c, r in per_step[1:])
+    ctx.close()
+
+
+def test_a_mask_that_hides_a_change_reuses_the_stale_logits():
+    # shows that the cache is what is read: with a mask that claims nothing changed, step 2 returns step 1's scores
+    wl = W.config5_action_iteration(T=2, D=256, H=4, d=64, n_txt=20, n_2d=150, n_3d=300, drift="visual_local")
+    ctx = mvla.context_for(wl, logit_cache=1)
+    wl.steps[1].k[:40] *= np.float32(-2.0)                            # a change no tolerance can hide (exact in bf16)
+    dev0, dev1 = device_tensors(wl, 0), device_tensors(wl, 1)
+    out0 = ctx.prune_step(0, wl.samples, wl.mode, dev0["q"], dev0["k"], dev0["v"], dev0["hidden"], flags=mvla.FLAG_RESET_STATE)
+    attn0 = out0.attn.clone()
+    lie = np.zeros(wl.samples[0].seq_len, dtype=np.uint8)
+    out1 = ctx.prune_step(0, wl.samples, wl.mode, dev1["q"], dev1["k"], dev1["v"], dev1["hidden"], changed_rows=lie)
+    torch.cuda.synchronize()
+    assert torch.equal(out1.attn, attn0)
+    t1 = wl.steps[1]
+    truth = oracle.salience(t1.q, t1.k, wl.n_heads, wl.head_dim, wl.samples[0])
+    got = out1.attn.cpu().numpy()
+    assert (np.abs(got - truth) > 20 * SALIENCE_RTOL * np.abs(truth)).sum() >= 20, "the stale logits were not what was used"
+    # and with the truthful mask the same step is right
+    ctx.prune_step(0, wl.samples, wl.mode, dev0["q"], dev0["k"], dev0["v"], dev0["hidden"], flags=mvla.FLAG_RESET_STATE)
+    out2 = ctx.prune_step(0, wl.samples, wl.mode, dev1["q"], dev1["k"], dev1["v"], dev1["hidden"],
+                          changed_rows=wl.extra["changed_rows"][1] | (np.arange(wl.samples[0].seq_len) < 40))
+    torch.cuda.synchronize()
+    assert_salience_close(out2.attn.cpu().numpy(), truth)
+    assert ctx.logit_cache_stats()[1] >= 5                            # step 2 reused all 2 + 3 tiles of step 1
+    ctx.close()
