@@ -47,29 +47,20 @@ def measured_peaks():
     return {"hbm_gbs": HBM_FALLBACK_GBS}, "fallback"
 
 
-# DRAM bytes (read + write) per launch of the stage's kernel(s) from one ncu capture of this benchmark
-# (summaries under profiles/), valid only for the kernel sources they were taken on: per stage a digest over
-# the source files its kernels are compiled from.
+# DRAM bytes (read + write) per launch of the step's kernels from one ncu capture of this benchmark
+# (summaries under profiles/), valid only for the kernel sources they were taken on: per kernel a digest over
+# the source files it is compiled from.
 NCU_SOURCES = {
-    "salience": ("fused.cu", "device_utils.cuh", "tmem_ld.cuh", "select_impl.cuh", "common.cuh"),
-    "select": ("select.cu", "select_impl.cuh", "common.cuh"),
-    "compact": ("compact.cu", "common.cuh"),
-    "patch_salience": ("fused.cu", "patch.cu", "device_utils.cuh", "tmem_ld.cuh", "select_impl.cuh", "common.cuh"),
-    "patch_select": ("patch.cu", "select_impl.cuh", "common.cuh"),
+    "scoring": ("fused.cu", "device_utils.cuh", "tmem_ld.cuh", "tmem_plan.h", "select_impl.cuh", "common.cuh"),
+    "tail": ("step.cu", "select_impl.cuh", "device_utils.cuh", "common.cuh"),
 }
-NCU_DIGEST = {             # stage -> sha256 of its sources when the counters were taken
-    "salience": "ffd62393d650c2e5efee3b5134b9c65f706d6194bcd7bab2db45ab591ca9d630",
-    "select": "4d8d621fb08d123bffa8c27634f0c2082dc1552bbf6292d5b331160edb121b84",
-    "compact": "27d2a238f0b0e282dbdbc78fc8456f3149d3b82f90688d8421ddd0830ffa6299",
-    "patch_salience": "bc910990d2d34e5090584ef1d24d33ef11b19d0f6cdf72918256a3500f7fb1a7",
-    "patch_select": "5e9cc17fa3b0a30e57bac3560d78233fc067a917a9373740935fea78df45dbe6",
+NCU_DIGEST = {             # kernel -> sha256 of its sources when the counters were taken
+    "scoring": "a71c3115ca1764f705ff3678e2f5a0b2355be532b75a2b6072d1d27960b990c3",
+    "tail": "60146e73679a19356f1832da9a7b75ac1f7693a32fbd2861aed3e5506e23272a",
 }
-NCU_TRAFFIC = {             # (workload, stage) -> dram__bytes_read.sum + dram__bytes_write.sum per launch
-    ("config2", "salience"): 6621952,      # salience_fast_kernel<32,1>
-    ("config2", "select"): 76928,          # select_kernel<512>
-    ("config2", "compact"): 7085824,       # compact_kernel: the written half is still in L2 when the kernel ends
-    ("patch_mla", "salience"): 4518528 + 6316544,   # salience_fast_kernel<32,1> + patch_indicators_kernel
-    ("patch_mla", "select"): 62336,        # patch_select_kernel
+NCU_TRAFFIC = {             # (workload, kernel) -> dram__bytes_read.sum + dram__bytes_write.sum per launch
+    ("config2", "scoring"): 6628608,       # salience_fast_kernel<32,1>
+    ("config2", "tail"): 7135744,          # select_copy_kernel<512,1024>: the written half is still in L2 when the kernel ends
 }
 
 
@@ -83,12 +74,11 @@ def source_digest(files) -> str:
     return h.hexdigest()
 
 
-def ncu_traffic(workload: str, stage: str):
-    """Null once a source of the stage's kernels has changed since the counters were taken."""
-    key = ("patch_" + stage) if workload.startswith("patch") and stage != "compact" else stage
-    if key not in NCU_DIGEST or source_digest(NCU_SOURCES[key]) != NCU_DIGEST[key]:
+def ncu_traffic(workload: str, kernel: str):
+    """Null once a source of the kernel has changed since the counters were taken."""
+    if kernel not in NCU_DIGEST or source_digest(NCU_SOURCES[kernel]) != NCU_DIGEST[kernel]:
         return None
-    return NCU_TRAFFIC.get((workload, stage))
+    return NCU_TRAFFIC.get((workload, kernel))
 
 
 def make_workload(name: str):
@@ -471,6 +461,60 @@ def other_config(name, dev, world, hbm_gbs):
         h.torch.cuda.empty_cache()
 
 
+def episode_sharing(dev, T=16):
+    """Action-iteration episode with a fixed instruction and local visual drift (consecutive frames share most of
+    their content): serial step time and key-stream bytes with and without the reuse of the previous step's
+    logits.  Every step has device tensors of its own (16 x 43 MB: far beyond L2); one CUDA graph per episode."""
+    import torch
+    from paper_2604_09244_b200 import mvla, workloads as W
+    wl = W.config5_action_iteration(T=T, drift="visual_local")
+    s = wl.samples[0]
+    tens = [{n: mvla.to_device(getattr(t, n), wl.dtype, dev) for n in ("q", "k", "v", "hidden")} for t in wl.steps]
+    res = {}
+    for label, cache in (("full", 0), ("shared", 1)):
+        ctx = mvla.context_for(wl, logit_cache=cache)
+        outs = [ctx.alloc_outputs(wl.samples, extras=False) for _ in range(T)]
+
+        def episode():
+            for t in range(T):
+                d = tens[t]
+                ctx.prune_step(0, wl.samples, wl.mode, d["q"], d["k"], d["v"], d["hidden"], out=outs[t],
+                               flags=mvla.FLAG_RESET_STATE if t == 0 else 0,
+                               changed_rows=wl.extra["changed_rows"][t] if (cache and t > 0) else None)
+        episode()
+        torch.cuda.synchronize()
+        c0 = ctx.logit_cache_stats()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            episode()
+        c1 = ctx.logit_cache_stats()
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 40
+        a.record()
+        for _ in range(reps):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        res[label] = {"serial_us": a.elapsed_time(b) * 1e3 / (reps * T),
+                      "tiles_computed_per_step": (c1[0] - c0[0]) / T, "tiles_reused_per_step": (c1[1] - c0[1]) / T}
+        ctx.close()
+    e = 2
+    row = wl.n_heads * wl.head_dim * e                          # bytes of one key row
+    cols = (s.n_txt + 15) // 16 * 16
+    lrow = wl.n_heads * cols * 4                                # bytes of one key's cached logits
+    tiles = -(-s.n_2d // 128) + -(-s.n_3d // 128)
+    sh = res["shared"]
+    res["key_stream_bytes_per_step"] = {
+        "full": (s.n_2d + s.n_3d) * row,
+        "shared": int(sh["tiles_computed_per_step"] * 128 * (row + lrow) + sh["tiles_reused_per_step"] * 128 * lrow),
+        "note": f"{tiles} key tiles of 128; a computed tile reads its key rows and stores its logits, a reused tile reads "
+                "its logits; step 1 of the episode (cold start: every row is kept and copied) is in both means"}
+    return res
+
+
 def run_ours(args, rank, local, world):
     import torch
     from paper_2604_09244_b200 import mvla
@@ -483,9 +527,10 @@ def run_ours(args, rank, local, world):
 
     # ---- the headline: K steps one after another in one stream, every kernel waiting for the work before it
     # (what one request inside a prefill sees), device-resident inputs rotating over sets larger than L2
+    quick = dict(min_seconds=0.0, min_replays=2) if args.quick else {}
     with ClockSampler(local) as clk:
         ms, g_serial = h.timed_exact(0, K, W)
-        serial_dist = h.distribution(g_serial)
+        serial_dist = h.distribution(g_serial, **quick)
     ms_per_step = ms / K
     tokens_per_step = wl.total_vis * world
     value = tokens_per_step / (ms_per_step * 1e-3)
@@ -493,16 +538,16 @@ def run_ours(args, rank, local, world):
     # ---- independent requests overlapping inside the library (MVLA_FLAG_INPUTS_STABLE): the benchmark's inputs
     # are static buffers and its output sets rotate, so the promise behind the flag holds
     ms_o, g_over = h.timed_exact(mvla.FLAG_INPUTS_STABLE, K, W)
-    over_dist = h.distribution(g_over)
-    iso = h.isolated()
-    kt = h.kernel_times()
-    e2e_ms, h2d, d2h = h.e2e(max(20, min(K, 400)))
+    over_dist = h.distribution(g_over, **quick)
+    iso = h.isolated(8 if args.quick else 64)
+    kt = h.kernel_times(2 if args.quick else 20)
+    e2e_ms, h2d, d2h = h.e2e(5 if args.quick else max(20, min(K, 400)))
     e2e_value = tokens_per_step / (e2e_ms * 1e-3)
 
     peaks, peak_kind = measured_peaks()
     ab = algorithmic_bytes(wl, h.kept_rows)
     others = {}
-    if rank == 0 and world == 1 and args.workload == "config2" and not args.no_other_configs:
+    if rank == 0 and world == 1 and args.workload == "config2" and not args.no_other_configs and not args.quick:
         n_sets, per_graph, touched = h.n_sets, h.per_graph, h.touched
         alloc_mib = (h.in_bytes + h.out_bytes_alloc) * h.n_sets / 2**20
         launches = h.launches_per_step
@@ -511,6 +556,8 @@ def run_ours(args, rank, local, world):
         torch.cuda.empty_cache()
         for name in ("config3", "config4", "config5", "patch_mla"):
             others[name] = other_config(name, dev, world, peaks["hbm_gbs"])
+        others["config5_visual_local_logit_reuse"] = episode_sharing(dev)
+        torch.cuda.empty_cache()
     else:
         n_sets, per_graph, touched = h.n_sets, h.per_graph, h.touched
         alloc_mib = (h.in_bytes + h.out_bytes_alloc) * h.n_sets / 2**20
@@ -543,8 +590,8 @@ def run_ours(args, rank, local, world):
     step_gbs = ab["total"] / (ms_per_step * 1e-3) / 1e9
     over_us = ms_o * 1e3 / K
 
-    cpu_sec, cpu_n, cores = time_oracle(wl, 10 ** 6, 8.0)
-    cpu1_sec, cpu1_n, _ = time_oracle(wl, 10 ** 6, 6.0, threads=1)
+    cpu_sec, cpu_n, cores = time_oracle(wl, 10 ** 6, 0.5 if args.quick else 8.0)
+    cpu1_sec, cpu1_n, _ = time_oracle(wl, 10 ** 6, 0.5 if args.quick else 6.0, threads=1)
     line = {"metric": "visual_tokens_per_s_pruned", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": K, "warmup": W, "ms_per_step": ms_per_step,
             "latency_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -608,6 +655,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config2")
     ap.add_argument("--no-other-configs", action="store_true", help="skip the compact records of the other workloads")
+    ap.add_argument("--quick", action="store_true",
+                    help="short secondary measurements (for runs under a profiler; the headline still times --steps steps)")
     args = ap.parse_args()
 
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
