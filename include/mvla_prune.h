@@ -199,8 +199,10 @@ typedef struct mvla_outputs {
 
 /*
  * Create a context on cfg->device: workspace, smoothed state for n_prune_points x
- * n_state_slots episodes, a device status word.  Supported: dtype bf16 or fp32,
- * head_dim a multiple of 32 in [64, 256] (fp32 with head_dim 256: up to 32 text tokens), max_text <= 64, max_2d + max_3d <= 4096, max_batch <= 64.
+ * n_state_slots episodes, a device status word.  Supported: dtype bf16, fp32, or 8-bit e4m3 for q / k / v
+ * (MVLA_DTYPE_FP8_E4M3: tensor-core path only, hidden stays bf16, no patch path); head_dim a multiple of 32 in
+ * [64, 256] (fp32 with head_dim 256: up to 32 text tokens); max_text <= 64, max_2d + max_3d <= 4096,
+ * max_batch <= 64; logit_cache: tensor-core path, budgeted modes.
  * The library owns *out until mvla_prune_destroy.  (Alg. 1 "Input" / "Init".)
  * Errors: INVALID_ARG, UNSUPPORTED, OOM, CUDA (no usable device).
  */
