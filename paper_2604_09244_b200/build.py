@@ -12,7 +12,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libmvla_prune.so")
-SOURCES = ["api.cu", "salience.cu", "fused.cu", "select.cu", "compact.cu", "step.cu", "patch.cu", "salience_noalloc.cu"]
+SOURCES = ["api.cu", "salience.cu", "fused.cu", "select.cu", "compact.cu", "step.cu", "patch.cu", "patch_step.cu", "salience_noalloc.cu"]
 
 
 def _stale() -> bool:

@@ -37,8 +37,9 @@ struct mvla_ctx {
     unsigned long long* acc64;   // [kSets][max_batch * max_vis] fixed-point score accumulators, zero between
                                  // calls; the sets rotate from step to step (a step's scoring may run beside
                                  // the selections of the steps before it)
-    int32_t* tail_list;          // [kSets][max_batch * (max_text + max_vis)] kept list as the copying CTAs read it (-1 between launches)
-    size_t rows_all;             // max_batch * (max_text + max_vis)
+    int32_t* tail_list;          // [kSets][rows_all] kept list as the copying CTAs read it (-1 between launches)
+    unsigned long long* patch_rec;   // [kSets][vis_all / 2][3] hand-over words of the patch-by-patch tail (all ones between launches)
+    size_t rows_all;             // max_batch * (kHandWords + max_text + max_vis)
     int sm_count;                // multiprocessors of the device
     // reuse of the previous step's logits (cfg.logit_cache)
     float* lcache;               // [n_prune_points * n_slots][H][max_vis][cache_cols] raw dot products
@@ -160,7 +161,7 @@ int32_t make_plan(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_
             for (int b2 = b + 1; b2 < batch; ++b2)
                 if (samples[b].state_slot == samples[b2].state_slot) return MVLA_ERR_STATE;   // two writers of one state
     }
-    int32_t vis_off = 0, out_off = 0;
+    int32_t vis_off = 0, out_off = 0, cap_off = 0;
     for (int b = 0; b < batch; ++b) {
         const mvla_sample& in = samples[b];
         SampleDev d;
@@ -169,6 +170,8 @@ int32_t make_plan(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_
         d.off_2d = in.off_2d; d.n_2d = in.n_2d; d.off_3d = in.off_3d; d.n_3d = in.n_3d;
         const int nv = in.n_2d + in.n_3d;
         d.vis_off = vis_off;
+        d.cap_off = cap_off;
+        cap_off += kHandWords + in.n_txt + nv;
         vis_off += nv;
         d.k_2d_fixed = -1;
         d.cache_state = -1;
@@ -282,7 +285,7 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
                            const void* hidden, float* l1, unsigned long long* acc64, bool* used_acc64,
                            bool free_running, cudaStream_t st, AlphaOut alpha = AlphaOut{nullptr, 0, 0},
                            int32_t* rearm = nullptr, bool norms_beside = false, unsigned long long* stamps = nullptr,
-                           bool with_cache = false)
+                           bool with_cache = false, unsigned long long* rearm_rec = nullptr)
 {
     if (used_acc64) *used_acc64 = false;
     const mvla_config& c = ctx->cfg;
@@ -314,7 +317,7 @@ int32_t run_salience_chunk(mvla_ctx* ctx, const BatchDesc& bd, const void* q, co
         e = launch_salience_fast(bd, c.n_heads, c.n_heads / ctx->kv_heads, c.head_dim, static_cast<int>(ctx->qk_elem), tq, tk,
                                  tiles_per_cta, cluster, npad,
                                  alpha.ptr && !acc64 ? nullptr : ctx->part,     // the patch path reads the attention copy only
-                                 ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, rearm, stamps,
+                                 ctx->part_stride, acc64, ctx->status_dev, free_running, alpha, rearm, rearm_rec, stamps,
                                  with_cache ? ctx->lcache : nullptr, ctx->max_vis, ctx->cache_cols, st);
         if (used_acc64) *used_acc64 = acc64 != nullptr;
     } else {
@@ -601,6 +604,33 @@ int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, cons
     cudaStream_t side_stream = forked ? ctx->aux[par] : st;
     float* attn = out->attn ? out->attn : ctx->patch_attn_ws + set * ctx->vis_all;
     float* x = out->patch_x ? out->patch_x : ctx->patch_x_ws + set * (ctx->vis_all / 2 + 1) * 4;
+    const BatchDesc whole = chunk_of(plan, 0, std::min(batch, kMaxChunk));
+    if (!forked && batch <= kMaxChunk && chunk_is_fast(ctx, whole) && patch_tail_supported(whole)) {
+        // two kernels: scoring (leaves the attention copy, re-arms the hand-over words), then indicators,
+        // stages 1-4 and the row copy in one
+        int32_t* list = ctx->tail_list + par * ctx->rows_all;
+        unsigned long long* rec = ctx->patch_rec + par * (ctx->vis_all / 2 + 1) * 3;
+        const AlphaOut alpha = alpha_of(ctx, set);
+        rc = run_salience_chunk(ctx, whole, in->q, in->k, in->rows, nullptr, nullptr, nullptr, nullptr, false, st, alpha,
+                                list, false, nullptr, false, rec);
+        if (rc != MVLA_OK) return rc;
+        const PatchParams pp = patch_params(ctx);
+        PatchIO io;
+        std::memset(&io, 0, sizeof io);
+        io.rand_u = in->rand_u;
+        io.xhat_state = ctx->xhat_patch; io.xhat_out = out->patch_xhat; io.info_out = out->patch_info; io.diag = out->patch_diag;
+        int32_t* ws = ctx->nout_ws + set * (2 * static_cast<size_t>(ctx->cfg.max_batch) + 1);
+        io.counts = out->budgets; io.nout_ws = ws; io.ready_ws = ws + ctx->cfg.max_batch;
+        io.done_ws = ws + 2 * ctx->cfg.max_batch; io.status = ctx->status_dev;
+        io.kept_idx = out->kept_idx; io.out_offsets = out->out_offsets; io.batch_total = batch;
+        io.chunk_first = 0;
+        const cudaError_t e = launch_patch_tail(whole, ctx->cfg.n_heads, alpha, ctx->hidden_dtype, ctx->cfg.d_model, in->hidden,
+                                                x, attn, rec, pp, io, job, list, ctx->sm_count, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        commit_steps(ctx, prune_point, plan, samples);
+        if (total_kept_out) *total_kept_out = static_cast<int32_t>(cap);
+        return MVLA_OK;
+    }
     rc = run_patch_indicators(ctx, set, plan, batch, in->q, in->k, in->hidden, in->rows, attn, x, side_stream);
     if (rc != MVLA_OK) return rc;
     if (forked) {
@@ -680,6 +710,7 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     ctx->part = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
     ctx->acc64 = nullptr;
     ctx->tail_list = nullptr;
+    ctx->patch_rec = nullptr;
     ctx->sm_count = prop.multiProcessorCount;
     ctx->stage_event = nullptr;
     ctx->stamps = nullptr;
@@ -723,7 +754,7 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
     alloc(&ctx->mhat_state, 2 * n_state * 4);
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->acc64), kSets * vis_all * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(ctx->acc64, 0, kSets * vis_all * sizeof(unsigned long long));
-    ctx->rows_all = static_cast<size_t>(c.max_batch) * (c.max_text + ctx->max_vis);
+    ctx->rows_all = static_cast<size_t>(c.max_batch) * (kHandWords + c.max_text + ctx->max_vis);
     // (+ 1: a word that no launch ever writes, for mvla_selftest_wait_timeout)
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->tail_list), (kSets * ctx->rows_all + 1) * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->tail_list, 0xFF, (kSets * ctx->rows_all + 1) * sizeof(int32_t));
@@ -738,6 +769,9 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
         alloc(&ctx->xhat_patch, n_state * std::max(ctx->max_patch, 1) * 4);
         alloc(&ctx->patch_x_ws, (vis_all / 2 + 1) * 4 * ctx->patch_sets);
         alloc(&ctx->patch_attn_ws, vis_all * ctx->patch_sets);
+        const size_t nrec = kSets * (vis_all / 2 + 1) * 3 * sizeof(unsigned long long);
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->patch_rec), nrec);
+        if (e == cudaSuccess) e = cudaMemset(ctx->patch_rec, 0xFF, nrec);
         const size_t nws = (2 * static_cast<size_t>(c.max_batch) + 1) * sizeof(int32_t) * ctx->patch_sets;
         if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->nout_ws), nws);
         if (e == cudaSuccess) e = cudaMemset(ctx->nout_ws, 0, nws);
@@ -781,6 +815,7 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     cudaFree(ctx->mhat_state);
     cudaFree(ctx->acc64);
     cudaFree(ctx->tail_list);
+    cudaFree(ctx->patch_rec);
     cudaFree(ctx->lcache);
     cudaFree(ctx->alpha_ws);
     cudaFree(ctx->xhat_patch);

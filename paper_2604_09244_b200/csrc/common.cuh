@@ -10,6 +10,11 @@
 
 namespace mvla {
 
+// Hand-over words of the patch-by-patch tail, per sample from word cap_off on: kHandLines lines of 32 words
+// (identical copies, so that the copying CTAs do not all poll one line of the L2: word 0 "the list is about
+// to be written", word 1 the sample's first output row), then one word per row of the sample.
+constexpr int kHandLines = 8;
+constexpr int kHandWords = kHandLines * 32;
 constexpr int kMaxChunk = 32;        // samples carried by one launch (descriptors travel as kernel parameters)
 constexpr int kKeyTile = 128;        // visual keys per tile = rows of one MMA
 constexpr int kMaxCluster = 8;       // portable cluster size
@@ -22,6 +27,7 @@ constexpr unsigned kStampSlots = 4096;      // CTAs per kernel that leave time s
 struct SampleDev {
     int32_t seq_off, off_txt, n_txt, off_2d, n_2d, off_3d, n_3d;
     int32_t vis_off;        // offset of the sample in packed [sum n_vis] arrays
+    int32_t cap_off;        // sum of (kHandWords + n_txt + n_vis) over the samples before this one: its hand-over words in the patch-by-patch tail
     int32_t out_off;        // first output row
     int32_t n_out;          // kept rows = n_txt + budget
     int32_t budget;         // kept visual tokens (host known)
@@ -103,7 +109,9 @@ int sm_count_of_current_device();
 // `stamps`: when not null, CTA c (linear index, below kStampSlots) writes the global timer when it was free to
 // start its loads to stamps[2 c] and when it ended to stamps[2 c + 1].
 // `rearm`: when not null, words [out_off, out_off + n_out) of every sample are set to -1 (the kept list that
-// launch_select_copy's CTAs exchange, see there).
+// launch_select_copy's CTAs exchange, see there).  With `rearm_rec` (the patch-by-patch tail, launch_patch_tail)
+// it is words [cap_off, cap_off + kHandWords + n_txt + n_vis) instead, and the three 8-byte words of every patch in
+// `rearm_rec` ([vis_off / 2 + p][3]) are set to all ones.
 // Optional copy of the attention itself for the patch-by-patch path:
 // ptr[(h * stride_h) + (i * stride_i) + vis_off + j] = alpha[h, i, j]   (null: not written).
 struct AlphaOut {
@@ -118,7 +126,7 @@ bool fast_salience_supported(int tiles_per_cta);
 cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
-                                 bool free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* stamps,
+                                 bool free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* rearm_rec, unsigned long long* stamps,
                                  float* lcache, int cache_vis, int cache_cols, cudaStream_t stream);
 
 
@@ -226,5 +234,12 @@ cudaError_t launch_patch_indicators(const BatchDesc& bd, int n_heads, AlphaOut a
                                     const void* hidden, float* x_out, float* attn_out, cudaStream_t stream);
 // Stages 1-4 of Alg. 1 for every patch, output offsets over the batch, ordered kept-position lists.
 cudaError_t launch_patch_select(const BatchDesc& bd, const PatchParams& pp, const PatchIO& io, cudaStream_t stream);
+// Indicators, stages 1-4 and the row copy of the patch-by-patch step in one kernel behind the scoring kernel
+// (which must have re-armed `list` and `rec`, see launch_salience_fast).  `rec`: [sum P][3] 8-byte words;
+// `list`: 4-byte words, kHandWords + n_txt + n_vis per sample from cap_off on.  io.x / io.attn are not read.
+bool patch_tail_supported(const BatchDesc& bd);
+cudaError_t launch_patch_tail(const BatchDesc& bd, int n_heads, AlphaOut alpha, int dtype, int d_model, const void* hidden,
+                              float* x_out, float* attn_out, unsigned long long* rec, const PatchParams& pp, const PatchIO& io,
+                              const CompactJob& job, int32_t* list, int sm_count, cudaStream_t stream);
 
 }  // namespace mvla

@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(kFastThreads, 1)
 salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
                      const __grid_constant__ CUtensorMap tmap_k, int n_heads, int kv_group, int head_dim, int esize, int npad_max,
                      float* __restrict__ part, int64_t part_stride, unsigned long long* __restrict__ acc64,
-                     int* status, int free_running, const AlphaOut alpha, int32_t* __restrict__ rearm,
+                     int* status, int free_running, const AlphaOut alpha, int32_t* __restrict__ rearm, unsigned long long* __restrict__ rearm_rec,
                      unsigned long long* __restrict__ stamps, float* __restrict__ lcache, int cache_vis, int cache_cols)
 {
     constexpr int CC = TCOL * NTILE;
@@ -159,8 +159,14 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     pdl_trigger();
     // One CTA per sample re-arms the words through which the kernel after this one hands the kept list from
     // its selecting CTA to its copying CTAs (-1: not yet known).  Their last users finished long ago.
-    if (rearm && blockIdx.x == 0 && blockIdx.y == 0)
-        for (int i = tid; i < s.n_out; i += kFastThreads) rearm[s.out_off + i] = -1;
+    if (rearm && blockIdx.x == 0 && blockIdx.y == 0) {
+        if (!rearm_rec) {
+            for (int i = tid; i < s.n_out; i += kFastThreads) rearm[s.out_off + i] = -1;
+        } else {                              // the patch-by-patch tail: its list words, and three words per patch
+            for (int i = tid; i < kHandWords + s.n_txt + s.n_2d + s.n_3d; i += kFastThreads) rearm[s.cap_off + i] = -1;
+            for (int i = tid; i < 3 * s.n_2d; i += kFastThreads) rearm_rec[static_cast<int64_t>(s.vis_off / 2) * 3 + i] = ~0ull;
+        }
+    }
 
     if (tid == 0) {
         bool got = mbar_wait(bar_full, 0);
@@ -342,7 +348,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
 template <int TCOL, int NTILE>
 cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tq,
                           const CUtensorMap* tk, int cluster, int npad, float* part, int64_t part_stride,
-                          unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* stamps,
+                          unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* rearm_rec, unsigned long long* stamps,
                           float* lcache, int cache_vis, int cache_cols, cudaStream_t stream)
 {
     size_t smem = 1024 + static_cast<size_t>((head_dim * esize + 127) / 128) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
@@ -370,7 +376,7 @@ cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int he
     attr[1] = pdl_attribute();
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, kv_group, head_dim, esize, npad, part, part_stride, acc64, status, free_running, alpha, rearm, stamps, lcache, cache_vis, cache_cols);
+    return cudaLaunchKernelEx(&cfg, kern, bd, *tq, *tk, n_heads, kv_group, head_dim, esize, npad, part, part_stride, acc64, status, free_running, alpha, rearm, rearm_rec, stamps, lcache, cache_vis, cache_cols);
 }
 
 }  // namespace
@@ -380,14 +386,14 @@ bool fast_salience_supported(int tiles_per_cta) { return tiles_per_cta >= 1 && t
 cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tmap_q,
                                  const CUtensorMap* tmap_k, int tiles_per_cta, int cluster, int npad,
                                  float* part, int64_t part_stride, unsigned long long* acc64, int* status,
-                                 bool free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* stamps,
+                                 bool free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* rearm_rec, unsigned long long* stamps,
                                  float* lcache, int cache_vis, int cache_cols, cudaStream_t stream)
 {
     const int tcol = npad <= 16 ? 16 : (npad <= 32 ? 32 : 64);
 #define MVLA_FAST(TC, NTL)                                                                                      \
     if (tcol == TC && tiles_per_cta == NTL)                                                                     \
         return launch_fast_t<TC, NTL>(bd, n_heads, kv_group, head_dim, esize, tmap_q, tmap_k, cluster, npad, part, part_stride, \
-                                      acc64, status, free_running ? 1 : 0, alpha, rearm, stamps, lcache, cache_vis, cache_cols, stream);
+                                      acc64, status, free_running ? 1 : 0, alpha, rearm, rearm_rec, stamps, lcache, cache_vis, cache_cols, stream);
     MVLA_FAST(16, 1) MVLA_FAST(32, 1) MVLA_FAST(64, 1) MVLA_FAST(16, 2) MVLA_FAST(32, 2) MVLA_FAST(64, 2)
 #undef MVLA_FAST
     return cudaErrorInvalidConfiguration;
