@@ -475,16 +475,16 @@ int32_t validate_patch(const mvla_ctx* ctx, int32_t batch, const mvla_sample* sa
     return MVLA_OK;
 }
 
+// Layout of the attention copy: [head][visual token of the batch][text query, padded to whole 128-byte lines]
+int64_t alpha_row(const mvla_ctx* ctx) { return (static_cast<int64_t>(ctx->cfg.max_text) + 31) / 32 * 32; }
 size_t alpha_floats(const mvla_ctx* ctx)
 {
-    return static_cast<size_t>(ctx->cfg.n_heads) * ctx->cfg.max_text * ctx->vis_all;
+    return static_cast<size_t>(ctx->cfg.n_heads) * ctx->vis_all * static_cast<size_t>(alpha_row(ctx));
 }
 
 AlphaOut alpha_of(const mvla_ctx* ctx, unsigned set)
 {
-    return AlphaOut{ctx->alpha_ws + set * alpha_floats(ctx),
-                    static_cast<int64_t>(ctx->cfg.max_text) * static_cast<int64_t>(ctx->vis_all),
-                    static_cast<int64_t>(ctx->vis_all)};
+    return AlphaOut{ctx->alpha_ws + set * alpha_floats(ctx), static_cast<int64_t>(ctx->vis_all) * alpha_row(ctx), alpha_row(ctx)};
 }
 
 PatchParams patch_params(const mvla_ctx* ctx)
@@ -763,7 +763,7 @@ int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
         alloc(&ctx->lcache, n_state * static_cast<size_t>(c.n_heads) * ctx->max_vis * ctx->cache_cols);
     }
     if (c.patch_path) {
-        const size_t alpha_n = static_cast<size_t>(c.n_heads) * c.max_text * vis_all;
+        const size_t alpha_n = alpha_floats(ctx);
         ctx->patch_sets = alpha_n * sizeof(float) * kSets <= (size_t(1) << 30) ? kSets : 1;   // at most 1 GiB of attention copies
         alloc(&ctx->alpha_ws, alpha_n * ctx->patch_sets);
         alloc(&ctx->xhat_patch, n_state * std::max(ctx->max_patch, 1) * 4);

@@ -112,11 +112,13 @@ int sm_count_of_current_device();
 // launch_select_copy's CTAs exchange, see there).  With `rearm_rec` (the patch-by-patch tail, launch_patch_tail)
 // it is words [cap_off, cap_off + kHandWords + n_txt + n_vis) instead, and the three 8-byte words of every patch in
 // `rearm_rec` ([vis_off / 2 + p][3]) are set to all ones.
-// Optional copy of the attention itself for the patch-by-patch path:
-// ptr[(h * stride_h) + (i * stride_i) + vis_off + j] = alpha[h, i, j]   (null: not written).
+// Optional copy of the attention itself for the patch-by-patch path, the text queries of a (head, token)
+// next to one another (what the scoring kernel's thread holds, and what the indicators of a patch read):
+// ptr[(h * stride_h) + (vis_off + j) * stride_j + i] = alpha[h, i, j]   (null: not written).
+// stride_j is a multiple of 4 and ptr 16-byte aligned; entries i in [n_txt, stride_j) may be overwritten.
 struct AlphaOut {
     float* ptr;
-    int64_t stride_h, stride_i;
+    int64_t stride_h, stride_j;
 };
 
 bool fast_salience_supported(int tiles_per_cta);

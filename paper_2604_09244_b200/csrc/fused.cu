@@ -72,7 +72,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     extern __shared__ uint8_t dyn_smem_raw[];
     uint8_t* dyn_smem = dyn_smem_raw + ((1024u - (smem_u32(dyn_smem_raw) & 1023u)) & 1023u);   // swizzle atoms are 1 KB
     __shared__ float s_m[kMaxText];                       // local max per query (scaled, log2 domain), -inf replaced by 0
-    __shared__ float s_w[kMaxText];                       // final weight per query
+    __shared__ alignas(16) float s_w[kMaxText];           // final weight per query
     __shared__ float2 s_peer[kMaxCluster][kMaxText];      // (raw local max, local sum) of every CTA of the cluster
     __shared__ float2 s_loc[kMaxText];                    // this CTA's pairs, staged for the push
     __shared__ float s_wred[4][kMaxText];
@@ -326,12 +326,17 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
                 atomicAdd(acc64 + s.vis_off + vis0[t] + tid, __float2ull_rn(acc * kFixScale));
             else if (part)                    // neither: the caller wants the attention copy only
                 part[static_cast<int64_t>(h) * part_stride + s.vis_off + vis0[t] + tid] = acc;
-            if (alpha.ptr) {              // the attention itself, for the per-patch indicators (coalesced over keys)
-                float* ap = alpha.ptr + static_cast<int64_t>(h) * alpha.stride_h + s.vis_off + vis0[t] + tid;
+            if (alpha.ptr) {              // the attention itself, for the per-patch indicators: this key's row of queries
+                float4* ap = reinterpret_cast<float4*>(alpha.ptr + static_cast<int64_t>(h) * alpha.stride_h +
+                                                       static_cast<int64_t>(s.vis_off + vis0[t] + tid) * alpha.stride_j);
                 const float hn = static_cast<float>(n_heads) * static_cast<float>(s.n_txt);   // s_w carries 1 / (H n_t)
 #pragma unroll
-                for (int i = 0; i < TCOL; ++i)
-                    if (i < s.n_txt) ap[static_cast<int64_t>(i) * alpha.stride_i] = L[t * TCOL + i] * s_w[i] * hn;
+                for (int g4 = 0; g4 < TCOL / 4; ++g4) {   // 16-byte stores: a handful of instructions (s_w is 0 past the text queries)
+                    if (4 * g4 >= npad || 4 * g4 >= alpha.stride_j) break;
+                    const float4 w4 = *reinterpret_cast<const float4*>(&s_w[4 * g4]);
+                    ap[g4] = make_float4(L[t * TCOL + 4 * g4] * w4.x * hn, L[t * TCOL + 4 * g4 + 1] * w4.y * hn,
+                                         L[t * TCOL + 4 * g4 + 2] * w4.z * hn, L[t * TCOL + 4 * g4 + 3] * w4.w * hn);
+                }
             }
         }
     }

@@ -22,7 +22,7 @@ patch_indicators_kernel(const __grid_constant__ BatchDesc bd, int n_heads, const
                         const T* __restrict__ hidden, int d_model, float* __restrict__ x_out,
                         float* __restrict__ attn_out)
 {
-    patch_indicators_block<T, PP>(bd.s[blockIdx.y], blockIdx.x, n_heads, alpha, hidden, d_model, x_out, attn_out, nullptr);
+    patch_indicators_block<T, PP>(bd.s[blockIdx.y], blockIdx.x, n_heads, alpha, hidden, d_model, x_out, attn_out, nullptr, true);
 }
 
 // grid = samples

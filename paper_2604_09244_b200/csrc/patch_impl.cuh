@@ -44,7 +44,7 @@ __device__ __forceinline__ unsigned long long ld_relaxed_gpu_u64(const unsigned 
 template <typename T, int PP>
 __device__ __forceinline__ void patch_indicators_block(const SampleDev& s, int blk, int n_heads, const AlphaOut& alpha,
                                                        const T* __restrict__ hidden, int d_model, float* __restrict__ x_out,
-                                                       float* __restrict__ attn_out, unsigned long long* __restrict__ rec)
+                                                       float* __restrict__ attn_out, unsigned long long* __restrict__ rec, bool norms_early)
 {
     constexpr int kIndPatches = PP;
     constexpr int kIndGroups = kIndThreads / PP;          // groups of (head, query) pairs
@@ -61,39 +61,48 @@ __device__ __forceinline__ void patch_indicators_block(const SampleDev& s, int b
     const int p = p0 + pl;
     const bool live = p < P;
     const int npairs = n_heads * s.n_txt;
-    const float* base = alpha.ptr + s.vis_off + p;
+    const float* base = alpha.ptr + static_cast<int64_t>(s.vis_off + p) * alpha.stride_j;   // the patch's 2D token; its 3D token is P rows on
+    const int64_t to3 = static_cast<int64_t>(P) * alpha.stride_j;
 
-    // ---- feature norms: row r of the CTA = 2D token p0 + r (r < PP) or 3D token p0 + r - PP
-    {
-        const int r = tid / kRowThreads, within = tid % kRowThreads;
-        const int pr = p0 + (r & (kIndPatches - 1));
-        float acc = 0.f;
-        if (pr < P) {
-            const int row = s.seq_off + (r < kIndPatches ? s.off_2d : s.off_3d) + pr;
-            constexpr int kVec = 16 / sizeof(T);
-            const uint4* src = reinterpret_cast<const uint4*>(hidden + static_cast<int64_t>(row) * d_model);
-            const int nvec = d_model / kVec;
-#pragma unroll 8
-            for (int i = within; i < nvec; i += kRowThreads) {
-                const uint4 u = __ldg(src + i);
-                if constexpr (sizeof(T) == 2) {
-                    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+    // ---- feature norms: row r of the CTA = 2D token p0 + r (r < PP) or 3D token p0 + r - PP.  The first
+    //      kNormKeep 16-byte pieces of a thread are loaded here and added up further down, once the loads of
+    //      the attention copy are in flight too.  `norms_early`: issue them before the wait for the kernel
+    //      before this one (they do not depend on it), else after it -- beside a scoring kernel in the middle
+    //      of its own stores the early loads were seen to cost that kernel more than they save here.
+    constexpr int kNormKeep = 8;
+    constexpr int kVec = 16 / sizeof(T);
+    const int nr = tid / kRowThreads, within = tid % kRowThreads;
+    const int pr = p0 + (nr & (kIndPatches - 1));
+    const int nvec = d_model / kVec;
+    const uint4* nsrc = nullptr;
+    if (pr < P)
+        nsrc = reinterpret_cast<const uint4*>(hidden + static_cast<int64_t>(s.seq_off + (nr < kIndPatches ? s.off_2d : s.off_3d) + pr) * d_model);
+    uint4 hv[kNormKeep];
+    auto norm_loads = [&]() {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        acc += fabsf(__uint_as_float(w[e] << 16));           // low bf16
-                        acc += fabsf(__uint_as_float(w[e] & 0xFFFF0000u));   // high bf16
-                    }
-                } else {
-                    acc += fabsf(__uint_as_float(u.x)) + fabsf(__uint_as_float(u.y)) +
-                           fabsf(__uint_as_float(u.z)) + fabsf(__uint_as_float(u.w));
-                }
-            }
+        for (int k = 0; k < kNormKeep; ++k) {
+            const int i = within + k * kRowThreads;
+            hv[k] = (nsrc && i < nvec) ? __ldg(nsrc + i) : make_uint4(0u, 0u, 0u, 0u);
         }
+    };
+    auto abs_sum = [](const uint4& u) {
+        if constexpr (sizeof(T) == 2) {
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+            float a = 0.f;
 #pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if (lane == 0) rown[warp] = acc;                  // read after the barriers of the first reduction
-    }
+            for (int e = 0; e < 4; ++e) {
+                a += fabsf(__uint_as_float(w[e] << 16));           // low bf16
+                a += fabsf(__uint_as_float(w[e] & 0xFFFF0000u));   // high bf16
+            }
+            return a;
+        } else {
+            return fabsf(__uint_as_float(u.x)) + fabsf(__uint_as_float(u.y)) +
+                   fabsf(__uint_as_float(u.z)) + fabsf(__uint_as_float(u.w));
+        }
+    };
+    if (norms_early) norm_loads();
     asm volatile("griddepcontrol.wait;" ::: "memory");    // the attention copy comes from the kernel before this one
+    if (!norms_early) norm_loads();
 
     // Sum over the lanes of a warp that hold the same patch (the lane bits above log2 PP), then over the
     // warps in a fixed order: tot[patch][c].
@@ -124,18 +133,34 @@ __device__ __forceinline__ void patch_indicators_block(const SampleDev& s, int b
     constexpr int kKeep = 16;
     float r2[kKeep], r3[kKeep];
     float v[4] = {0.f, 0.f, 0.f, 0.f};
+    const int nq = min(kKeep, (npairs + kIndGroups - 1) / kIndGroups);   // block-uniform: slots in use
+    // pair idx = g + q kIndGroups is (head h, query i); stepping q moves (h, i) by a fixed amount
+    const int step_h = kIndGroups / s.n_txt, step_i = kIndGroups - step_h * s.n_txt;
+    int h = g / s.n_txt, i = g - h * s.n_txt;
 #pragma unroll
     for (int q = 0; q < kKeep; ++q) {                     // all loads of the thread in flight at once
-        const int idx = g + q * kIndGroups;
         r2[q] = 0.f; r3[q] = 0.f;
-        if (live && idx < npairs) {
-            const int h = idx / s.n_txt, i = idx - h * s.n_txt;
-            const float* a = base + static_cast<int64_t>(h) * alpha.stride_h + static_cast<int64_t>(i) * alpha.stride_i;
-            r2[q] = __ldcg(a); r3[q] = __ldcg(a + P);
+        if (q >= nq) continue;                            // uniform
+        if (live && g + q * kIndGroups < npairs) {
+            const float* a = base + static_cast<int64_t>(h) * alpha.stride_h + i;
+            r2[q] = __ldcg(a); r3[q] = __ldcg(a + to3);
         }
+        h += step_h; i += step_i;
+        if (i >= s.n_txt) { i -= s.n_txt; ++h; }
+    }
+    {                                                     // the feature norms, now that every load is in flight
+        float acc = 0.f;
+#pragma unroll
+        for (int k = 0; k < kNormKeep; ++k) acc += abs_sum(hv[k]);
+        if (nsrc)
+            for (int k = within + kNormKeep * kRowThreads; k < nvec; k += kRowThreads) acc += abs_sum(__ldg(nsrc + k));
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (lane == 0) rown[warp] = acc;                  // read after the barriers of the first reduction
     }
 #pragma unroll
     for (int q = 0; q < kKeep; ++q) {                     // (a pair that does not exist adds zeros)
+        if (q >= nq) break;                               // uniform
         v[0] = fmaf(r3[q], r2[q], v[0]);
         v[1] = fmaf(r2[q], r2[q], v[1]);
         v[2] += fabsf(r2[q]);
@@ -144,9 +169,9 @@ __device__ __forceinline__ void patch_indicators_block(const SampleDev& s, int b
     if (live) {
 #pragma unroll 4
         for (int idx = g + kKeep * kIndGroups; idx < npairs; idx += kIndGroups) {
-            const int h = idx / s.n_txt, i = idx - h * s.n_txt;
-            const float* a = base + static_cast<int64_t>(h) * alpha.stride_h + static_cast<int64_t>(i) * alpha.stride_i;
-            const float a2 = __ldcg(a), a3 = __ldcg(a + P);
+            const int hh = idx / s.n_txt, ii = idx - hh * s.n_txt;
+            const float* a = base + static_cast<int64_t>(hh) * alpha.stride_h + ii;
+            const float a2 = __ldcg(a), a3 = __ldcg(a + to3);
             v[0] = fmaf(a3, a2, v[0]);
             v[1] = fmaf(a2, a2, v[1]);
             v[2] += fabsf(a2);
@@ -160,13 +185,16 @@ __device__ __forceinline__ void patch_indicators_block(const SampleDev& s, int b
     // pass 2: || a3 - coef a2 ||_1, the part of the 3D token's attention that the 2D token's does not explain
     float o[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int q = 0; q < kKeep; ++q) o[0] += fabsf(fmaf(-coef, r2[q], r3[q]));
+    for (int q = 0; q < kKeep; ++q) {
+        if (q >= nq) break;                               // uniform
+        o[0] += fabsf(fmaf(-coef, r2[q], r3[q]));
+    }
     if (live) {
 #pragma unroll 4
         for (int idx = g + kKeep * kIndGroups; idx < npairs; idx += kIndGroups) {
-            const int h = idx / s.n_txt, i = idx - h * s.n_txt;
-            const float* a = base + static_cast<int64_t>(h) * alpha.stride_h + static_cast<int64_t>(i) * alpha.stride_i;
-            o[0] += fabsf(fmaf(-coef, __ldcg(a), __ldcg(a + P)));
+            const int hh = idx / s.n_txt, ii = idx - hh * s.n_txt;
+            const float* a = base + static_cast<int64_t>(hh) * alpha.stride_h + ii;
+            o[0] += fabsf(fmaf(-coef, __ldcg(a), __ldcg(a + to3)));
         }
     }
     reduce(o, 1);
@@ -200,7 +228,10 @@ template <int NT>
 struct PatchSmemT {
     double mass[kMaxPatch];                 // attention mass of every patch (what K-Means clusters)
     uint8_t label[kMaxPatch];
-    uint8_t keep[2 * kMaxPatch];            // keep flags in visual order: 2D tokens, then 3D tokens
+    union {                                 // one after the other in time:
+        float massf[kMaxPatch];             //   the masses rounded to fp32 (first look of the K-Means assignment)
+        uint8_t keep[2 * kMaxPatch];        //   keep flags in visual order: 2D tokens, then 3D tokens (written after the K-Means)
+    };
     float2 share[kMaxPatch];                // smoothed attention shares of every patch (M^S2_2D, M^S2_3D)
     double mu[2];                           // their means over the patches (the baselines of the robot rule)
     float thr[8];                           // the thresholds of stages 2-3 as fp32 numbers that decide like the doubles
@@ -289,7 +320,6 @@ __device__ __forceinline__ void patch_select_block(const SampleDev& s, int b_loc
                     w0 = ld_relaxed_gpu_u64(r); w1 = ld_relaxed_gpu_u64(r + 1); w2 = ld_relaxed_gpu_u64(r + 2);
                     if (w0 != ~0ull && w1 != ~0ull && w2 != ~0ull) break;
                     if ((it & 63u) == 63u && global_ns() - t_start > 1000000000ull) break;
-                    __nanosleep(40);
                 }
                 ok &= w0 != ~0ull && w1 != ~0ull && w2 != ~0ull;
                 x[e] = make_float4(__uint_as_float(static_cast<unsigned>(w0)), __uint_as_float(static_cast<unsigned>(w0 >> 32)),
@@ -319,7 +349,9 @@ __device__ __forceinline__ void patch_select_block(const SampleDev& s, int b_loc
             if (s.update_state) state[p] = v;
             if (io.xhat_out) reinterpret_cast<float4*>(io.xhat_out)[pat_off + p] = v;
             // the patch's attention response: the mass of its two tokens
-            sm.mass[p] = static_cast<double>(a2[e]) + static_cast<double>(a3[e]);
+            const double m = static_cast<double>(a2[e]) + static_cast<double>(a3[e]);
+            sm.mass[p] = m;
+            sm.massf[p] = static_cast<float>(m);
             sm.label[p] = 255;
             sm.share[p] = make_float2(v.z, v.w);
         }
@@ -370,13 +402,27 @@ __device__ __forceinline__ void patch_select_block(const SampleDev& s, int b_loc
             int changed = 0;
             double s0 = 0.0, s1 = 0.0, s2 = 0.0;
             int n0 = 0, n1 = 0, n2 = 0;
+            // Nearest centre.  fp32 decides wherever it can be sure: with m and the centres rounded to fp32
+            // a distance is off by at most 2^-23 (m + c), so a comparison of two distances whose fp32 values
+            // differ by more than `tol` comes out as in double; anything closer (ties included) is redone
+            // in double.  Class sums stay in double.
+            const float f0 = static_cast<float>(c0), f1 = static_cast<float>(c1), f2 = static_cast<float>(c2);
             for (int p = lane; p < P; p += 32) {
                 const double m = sm.mass[p];
-                int best = 0;
-                double bdist = fabs(m - c0);
-                const double d1 = fabs(m - c1), d2 = fabs(m - c2);
-                if (d1 < bdist) { bdist = d1; best = 1; }
-                if (d2 < bdist) { bdist = d2; best = 2; }
+                const float mf = sm.massf[p];
+                const float tol = 4e-7f * (fabsf(mf) + fmaxf(fabsf(f0), fmaxf(fabsf(f1), fabsf(f2))));
+                const float e0 = fabsf(mf - f0), e1 = fabsf(mf - f1), e2 = fabsf(mf - f2);
+                int best = e1 < e0 ? 1 : 0;
+                const float eb = fminf(e0, e1);
+                bool sure = fabsf(e1 - e0) > tol && fabsf(e2 - eb) > tol;
+                if (e2 < eb) best = 2;
+                if (!sure) {
+                    best = 0;
+                    double bdist = fabs(m - c0);
+                    const double d1 = fabs(m - c1), d2 = fabs(m - c2);
+                    if (d1 < bdist) { bdist = d1; best = 1; }
+                    if (d2 < bdist) { bdist = d2; best = 2; }
+                }
                 if (sm.label[p] != best) { sm.label[p] = static_cast<uint8_t>(best); changed = 1; }
                 s0 += best == 0 ? m : 0.0; n0 += best == 0;
                 s1 += best == 1 ? m : 0.0; n1 += best == 1;

@@ -35,7 +35,7 @@ patch_tail_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ 
     if (c < n_ind) {
         int b = 0;
         while (b + 1 < bd.n && c >= tp.ind0[b + 1]) ++b;
-        patch_indicators_block<T, PP>(bd.s[b], c - tp.ind0[b], n_heads, alpha, hidden, d_model, x_out, attn_out, rec);
+        patch_indicators_block<T, PP>(bd.s[b], c - tp.ind0[b], n_heads, alpha, hidden, d_model, x_out, attn_out, rec, true);
         return;
     }
     c -= n_ind;

@@ -265,8 +265,8 @@ salience_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CU
                     const float pr = (cb + i < s.n_txt) ? e * s_w[cb + i] : 0.f;
                     acc += pr;
                     if (alpha.ptr && cb + i < s.n_txt && tid < ti.valid)   // the attention itself (per-patch indicators)
-                        alpha.ptr[static_cast<int64_t>(h) * alpha.stride_h + static_cast<int64_t>(cb + i) * alpha.stride_i +
-                                  s.vis_off + ti.vis0 + tid] = pr * (static_cast<float>(n_heads) * static_cast<float>(s.n_txt));
+                        alpha.ptr[static_cast<int64_t>(h) * alpha.stride_h + static_cast<int64_t>(s.vis_off + ti.vis0 + tid) * alpha.stride_j +
+                                  cb + i] = pr * (static_cast<float>(n_heads) * static_cast<float>(s.n_txt));
                 }
             }
         }
