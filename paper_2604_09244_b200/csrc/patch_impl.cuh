@@ -365,7 +365,8 @@ __device__ __forceinline__ void patch_select_block(const SampleDev& s, int b_loc
     if (warp == 0) {
         double sum_m = 0.0, sum_z = 0.0, sum_w = 0.0;
         long long mx = 0, mn = 0x7FF0000000000000ll;             // masses are >= 0: their bit patterns order like the values
-        for (int p = lane; p < P; p += 32) {
+#pragma unroll 8
+        for (int p = lane; p < P; p += 32) {                      // (unrolled: the shared-memory loads of eight patches overlap)
             const double m = sm.mass[p];
             const float2 zw = sm.share[p];
             sum_m += m;
@@ -407,6 +408,7 @@ __device__ __forceinline__ void patch_select_block(const SampleDev& s, int b_loc
             // differ by more than `tol` comes out as in double; anything closer (ties included) is redone
             // in double.  Class sums stay in double.
             const float f0 = static_cast<float>(c0), f1 = static_cast<float>(c1), f2 = static_cast<float>(c2);
+#pragma unroll 8
             for (int p = lane; p < P; p += 32) {
                 const double m = sm.mass[p];
                 const float mf = sm.massf[p];
