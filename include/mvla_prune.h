@@ -288,7 +288,8 @@ int32_t mvla_logit_cache_stats(mvla_ctx *ctx, int64_t *tiles_computed, int64_t *
  * between two kernels of a step removes their overlap and costs microseconds inside a CUDA graph, so it
  * cannot time them as the step runs them; a handful of stores of the global nanosecond timer can.  While
  * `device_buffer` (device memory, 2 x 4096 x 2 uint64, zero-filled by the caller; null switches it off) is
- * set, every non-overlapped mvla_prune_step on shapes the fused kernels cover makes CTA c (linear index,
+ * set, every non-overlapped mvla_prune_step of the budgeted modes (MVLA_MODE_PATCH steps take no stamps) on
+ * shapes the fused kernels cover makes CTA c (linear index,
  * c < 4096) of its scoring kernel write buffer[0][c][0] = the time it was free to start its loads (its
  * predecessor complete) and buffer[0][c][1] = the time it ended, and CTA c of its selection + row-copy kernel
  * the same into buffer[1][c][..] (start: past its wait for the scoring kernel; the selecting CTAs, which come
