@@ -58,17 +58,24 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
     return false;
 }
 
-// grid = (cluster size, n_heads, samples), cluster = (cluster size, 1, 1), 128 threads.
+// grid = (cluster size, n_heads, samples), cluster = (cluster size, 1, 1), 128 x SPLIT threads.
 // TCOL: tensor-memory columns per tile (>= padded query count); NTILE: key tiles per CTA.
-template <int TCOL, int NTILE>
-__global__ void __launch_bounds__(kFastThreads, 1)
+// SPLIT: threads per key.  1: a thread holds all the logits of its key.  2 (fixed-point accumulators only, no
+// attention copy): threads t and t + 128 hold one half of the text queries each -- the chain through max,
+// exponentials, sums and weighted sum is half as long per warp, and a scheduler has two warps to alternate
+// between; both halves add into the key's accumulator.
+template <int TCOL, int NTILE, int SPLIT>
+__global__ void __launch_bounds__(kFastThreads * SPLIT, 1)
 salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ CUtensorMap tmap_q,
                      const __grid_constant__ CUtensorMap tmap_k, int n_heads, int kv_group, int head_dim, int esize, int npad_max,
                      float* __restrict__ part, int64_t part_stride, unsigned long long* __restrict__ acc64,
                      int* status, int free_running, const AlphaOut alpha, int32_t* __restrict__ rearm, unsigned long long* __restrict__ rearm_rec,
                      unsigned long long* __restrict__ stamps, float* __restrict__ lcache, int cache_vis, int cache_cols)
 {
-    constexpr int CC = TCOL * NTILE;
+    constexpr int CC = TCOL * NTILE;                      // tensor-memory columns of the CTA
+    constexpr int TC = TCOL / SPLIT;                      // columns (text queries) of a tile that one thread holds
+    constexpr int NT = kFastThreads * SPLIT;
+    static_assert(TC % 16 == 0, "a thread holds whole groups of 16 queries");
     extern __shared__ uint8_t dyn_smem_raw[];
     uint8_t* dyn_smem = dyn_smem_raw + ((1024u - (smem_u32(dyn_smem_raw) & 1023u)) & 1023u);   // swizzle atoms are 1 KB
     __shared__ float s_m[kMaxText];                       // local max per query (scaled, log2 domain), -inf replaced by 0
@@ -82,6 +89,9 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     const SampleDev& s = bd.s[blockIdx.z];
     const int h = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int key = tid & (kFastThreads - 1);            // key of the tile(s) this thread works on
+    const int kwarp = warp & 3;                           // its warp among the four that cover the 128 keys (= tensor-memory lane quarter)
+    const int c0 = (tid / kFastThreads) * TC;             // first of its text queries
     // queries padded to the MMA's N granularity for THIS sample (the launch is sized for the longest text)
     const int npad = min(npad_max, (s.n_txt + 15) & ~15);
     const uint32_t crank = cluster_ctarank();
@@ -161,10 +171,10 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     // its selecting CTA to its copying CTAs (-1: not yet known).  Their last users finished long ago.
     if (rearm && blockIdx.x == 0 && blockIdx.y == 0) {
         if (!rearm_rec) {
-            for (int i = tid; i < s.n_out; i += kFastThreads) rearm[s.out_off + i] = -1;
+            for (int i = tid; i < s.n_out; i += NT) rearm[s.out_off + i] = -1;
         } else {                              // the patch-by-patch tail: its list words, and three words per patch
-            for (int i = tid; i < kHandWords + s.n_txt + s.n_2d + s.n_3d; i += kFastThreads) rearm[s.cap_off + i] = -1;
-            for (int i = tid; i < 3 * s.n_2d; i += kFastThreads) rearm_rec[static_cast<int64_t>(s.vis_off / 2) * 3 + i] = ~0ull;
+            for (int i = tid; i < kHandWords + s.n_txt + s.n_2d + s.n_3d; i += NT) rearm[s.cap_off + i] = -1;
+            for (int i = tid; i < 3 * s.n_2d; i += NT) rearm_rec[static_cast<int64_t>(s.vis_off / 2) * 3 + i] = ~0ull;
         }
     }
 
@@ -202,28 +212,38 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     tc_fence_after();
 
     // ---- all logits of this thread's key(s) into registers, scaled to the log2 domain, masked
-    float L[CC];
+    float L[NTILE * TC];                      // L[t * TC + i]: tile t, text query c0 + i
     if (any_live && ok) {
-        tmem_ld_cols<CC>(tmem_base + (static_cast<uint32_t>(warp * 32) << 16), L);
+        if constexpr (SPLIT == 1) {
+            tmem_ld_cols<CC>(tmem_base + (static_cast<uint32_t>(kwarp * 32) << 16), L);
+        } else {
+#pragma unroll
+            for (int t = 0; t < NTILE; ++t) {
+                float part_l[TC];
+                tmem_ld_cols<TC>(tmem_base + static_cast<uint32_t>(t * TCOL + c0) + (static_cast<uint32_t>(kwarp * 32) << 16), part_l);
+#pragma unroll
+                for (int i = 0; i < TC; ++i) L[t * TC + i] = part_l[i];
+            }
+        }
     } else {
 #pragma unroll
-        for (int i = 0; i < CC; ++i) L[i] = 0.f;
+        for (int i = 0; i < NTILE * TC; ++i) L[i] = 0.f;
     }
     // Logit cache: a computed tile leaves its raw dot products for the next action step, a reused tile takes
     // the previous step's instead (128 bytes per key and head at 32 queries: half a key row, and no MMA).
     if (caching && ok) {
 #pragma unroll
         for (int t = 0; t < NTILE; ++t) {
-            if (tid >= valid[t]) continue;
-            float4* row = reinterpret_cast<float4*>(lcache + cache_row0 + static_cast<int64_t>(vis0[t] + tid) * cache_cols);
+            if (key >= valid[t]) continue;
+            float4* row = reinterpret_cast<float4*>(lcache + cache_row0 + static_cast<int64_t>(vis0[t] + key) * cache_cols + c0);
 #pragma unroll
-            for (int i = 0; i < TCOL / 4; ++i) {
-                if (4 * i >= npad) break;
+            for (int i = 0; i < TC / 4; ++i) {
+                if (c0 + 4 * i >= npad) break;
                 if (from_k[t]) {
-                    row[i] = make_float4(L[t * TCOL + 4 * i], L[t * TCOL + 4 * i + 1], L[t * TCOL + 4 * i + 2], L[t * TCOL + 4 * i + 3]);
+                    row[i] = make_float4(L[t * TC + 4 * i], L[t * TC + 4 * i + 1], L[t * TC + 4 * i + 2], L[t * TC + 4 * i + 3]);
                 } else {
                     const float4 v = __ldcg(row + i);
-                    L[t * TCOL + 4 * i] = v.x; L[t * TCOL + 4 * i + 1] = v.y; L[t * TCOL + 4 * i + 2] = v.z; L[t * TCOL + 4 * i + 3] = v.w;
+                    L[t * TC + 4 * i] = v.x; L[t * TC + 4 * i + 1] = v.y; L[t * TC + 4 * i + 2] = v.z; L[t * TC + 4 * i + 3] = v.w;
                 }
             }
         }
@@ -234,24 +254,24 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
 #pragma unroll
     for (int t = 0; t < NTILE; ++t) {
         if (ok && valid[t] == kKeyTile) continue;         // block-uniform
-        const bool live = ok && tid < valid[t];
+        const bool live = ok && key < valid[t];
 #pragma unroll
-        for (int i = 0; i < TCOL; ++i) L[t * TCOL + i] = live ? L[t * TCOL + i] : -CUDART_INF_F;
+        for (int i = 0; i < TC; ++i) L[t * TC + i] = live ? L[t * TC + i] : -CUDART_INF_F;
     }
 
     // ---- local maximum per query
 #pragma unroll
-    for (int qc = 0; qc < TCOL / 16; ++qc) {
-        if (qc * 16 >= npad) break;
+    for (int qc = 0; qc < TC / 16; ++qc) {
+        if (c0 + qc * 16 >= npad) break;
         float m[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
             m[i] = L[qc * 16 + i];
 #pragma unroll
-            for (int t = 1; t < NTILE; ++t) m[i] = fmaxf(m[i], L[t * TCOL + qc * 16 + i]);
+            for (int t = 1; t < NTILE; ++t) m[i] = fmaxf(m[i], L[t * TC + qc * 16 + i]);
         }
         const float red = warp_reduce16<true>(m, lane);
-        if ((lane & 1) == 0) s_wred[warp][qc * 16 + col16(lane)] = red;
+        if ((lane & 1) == 0) s_wred[kwarp][c0 + qc * 16 + col16(lane)] = red;
     }
     __syncthreads();
     float m_raw = -CUDART_INF_F;
@@ -263,22 +283,22 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
 
     // ---- exponentials (kept in registers) and the local denominator per query
 #pragma unroll
-    for (int qc = 0; qc < TCOL / 16; ++qc) {
-        if (qc * 16 >= npad) break;
+    for (int qc = 0; qc < TC / 16; ++qc) {
+        if (c0 + qc * 16 >= npad) break;
         float sum[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-            const float mm = s_m[qc * 16 + i];
+            const float mm = s_m[c0 + qc * 16 + i];
             sum[i] = 0.f;
 #pragma unroll
             for (int t = 0; t < NTILE; ++t) {
-                const float e = ex2_approx(fmaf(L[t * TCOL + qc * 16 + i], cscale, -mm));
-                L[t * TCOL + qc * 16 + i] = e;
+                const float e = ex2_approx(fmaf(L[t * TC + qc * 16 + i], cscale, -mm));
+                L[t * TC + qc * 16 + i] = e;
                 sum[i] += e;
             }
         }
         const float red = warp_reduce16<false>(sum, lane);
-        if ((lane & 1) == 0) s_wred[warp][qc * 16 + col16(lane)] = red;
+        if ((lane & 1) == 0) s_wred[kwarp][c0 + qc * 16 + col16(lane)] = red;
     }
     __syncthreads();
 
@@ -287,7 +307,7 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         s_loc[tid] = make_float2(m_raw, (s_wred[0][tid] + s_wred[1][tid]) + (s_wred[2][tid] + s_wred[3][tid]));
     __syncthreads();
     cluster_wait_acquire();                   // every peer is running and has initialised its barriers
-    for (int p = tid; p < npad * static_cast<int>(csize); p += kFastThreads) {
+    for (int p = tid; p < npad * static_cast<int>(csize); p += NT) {
         const int i = p % npad;
         const uint32_t r = static_cast<uint32_t>(p / npad);
         st_async_peer_f32x2(smem_u32(&s_peer[crank][i]), bar_x, r, s_loc[i]);
@@ -315,27 +335,29 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
         if (valid[t] <= 0) continue;
         float acc = 0.f;
 #pragma unroll
-        for (int qc = 0; qc < TCOL / 16; ++qc) {
-            if (qc * 16 >= npad) break;       // columns past the padded query count were never exponentiated
+        for (int qc = 0; qc < TC / 16; ++qc) {
+            if (c0 + qc * 16 >= npad) break;  // columns past the padded query count were never exponentiated
 #pragma unroll
             for (int i = 0; i < 16; ++i)      // s_w is 0 past the text queries
-                acc = fmaf(L[t * TCOL + qc * 16 + i], s_w[qc * 16 + i], acc);
+                acc = fmaf(L[t * TC + qc * 16 + i], s_w[c0 + qc * 16 + i], acc);
         }
-        if (tid < valid[t]) {
-            if (acc64)
-                atomicAdd(acc64 + s.vis_off + vis0[t] + tid, __float2ull_rn(acc * kFixScale));
-            else if (part)                    // neither: the caller wants the attention copy only
-                part[static_cast<int64_t>(h) * part_stride + s.vis_off + vis0[t] + tid] = acc;
-            if (alpha.ptr) {              // the attention itself, for the per-patch indicators: this key's row of queries
-                float4* ap = reinterpret_cast<float4*>(alpha.ptr + static_cast<int64_t>(h) * alpha.stride_h +
-                                                       static_cast<int64_t>(s.vis_off + vis0[t] + tid) * alpha.stride_j);
-                const float hn = static_cast<float>(n_heads) * static_cast<float>(s.n_txt);   // s_w carries 1 / (H n_t)
+        if (key < valid[t]) {
+            if (acc64)                        // (with SPLIT = 2 both halves of the queries add into the key's accumulator)
+                atomicAdd(acc64 + s.vis_off + vis0[t] + key, __float2ull_rn(acc * kFixScale));
+            if constexpr (SPLIT == 1) {
+                if (!acc64 && part)           // neither: the caller wants the attention copy only
+                    part[static_cast<int64_t>(h) * part_stride + s.vis_off + vis0[t] + key] = acc;
+                if (alpha.ptr) {              // the attention itself, for the per-patch indicators: this key's row of queries
+                    float4* ap = reinterpret_cast<float4*>(alpha.ptr + static_cast<int64_t>(h) * alpha.stride_h +
+                                                           static_cast<int64_t>(s.vis_off + vis0[t] + key) * alpha.stride_j);
+                    const float hn = static_cast<float>(n_heads) * static_cast<float>(s.n_txt);   // s_w carries 1 / (H n_t)
 #pragma unroll
-                for (int g4 = 0; g4 < TCOL / 4; ++g4) {   // 16-byte stores: a handful of instructions (s_w is 0 past the text queries)
-                    if (4 * g4 >= npad || 4 * g4 >= alpha.stride_j) break;
-                    const float4 w4 = *reinterpret_cast<const float4*>(&s_w[4 * g4]);
-                    ap[g4] = make_float4(L[t * TCOL + 4 * g4] * w4.x * hn, L[t * TCOL + 4 * g4 + 1] * w4.y * hn,
-                                         L[t * TCOL + 4 * g4 + 2] * w4.z * hn, L[t * TCOL + 4 * g4 + 3] * w4.w * hn);
+                    for (int g4 = 0; g4 < TCOL / 4; ++g4) {   // 16-byte stores: a handful of instructions (s_w is 0 past the text queries)
+                        if (4 * g4 >= npad || 4 * g4 >= alpha.stride_j) break;
+                        const float4 w4 = *reinterpret_cast<const float4*>(&s_w[4 * g4]);
+                        ap[g4] = make_float4(L[t * TCOL + 4 * g4] * w4.x * hn, L[t * TCOL + 4 * g4 + 1] * w4.y * hn,
+                                             L[t * TCOL + 4 * g4 + 2] * w4.z * hn, L[t * TCOL + 4 * g4 + 3] * w4.w * hn);
+                    }
                 }
             }
         }
@@ -350,14 +372,14 @@ salience_fast_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant
     }
 }
 
-template <int TCOL, int NTILE>
+template <int TCOL, int NTILE, int SPLIT>
 cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int head_dim, int esize, const CUtensorMap* tq,
                           const CUtensorMap* tk, int cluster, int npad, float* part, int64_t part_stride,
                           unsigned long long* acc64, int* status, int free_running, AlphaOut alpha, int32_t* rearm, unsigned long long* rearm_rec, unsigned long long* stamps,
                           float* lcache, int cache_vis, int cache_cols, cudaStream_t stream)
 {
     size_t smem = 1024 + static_cast<size_t>((head_dim * esize + 127) / 128) * (static_cast<size_t>(NTILE) * 16384 + npad * 128);
-    auto kern = salience_fast_kernel<TCOL, NTILE>;
+    auto kern = salience_fast_kernel<TCOL, NTILE, SPLIT>;
     // resident CTAs x tensor-memory columns must not exceed the 512 of a multiprocessor
     const int tmem_cols = tmem_cols_for(TCOL * NTILE);
     smem = smem_for_tmem(smem, tmem_cols);
@@ -365,12 +387,12 @@ cudaError_t launch_fast_t(const BatchDesc& bd, int n_heads, int kv_group, int he
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     int resident = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kern, kFastThreads, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kern, kFastThreads * SPLIT, smem);
     if (e != cudaSuccess) return e;
     if (resident * tmem_cols > kTmemColsPerSm) return cudaErrorInvalidConfiguration;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cluster, n_heads, bd.n);
-    cfg.blockDim = dim3(kFastThreads);
+    cfg.blockDim = dim3(kFastThreads * SPLIT);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
@@ -395,11 +417,14 @@ cudaError_t launch_salience_fast(const BatchDesc& bd, int n_heads, int kv_group,
                                  float* lcache, int cache_vis, int cache_cols, cudaStream_t stream)
 {
     const int tcol = npad <= 16 ? 16 : (npad <= 32 ? 32 : 64);
-#define MVLA_FAST(TC, NTL)                                                                                      \
-    if (tcol == TC && tiles_per_cta == NTL)                                                                     \
-        return launch_fast_t<TC, NTL>(bd, n_heads, kv_group, head_dim, esize, tmap_q, tmap_k, cluster, npad, part, part_stride, \
-                                      acc64, status, free_running ? 1 : 0, alpha, rearm, rearm_rec, stamps, lcache, cache_vis, cache_cols, stream);
-    MVLA_FAST(16, 1) MVLA_FAST(32, 1) MVLA_FAST(64, 1) MVLA_FAST(16, 2) MVLA_FAST(32, 2) MVLA_FAST(64, 2)
+    // two threads per key where the kernel's outputs allow it (see the kernel) and a thread still holds 16 queries
+    const int split = (acc64 && !alpha.ptr && tcol >= 32) ? 2 : 1;
+#define MVLA_FAST(TC, NTL, SP)                                                                                  \
+    if (tcol == TC && tiles_per_cta == NTL && split == SP)                                                      \
+        return launch_fast_t<TC, NTL, SP>(bd, n_heads, kv_group, head_dim, esize, tmap_q, tmap_k, cluster, npad, part, part_stride, \
+                                          acc64, status, free_running ? 1 : 0, alpha, rearm, rearm_rec, stamps, lcache, cache_vis, cache_cols, stream);
+    MVLA_FAST(16, 1, 1) MVLA_FAST(32, 1, 1) MVLA_FAST(64, 1, 1) MVLA_FAST(16, 2, 1) MVLA_FAST(32, 2, 1) MVLA_FAST(64, 2, 1)
+    MVLA_FAST(32, 1, 2) MVLA_FAST(64, 1, 2) MVLA_FAST(32, 2, 2) MVLA_FAST(64, 2, 2)
 #undef MVLA_FAST
     return cudaErrorInvalidConfiguration;
 }
