@@ -28,6 +28,11 @@
  *     `attn`, `l1`, `ahat` hold sum(n_2d + n_3d) floats, samples back to back in batch order.
  *   - Inputs must be finite.
  *   - A context is not thread-safe; use one per host thread / stream.
+ *   - Tracing and logging (the paper has no counterpart; host side only, nothing on the device's path):
+ *     every call of the stage and step functions is an NVTX range named after the function, and
+ *     mvla_prune_step marks its phases inside it ("mvla: scoring", "mvla: selection + row copy", ...) around
+ *     the kernels they enqueue; with MVLA_LOG=1 in the environment (read once per process) each of those
+ *     calls also prints one line "[mvla] name(arguments) -> status" to stderr.
  */
 #ifndef MVLA_PRUNE_H
 #define MVLA_PRUNE_H

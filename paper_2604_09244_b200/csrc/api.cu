@@ -9,6 +9,9 @@
 #include <cstring>
 #include <new>
 #include <vector>
+#include <cstdio>
+
+#include <nvtx3/nvToolsExt.h>
 
 using namespace mvla;
 
@@ -18,6 +21,36 @@ constexpr int kSets = 6;            // scratch sets = prune steps that may be in
 #define MVLA_TAIL_CTAS_PER_SM 2
 #endif
 constexpr int kTailCtasPerSm = MVLA_TAIL_CTAS_PER_SM;   // grid of the selection + row copy kernel
+
+// Tracing and logging, both on the host and off the device's path: every public call is an NVTX range (a profiler
+// shows the call and, inside mvla_prune_step, its phases around the kernels they enqueue; without a profiler
+// attached a range costs a few nanoseconds), and with MVLA_LOG=1 in the environment every call prints one line
+// with its arguments and its result to stderr.
+struct ApiRange {
+    explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+    ~ApiRange() { nvtxRangePop(); }
+    ApiRange(const ApiRange&) = delete;
+    ApiRange& operator=(const ApiRange&) = delete;
+};
+// The phases of a step inside the call's range: mark() closes the phase before it.
+struct PhaseRange {
+    bool open = false;
+    void mark(const char* name)
+    {
+        if (open) nvtxRangePop();
+        nvtxRangePushA(name);
+        open = true;
+    }
+    ~PhaseRange() { if (open) nvtxRangePop(); }
+};
+bool log_enabled()
+{
+    static const bool on = [] {
+        const char* e = std::getenv("MVLA_LOG");
+        return e && *e && *e != '0';
+    }();
+    return on;
+}
 }
 
 struct mvla_ctx {
@@ -544,6 +577,7 @@ int32_t run_patch_select(mvla_ctx* ctx, unsigned set, const Plan& plan, int32_t 
 int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, uint32_t flags,
                          const mvla_tensors* in, const mvla_outputs* out, int32_t* total_kept_out, void* stream)
 {
+    PhaseRange ph;
     if (!in->hidden || !in->rand_u) return MVLA_ERR_INVALID_ARG;
     if (flags & ~(MVLA_FLAG_RESET_STATE | MVLA_FLAG_NO_STATE_UPDATE | MVLA_FLAG_INPUTS_STABLE)) return MVLA_ERR_INVALID_ARG;
     const void* src[3] = {in->hidden, in->k, in->v};
@@ -611,6 +645,7 @@ int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, cons
         int32_t* list = ctx->tail_list + par * ctx->rows_all;
         unsigned long long* rec = ctx->patch_rec + par * (ctx->vis_all / 2 + 1) * 3;
         const AlphaOut alpha = alpha_of(ctx, set);
+        ph.mark("mvla: scoring (+ attention copy)");
         rc = run_salience_chunk(ctx, whole, in->q, in->k, in->rows, nullptr, nullptr, nullptr, nullptr, false, st, alpha,
                                 list, false, nullptr, false, rec);
         if (rc != MVLA_OK) return rc;
@@ -624,6 +659,7 @@ int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, cons
         io.done_ws = ws + 2 * ctx->cfg.max_batch; io.status = ctx->status_dev;
         io.kept_idx = out->kept_idx; io.out_offsets = out->out_offsets; io.batch_total = batch;
         io.chunk_first = 0;
+        ph.mark("mvla: indicators + stages 1-4 + row copy");
         const cudaError_t e = launch_patch_tail(whole, ctx->cfg.n_heads, alpha, ctx->hidden_dtype, ctx->cfg.d_model, in->hidden,
                                                 x, attn, rec, pp, io, job, list, ctx->sm_count, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
@@ -631,12 +667,14 @@ int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, cons
         if (total_kept_out) *total_kept_out = static_cast<int32_t>(cap);
         return MVLA_OK;
     }
+    ph.mark("mvla: scoring + indicators");
     rc = run_patch_indicators(ctx, set, plan, batch, in->q, in->k, in->hidden, in->rows, attn, x, side_stream);
     if (rc != MVLA_OK) return rc;
     if (forked) {
         rc = wait_state_deps(ctx, fp, side_stream);
         if (rc != MVLA_OK) return rc;
     }
+    ph.mark("mvla: stages 1-4");
     rc = run_patch_select(ctx, set, plan, batch, attn, x, in->rand_u, out->kept_idx, out->out_offsets, out->budgets,
                           out->patch_xhat, out->patch_info, out->patch_diag, side_stream);
     if (rc != MVLA_OK) return rc;
@@ -646,6 +684,7 @@ int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, cons
     }
     for (int first = 0; first < batch; first += kMaxChunk) {
         const BatchDesc bd = chunk_of(plan, first, std::min(kMaxChunk, batch - first));
+        ph.mark("mvla: row copy");
         const cudaError_t e = launch_compact(bd, job, out->kept_idx, static_cast<int32_t>(cap), 0, out->out_offsets, first, batch, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
     }
@@ -659,7 +698,7 @@ int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, cons
 
 extern "C" {
 
-int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
+static int32_t mvla_prune_create_impl(const mvla_config* cfg, mvla_ctx** out)
 {
     if (!cfg || !out) return MVLA_ERR_INVALID_ARG;
     *out = nullptr;
@@ -836,7 +875,7 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     delete ctx;
 }
 
-int32_t mvla_salience(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const void* q, const void* k,
+static int32_t mvla_salience_impl(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const void* q, const void* k,
                       const void* hidden, int64_t rows, float* attn_out, float* l1_out, void* stream)
 {
     if (!ctx || !q || !k || !attn_out || rows < 1) return MVLA_ERR_INVALID_ARG;
@@ -863,7 +902,7 @@ int32_t mvla_salience(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, 
     return MVLA_OK;
 }
 
-int32_t mvla_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, int32_t mode,
+static int32_t mvla_select_impl(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, int32_t mode,
                     uint32_t flags, const float* attn, const float* l1, int32_t* kept_idx, int32_t* out_offsets,
                     int32_t* budgets, float* ahat_out, float* z_out, mvla_diag* diag, void* stream)
 {
@@ -900,7 +939,7 @@ int32_t mvla_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvl
     return MVLA_OK;
 }
 
-int32_t mvla_compact(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const int32_t* kept_idx,
+static int32_t mvla_compact_impl(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const int32_t* kept_idx,
                      const int32_t* out_offsets, int32_t total_kept, const void* hidden, const void* k,
                      const void* v, void* out_hidden, void* out_k, void* out_v, void* stream)
 {
@@ -969,7 +1008,7 @@ int32_t mvla_selftest_wait_timeout(mvla_ctx* ctx, uint32_t limit_us, void* strea
     return MVLA_OK;
 }
 
-int32_t mvla_patch_indicators(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const void* q, const void* k,
+static int32_t mvla_patch_indicators_impl(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const void* q, const void* k,
                               const void* hidden, int64_t rows, float* attn_out, float* x_out, void* stream)
 {
     if (!ctx || !q || !k || !hidden || !attn_out || !x_out || rows < 1) return MVLA_ERR_INVALID_ARG;
@@ -989,7 +1028,7 @@ int32_t mvla_patch_indicators(mvla_ctx* ctx, int32_t batch, const mvla_sample* s
     return run_patch_indicators(ctx, 0, plan, batch, q, k, hidden, rows, attn_out, x_out, static_cast<cudaStream_t>(stream));
 }
 
-int32_t mvla_patch_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, uint32_t flags,
+static int32_t mvla_patch_select_impl(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, uint32_t flags,
                           const float* attn, const float* x, const float* rand_u, int32_t* kept_idx,
                           int32_t* out_offsets, int32_t* counts, float* xhat_out, int32_t* info_out,
                           mvla_patch_diag* diag, void* stream)
@@ -1016,12 +1055,13 @@ int32_t mvla_patch_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, con
     return MVLA_OK;
 }
 
-int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples,
+static int32_t mvla_prune_step_impl(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples,
                         int32_t mode, uint32_t flags, const mvla_tensors* in, const mvla_outputs* out,
                         int32_t* total_kept_out, void* stream)
 {
     if (!ctx || !in || !out || !in->q || !in->k || !out->kept_idx || !out->out_offsets || in->rows < 1)
         return MVLA_ERR_INVALID_ARG;
+    PhaseRange ph;
     if (mode == MVLA_MODE_PATCH)
         return prune_step_patch(ctx, prune_point, batch, samples, flags, in, out, total_kept_out, stream);
     if (flags & ~(MVLA_FLAG_RESET_STATE | MVLA_FLAG_NO_STATE_UPDATE | MVLA_FLAG_INPUTS_STABLE)) return MVLA_ERR_INVALID_ARG;
@@ -1124,6 +1164,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         bool used_acc64 = false;
         // the fused selection + copy kernel (below) wants its list words re-armed by the scoring kernel
         const bool tail = !forked && select_copy_supported(bd);
+        ph.mark("mvla: scoring");
         rc = run_salience_chunk(ctx, bd, in->q, in->k, in->rows, adaptive ? in->hidden : nullptr, l1_ws, acc64,
                                 &used_acc64, false, forked ? ctx->aux[par] : st, AlphaOut{nullptr, 0, 0},
                                 tail ? ctx->tail_list + par * ctx->rows_all : nullptr, tail, tail ? ctx->stamps : nullptr,
@@ -1159,6 +1200,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
             ctx->sel_valid[par] = false;             // this set was used outside the event chain
             const bool copying = (job.src[0] && job.dst[0]) || (job.src[1] && job.dst[1]) || (job.src[2] && job.dst[2]);
             (void)copying;
+            ph.mark("mvla: selection + row copy");
             const cudaError_t e2 = launch_select_copy(bd, gp, io, job, ctx->tail_list + par * ctx->rows_all,
                                                       ctx->status_dev, ctx->sm_count * kTailCtasPerSm - n,
                                                       ctx->stamps ? ctx->stamps + 2 * kStampSlots : nullptr, st);
@@ -1168,6 +1210,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
             }
             continue;
         }
+        ph.mark("mvla: selection");
         cudaError_t e = launch_select(bd, gp, io, sel_stream);
         if (e != cudaSuccess) {
             if (used_acc64) clear_accumulators(acc64, bd, sel_stream);
@@ -1181,6 +1224,7 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
         }
         const int32_t row0 = bd.s[0].out_off;
         const int32_t nrows = bd.s[n - 1].out_off + bd.s[n - 1].n_out - row0;
+        ph.mark("mvla: row copy");
         e = launch_compact(bd, job, out->kept_idx, nrows, row0, nullptr, first, batch, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
         if (forked && cudaEventRecord(ctx->ev_copy[par], st) != cudaSuccess) return fail_cuda(ctx, cudaGetLastError());
@@ -1188,6 +1232,75 @@ int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const
     commit_steps(ctx, prune_point, plan, samples);
     if (total_kept_out) *total_kept_out = plan.total_out;
     return MVLA_OK;
+}
+
+// ---- the public entry points: an NVTX range around each call, and with MVLA_LOG=1 a line on stderr per call
+
+int32_t mvla_prune_create(const mvla_config* cfg, mvla_ctx** out)
+{
+    ApiRange range("mvla_prune_create");
+    const int32_t rc = mvla_prune_create_impl(cfg, out);
+    if (log_enabled()) std::fprintf(stderr, "[mvla] mvla_prune_create(heads %lld x %lld, d_model %lld, dtype %lld, max batch %lld, text %lld, 2D %lld, 3D %lld) -> %d\n", static_cast<long long>(cfg ? cfg->n_heads : -1), static_cast<long long>(cfg ? cfg->head_dim : -1), static_cast<long long>(cfg ? cfg->d_model : -1), static_cast<long long>(cfg ? cfg->dtype : -1), static_cast<long long>(cfg ? cfg->max_batch : -1), static_cast<long long>(cfg ? cfg->max_text : -1), static_cast<long long>(cfg ? cfg->max_2d : -1), static_cast<long long>(cfg ? cfg->max_3d : -1), rc);
+    return rc;
+}
+
+int32_t mvla_salience(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const void* q, const void* k,
+                      const void* hidden, int64_t rows, float* attn_out, float* l1_out, void* stream)
+{
+    ApiRange range("mvla_salience");
+    const int32_t rc = mvla_salience_impl(ctx, batch, samples, q, k, hidden, rows, attn_out, l1_out, stream);
+    if (log_enabled()) std::fprintf(stderr, "[mvla] mvla_salience(batch %lld, rows %lld) -> %d\n", static_cast<long long>(batch), static_cast<long long>(rows), rc);
+    return rc;
+}
+
+int32_t mvla_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, int32_t mode,
+                    uint32_t flags, const float* attn, const float* l1, int32_t* kept_idx, int32_t* out_offsets,
+                    int32_t* budgets, float* ahat_out, float* z_out, mvla_diag* diag, void* stream)
+{
+    ApiRange range("mvla_select");
+    const int32_t rc = mvla_select_impl(ctx, prune_point, batch, samples, mode, flags, attn, l1, kept_idx, out_offsets, budgets, ahat_out, z_out, diag, stream);
+    if (log_enabled()) std::fprintf(stderr, "[mvla] mvla_select(prune_point %lld, batch %lld, mode %lld, flags %lld) -> %d\n", static_cast<long long>(prune_point), static_cast<long long>(batch), static_cast<long long>(mode), static_cast<long long>(flags), rc);
+    return rc;
+}
+
+int32_t mvla_compact(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const int32_t* kept_idx,
+                     const int32_t* out_offsets, int32_t total_kept, const void* hidden, const void* k,
+                     const void* v, void* out_hidden, void* out_k, void* out_v, void* stream)
+{
+    ApiRange range("mvla_compact");
+    const int32_t rc = mvla_compact_impl(ctx, batch, samples, kept_idx, out_offsets, total_kept, hidden, k, v, out_hidden, out_k, out_v, stream);
+    if (log_enabled()) std::fprintf(stderr, "[mvla] mvla_compact(batch %lld) -> %d\n", static_cast<long long>(batch), rc);
+    return rc;
+}
+
+int32_t mvla_patch_indicators(mvla_ctx* ctx, int32_t batch, const mvla_sample* samples, const void* q, const void* k,
+                              const void* hidden, int64_t rows, float* attn_out, float* x_out, void* stream)
+{
+    ApiRange range("mvla_patch_indicators");
+    const int32_t rc = mvla_patch_indicators_impl(ctx, batch, samples, q, k, hidden, rows, attn_out, x_out, stream);
+    if (log_enabled()) std::fprintf(stderr, "[mvla] mvla_patch_indicators(batch %lld, rows %lld) -> %d\n", static_cast<long long>(batch), static_cast<long long>(rows), rc);
+    return rc;
+}
+
+int32_t mvla_patch_select(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples, uint32_t flags,
+                          const float* attn, const float* x, const float* rand_u, int32_t* kept_idx,
+                          int32_t* out_offsets, int32_t* counts, float* xhat_out, int32_t* info_out,
+                          mvla_patch_diag* diag, void* stream)
+{
+    ApiRange range("mvla_patch_select");
+    const int32_t rc = mvla_patch_select_impl(ctx, prune_point, batch, samples, flags, attn, x, rand_u, kept_idx, out_offsets, counts, xhat_out, info_out, diag, stream);
+    if (log_enabled()) std::fprintf(stderr, "[mvla] mvla_patch_select(prune_point %lld, batch %lld, flags %lld) -> %d\n", static_cast<long long>(prune_point), static_cast<long long>(batch), static_cast<long long>(flags), rc);
+    return rc;
+}
+
+int32_t mvla_prune_step(mvla_ctx* ctx, int32_t prune_point, int32_t batch, const mvla_sample* samples,
+                        int32_t mode, uint32_t flags, const mvla_tensors* in, const mvla_outputs* out,
+                        int32_t* total_kept_out, void* stream)
+{
+    ApiRange range("mvla_prune_step");
+    const int32_t rc = mvla_prune_step_impl(ctx, prune_point, batch, samples, mode, flags, in, out, total_kept_out, stream);
+    if (log_enabled()) std::fprintf(stderr, "[mvla] mvla_prune_step(prune_point %lld, batch %lld, mode %lld, flags %lld, rows %lld) -> %d\n", static_cast<long long>(prune_point), static_cast<long long>(batch), static_cast<long long>(mode), static_cast<long long>(flags), static_cast<long long>(in ? in->rows : -1), rc);
+    return rc;
 }
 
 }  // extern "C"

@@ -70,3 +70,36 @@ def test_no_device_is_an_error_not_a_fallback(lib):
 def test_missing_library_fails_loudly(tmp_path):
     with pytest.raises(OSError):
         mvla.load_library(str(tmp_path / "libmvla_prune.so"))
+
+
+def test_mvla_log_prints_one_line_per_call():
+    """MVLA_LOG=1: every public call reports its arguments and its result on stderr (host side only); without the
+    variable nothing is printed.  Runs in a child process: the variable is read once per process."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = ("import ctypes as C, sys\n"
+            f"sys.path.insert(0, {root!r})\n"
+            "from paper_2604_09244_b200 import mvla\n"
+            "lib = mvla.load_library()\n"
+            "h = C.c_void_p()\n"
+            "cfg = mvla.Config(0, mvla.DTYPE_BF16, 32, 128, 4096, 1, 32, 256, 512, 1, 0, 7, 1, 0, 0.08, 0.2, 0.85, 0.02, 0.1)\n"
+            "rc = lib.mvla_prune_create(C.byref(cfg), C.byref(h))\n"
+            "rc2 = lib.mvla_salience(None, 1, None, None, None, None, 0, None, None, None)\n"
+            "print(rc, rc2)\n")
+    for on in (True, False):
+        env = dict(os.environ)
+        env.pop("MVLA_LOG", None)
+        if on:
+            env["MVLA_LOG"] = "1"
+        r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
+        assert r.returncode == 0, r.stderr
+        rc, rc2 = (int(x) for x in r.stdout.split())
+        lines = [ln for ln in r.stderr.splitlines() if ln.startswith("[mvla] ")]
+        if on:
+            assert len(lines) == 2
+            assert lines[0].startswith("[mvla] mvla_prune_create(heads 32 x 128, d_model 4096") and lines[0].endswith(f"-> {rc}")
+            assert lines[1].startswith("[mvla] mvla_salience(batch 1") and lines[1].endswith(f"-> {rc2}")
+        else:
+            assert not lines
