@@ -715,3 +715,17 @@ def test_a_mask_that_hides_a_change_reuses_the_stale_logits():
     assert_salience_close(out2.attn.cpu().numpy(), truth)
     assert ctx.logit_cache_stats()[1] >= 5                            # step 2 reused all 2 + 3 tiles of step 1
     ctx.close()
+
+
+@pytest.mark.parametrize("n_txt,n_2d,n_3d", [(40, 700, 900), (64, 512, 640), (17, 1500, 500), (48, 100, 60)])
+def test_step_with_two_threads_per_key_in_every_shape_of_the_scoring_kernel(n_txt, n_2d, n_3d):
+    # more than 16 text queries: the scoring kernel of the fused step runs with two threads per key, half of the
+    # queries each; 33-64 queries use 64 tensor-memory columns (the second half partly empty at 40 and 48), more
+    # than 1024 visual tokens put two key tiles on a CTA
+    wl = W.small_workload(97, batch=1, D=128, H=2, d=64, dtype="bf16", n_txt=(n_txt,), n_2d=(n_2d,), n_3d=(n_3d,),
+                          keep=(0.4,), steps=2)
+    ctx = mvla.context_for(wl)
+    states = _fresh_states(wl)
+    for t in range(2):
+        run_and_check_step(ctx, wl, t, states)
+    ctx.close()
