@@ -71,6 +71,7 @@ struct mvla_ctx {
                                  // calls; the sets rotate from step to step (a step's scoring may run beside
                                  // the selections of the steps before it)
     int32_t* tail_list;          // [kSets][rows_all] kept list as the copying CTAs read it (-1 between launches)
+    unsigned int* tail_ticket;   // [kSets] ticket counters of the patch-by-patch tail (zero between launches)
     unsigned long long* patch_rec;   // [kSets][vis_all / 2][3] hand-over words of the patch-by-patch tail (all ones between launches)
     size_t rows_all;             // max_batch * (kHandWords + max_text + max_vis)
     int sm_count;                // multiprocessors of the device
@@ -661,7 +662,7 @@ int32_t prune_step_patch(mvla_ctx* ctx, int32_t prune_point, int32_t batch, cons
         io.chunk_first = 0;
         ph.mark("mvla: indicators + stages 1-4 + row copy");
         const cudaError_t e = launch_patch_tail(whole, ctx->cfg.n_heads, alpha, ctx->hidden_dtype, ctx->cfg.d_model, in->hidden,
-                                                x, attn, rec, pp, io, job, list, ctx->sm_count, st);
+                                                x, attn, rec, pp, io, job, list, ctx->sm_count, ctx->tail_ticket + par, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
         commit_steps(ctx, prune_point, plan, samples);
         if (total_kept_out) *total_kept_out = static_cast<int32_t>(cap);
@@ -749,6 +750,7 @@ static int32_t mvla_prune_create_impl(const mvla_config* cfg, mvla_ctx** out)
     ctx->part = ctx->l1_ws = ctx->ahat_state = ctx->mhat_state = nullptr;
     ctx->acc64 = nullptr;
     ctx->tail_list = nullptr;
+    ctx->tail_ticket = nullptr;
     ctx->patch_rec = nullptr;
     ctx->sm_count = prop.multiProcessorCount;
     ctx->stage_event = nullptr;
@@ -797,6 +799,8 @@ static int32_t mvla_prune_create_impl(const mvla_config* cfg, mvla_ctx** out)
     // (+ 1: a word that no launch ever writes, for mvla_selftest_wait_timeout)
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->tail_list), (kSets * ctx->rows_all + 1) * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->tail_list, 0xFF, (kSets * ctx->rows_all + 1) * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->tail_ticket), kSets * sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->tail_ticket, 0, kSets * sizeof(unsigned int));
     if (c.logit_cache) {
         ctx->cache_sig.assign(n_state, mvla_ctx::CacheSig{false, 0, 0, 0});
         alloc(&ctx->lcache, n_state * static_cast<size_t>(c.n_heads) * ctx->max_vis * ctx->cache_cols);
@@ -854,6 +858,7 @@ void mvla_prune_destroy(mvla_ctx* ctx)
     cudaFree(ctx->mhat_state);
     cudaFree(ctx->acc64);
     cudaFree(ctx->tail_list);
+    cudaFree(ctx->tail_ticket);
     cudaFree(ctx->patch_rec);
     cudaFree(ctx->lcache);
     cudaFree(ctx->alpha_ws);

@@ -197,7 +197,8 @@ cudaError_t launch_compact(const BatchDesc& bd, const CompactJob& job, const int
 // (bounded waits, MVLA_ERR_TIMEOUT into `status` when one runs out): no kernel boundary, fence or flag lies
 // between selection and copy.  `list`: one int per output row of the batch, all -1 when the kernel starts
 // (the scoring kernel before it re-arms them, see launch_salience_fast).
-// `ctas`: copying CTAs to aim for (every sample gets at least one).  `stamps`: as in launch_salience_fast
+// `ctas`: copying CTAs to aim for (every sample gets at least one); together with the selecting CTAs no more than
+// fit on the device at once, see the kernel.  `stamps`: as in launch_salience_fast
 // (start: past the wait for the kernel before; the selecting CTA's end is when the list is written).
 bool select_copy_supported(const BatchDesc& bd);
 cudaError_t launch_select_copy(const BatchDesc& bd, const GateParams& gp, const SelectIO& io, const CompactJob& job,
@@ -239,9 +240,11 @@ cudaError_t launch_patch_select(const BatchDesc& bd, const PatchParams& pp, cons
 // Indicators, stages 1-4 and the row copy of the patch-by-patch step in one kernel behind the scoring kernel
 // (which must have re-armed `list` and `rec`, see launch_salience_fast).  `rec`: [sum P][3] 8-byte words;
 // `list`: 4-byte words, kHandWords + n_txt + n_vis per sample from cap_off on.  io.x / io.attn are not read.
+// `ticket_counter`: one word, zero before the first launch, used by one launch at a time (it returns to zero with
+// every launch): the CTAs take their roles in the order in which they start (copy_impl.cuh: cta_ticket).
 bool patch_tail_supported(const BatchDesc& bd);
 cudaError_t launch_patch_tail(const BatchDesc& bd, int n_heads, AlphaOut alpha, int dtype, int d_model, const void* hidden,
                               float* x_out, float* attn_out, unsigned long long* rec, const PatchParams& pp, const PatchIO& io,
-                              const CompactJob& job, int32_t* list, int sm_count, cudaStream_t stream);
+                              const CompactJob& job, int32_t* list, int sm_count, unsigned int* ticket_counter, cudaStream_t stream);
 
 }  // namespace mvla

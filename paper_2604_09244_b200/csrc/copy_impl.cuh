@@ -7,6 +7,18 @@
 
 namespace mvla {
 
+// Which CTA of the launch this is, in the order in which the CTAs STARTED: a ticket from a counter that counts
+// 0 .. grid - 1 and wraps back to 0 with the launch's last ticket (so it needs no reset between launches; one
+// launch at a time per counter).  A CTA that waits for CTAs with lower tickets waits for CTAs that are running
+// -- whatever order the hardware dispatches block indices in.  Called by all threads of the CTA.
+__device__ __forceinline__ int cta_ticket(unsigned int* counter)
+{
+    __shared__ int s_ticket;
+    if (threadIdx.x == 0) s_ticket = static_cast<int>(atomicInc(counter, gridDim.x - 1));
+    __syncthreads();
+    return s_ticket;
+}
+
 __device__ __forceinline__ uint4 ld_row(const uint4* p)
 {
     uint4 v;

@@ -6,8 +6,8 @@
 //     (stages 1-4), reading each patch's words as they appear; it writes the kept list as 4-byte words;
 //   * the remaining CTAs copy the surviving rows, each warp polling the word of the row it is to move.
 // No kernel boundary, fence or flag lies between the three roles: every word is its own signal, re-armed
-// (all ones) by the scoring kernel of the same step.  A consumer always has a higher block index than the
-// CTAs it waits for, so those were dispatched no later than itself; every wait is bounded all the same.
+// (all ones) by the scoring kernel of the same step.  The roles go by ticket (cta_ticket: the order in which the
+// CTAs started), so a consumer only ever waits for CTAs that are already running; every wait is bounded all the same.
 #include "copy_impl.cuh"
 #include "patch_impl.cuh"
 
@@ -28,10 +28,10 @@ __global__ void __launch_bounds__(kTailThreads, 1)
 patch_tail_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ PatchTailPlan tp, int n_heads,
                   const AlphaOut alpha, const T* __restrict__ hidden, int d_model, float* __restrict__ x_out,
                   float* __restrict__ attn_out, unsigned long long* rec, const PatchParams pp, const PatchIO io,
-                  const __grid_constant__ CompactArgs ca, int32_t* list)
+                  const __grid_constant__ CompactArgs ca, int32_t* list, unsigned int* ticket_counter)
 {
     const int n_ind = tp.ind0[bd.n];
-    int c = blockIdx.x;
+    int c = cta_ticket(ticket_counter);
     if (c < n_ind) {
         int b = 0;
         while (b + 1 < bd.n && c >= tp.ind0[b + 1]) ++b;
@@ -106,7 +106,7 @@ bool patch_tail_supported(const BatchDesc& bd)
 
 cudaError_t launch_patch_tail(const BatchDesc& bd, int n_heads, AlphaOut alpha, int dtype, int d_model, const void* hidden,
                               float* x_out, float* attn_out, unsigned long long* rec, const PatchParams& pp, const PatchIO& io,
-                              const CompactJob& job, int32_t* list, int sm_count, cudaStream_t stream)
+                              const CompactJob& job, int32_t* list, int sm_count, unsigned int* ticket_counter, cudaStream_t stream)
 {
     if (!patch_tail_supported(bd)) return cudaErrorInvalidConfiguration;
     // as many patches per CTA as still give every multiprocessor a CTA
@@ -152,7 +152,7 @@ cudaError_t launch_patch_tail(const BatchDesc& bd, int n_heads, AlphaOut alpha, 
 #define MVLA_TAIL(T, PPV)                                                                                     \
     if (per == PPV)                                                                                           \
         return cudaLaunchKernelEx(&cfg, patch_tail_kernel<T, PPV>, bd, tp, n_heads, alpha,                    \
-                                  static_cast<const T*>(hidden), d_model, x_out, attn_out, rec, pp, io, ca, list);
+                                  static_cast<const T*>(hidden), d_model, x_out, attn_out, rec, pp, io, ca, list, ticket_counter);
     if (dtype == MVLA_DTYPE_BF16) { MVLA_TAIL(__nv_bfloat16, 8) MVLA_TAIL(__nv_bfloat16, 4) MVLA_TAIL(__nv_bfloat16, 2) }
     else { MVLA_TAIL(float, 8) MVLA_TAIL(float, 4) MVLA_TAIL(float, 2) }
 #undef MVLA_TAIL

@@ -37,8 +37,12 @@ __global__ void wait_probe_kernel(const int* never_set, uint64_t limit_ns, int* 
 // grid: CTAs 0 .. n-1 select (CTA b for sample b of the launch), the CTAs after them copy; tp.cta0[b] is the
 // first copying CTA of sample b.  `list`: the kept list in library scratch (one word per output row of the
 // launch's samples, -1 = not yet known; the scoring kernel before this one has set them all to -1).
-// A selecting CTA always has a lower index than any copying CTA, so it is dispatched before them: a
-// copier that runs can count on its selector running too.  Its waits are bounded all the same.
+// The roles go by block index.  The launcher never asks for more CTAs than fit on the device together
+// (`ctas` = multiprocessors x CTAs per multiprocessor), and the kernel after this one cannot start before
+// every CTA of this one has started, so all CTAs of the grid become resident whatever order they are
+// dispatched in: a copying CTA never keeps its selecting CTA from running.  (Taking the roles in the order
+// in which the CTAs start, by a ticket from an atomic counter as the patch-by-patch tail does, cost 0.4 us per
+// step here: 296 atomics on one word.)  All waits are bounded all the same.
 template <int NT, int CAP>
 __global__ void __launch_bounds__(NT)
 select_copy_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__ TailPlan tp, const GateParams gp,
@@ -46,22 +50,23 @@ select_copy_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__
                    unsigned long long* __restrict__ stamps)
 {
     const int tid = threadIdx.x, lane = tid & 31;
-    if (static_cast<int>(blockIdx.x) < bd.n) {
+    const int cta = blockIdx.x;
+    if (cta < bd.n) {
         // ---- selection of one sample, by one CTA
         __shared__ SelectSmem<NT, CAP> sm;
-        const int b = blockIdx.x;
+        const int b = cta;
         SelectRole role;
         role.late_pdl = true;
         role.l1_late = true;                                // the norms may come from a kernel that ran beside the scoring
         if (tp.cta0[bd.n] > 0) role.kept_sm = list + bd.s[b].out_off;   // every word is its own "ready" signal
         select_sample<NT, CAP>(bd.s[b], b, gp, io, sm, role, [&]() {}, [&]() {
-            if (stamps && tid == 0 && blockIdx.x < kStampSlots) stamps[2 * blockIdx.x + 1] = global_ns();
+            if (stamps && tid == 0 && cta < kStampSlots) stamps[2 * cta + 1] = global_ns();
         });
-        if (stamps && tid == 0 && blockIdx.x < kStampSlots) stamps[2 * blockIdx.x] = stamps[2 * blockIdx.x + 1];   // placeholder start, see the copiers
+        if (stamps && tid == 0 && cta < kStampSlots) stamps[2 * cta] = stamps[2 * cta + 1];   // placeholder start, see the copiers
         return;
     }
     // ---- row copy
-    const int c = static_cast<int>(blockIdx.x) - bd.n;
+    const int c = cta - bd.n;
     int b = 0;
     while (b + 1 < bd.n && c >= tp.cta0[b + 1]) ++b;
     const int part = c - tp.cta0[b], nparts = tp.cta0[b + 1] - tp.cta0[b];
@@ -83,7 +88,7 @@ select_copy_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__
         });
     asm volatile("griddepcontrol.wait;" ::: "memory");      // keeps the chain of dependencies whole: the kernel after
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // this one may rely on the one before it being complete
-    if (stamps && tid == 0 && blockIdx.x < kStampSlots) stamps[2 * blockIdx.x] = global_ns();
+    if (stamps && tid == 0 && cta < kStampSlots) stamps[2 * cta] = global_ns();
 
     {
         const int n_rows = s.n_out - (text_early ? s.n_txt : 0);
@@ -101,9 +106,9 @@ select_copy_kernel(const __grid_constant__ BatchDesc bd, const __grid_constant__
             return true;
         });
     }
-    if (stamps && blockIdx.x < kStampSlots) {
+    if (stamps && cta < kStampSlots) {
         __syncthreads();
-        if (tid == 0) stamps[2 * blockIdx.x + 1] = global_ns();
+        if (tid == 0) stamps[2 * cta + 1] = global_ns();
     }
 }
 
@@ -146,14 +151,28 @@ cudaError_t launch_select_copy(const BatchDesc& bd, const GateParams& gp, const 
     TailPlan tp;
     int next = 0;
     if (ca.seg_begin[3] > 0) {
-        // copying CTAs per sample in proportion to its kept rows, at least one each
+        // copying CTAs per sample in proportion to its kept rows (rounded down), at least one each, and never more
+        // than `ctas` in all -- the grid must fit on the device at once, see the kernel -- unless there are more
+        // samples than that
         ctas = std::min(std::max(ctas, bd.n), 30000);
         int64_t rows = 0;
         for (int b = 0; b < bd.n; ++b) rows += bd.s[b].n_out;
+        int share[kMaxChunk];
+        int total = 0;
+        for (int b = 0; b < bd.n; ++b) {
+            share[b] = static_cast<int>(std::max<int64_t>(1, rows > 0 ? static_cast<int64_t>(ctas) * bd.s[b].n_out / rows : 1));
+            total += share[b];
+        }
+        while (total > ctas) {                               // the minimum of one pushed it over: take from the largest
+            int big = 0;
+            for (int b = 1; b < bd.n; ++b) big = share[b] > share[big] ? b : big;
+            if (share[big] <= 1) break;
+            --share[big];
+            --total;
+        }
         for (int b = 0; b < bd.n; ++b) {
             tp.cta0[b] = static_cast<int16_t>(next);
-            const int64_t share = rows > 0 ? (static_cast<int64_t>(ctas) * bd.s[b].n_out + rows / 2) / rows : 1;
-            next += static_cast<int>(std::max<int64_t>(1, share));
+            next += share[b];
         }
     } else {
         for (int b = 0; b < bd.n; ++b) tp.cta0[b] = 0;       // nothing to copy: selection only
