@@ -308,3 +308,19 @@ def test_patch_step_leaves_the_bytes_behind_its_outputs_alone():
     for t in (out.out_hidden, out.out_k, out.out_v):
         assert bool((t[n:].view(torch.int16) == 0x5A5A).all()), "rows past the total were written"
     ctx.close()
+
+
+@pytest.mark.parametrize("batch,n_txt,n_patch", [(1, (20,), (1000,)), (2, (48, 9), (600, 515)), (32, (7, 12, 5), (24, 40, 33))])
+def test_patch_step_in_one_tail_kernel_at_the_edges_of_its_shapes(batch, n_txt, n_patch):
+    # the serial step's single tail kernel: more patches than the selecting CTA has threads (several patches per
+    # thread, two key tiles per scoring CTA), more than 32 text queries, and as many samples as one launch carries
+    wl = W.patch_workload(57, batch=batch, D=128, H=2, d=64, n_txt=n_txt, n_patch=n_patch, steps=2)
+    ctx = mvla.context_for(wl)
+    states = [oracle.PatchState(s.n_2d) for s in wl.samples]
+    checked = total = 0
+    for step in (0, 1):
+        _, c, n = run_patch_step(ctx, wl, step, states)
+        checked += c
+        total += n
+    assert checked >= 0.8 * total
+    ctx.close()
